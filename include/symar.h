@@ -1,0 +1,208 @@
+/*
+ * symar -- barrier-free symmetric-memory AllReduce(sum) for one B200.
+ *
+ * C ABI of libsymar.so.  Plain pointers and sizes only; no C++ or framework
+ * types cross this boundary.  Unless a parameter says "host", a pointer is a
+ * DEVICE address.
+ *
+ * Model.  P ranks are emulated on one GPU as disjoint CTA partitions of ONE
+ * kernel launch.  They share a symmetric heap (paper Sec. II-B, "symmetric
+ * objects ... identical type, size, and layout on each processing element"):
+ * P equally laid-out rank segments, so that the object at byte offset `o` of
+ * rank q is always  base + q * stride + o.  Ranks meet only through that memory,
+ * exactly as GPUs of one NVLink domain meet through load/store-accessible
+ * peer memory.  Synchronisation never uses a grid-wide or memory barrier
+ * (Sec. III-B): one-shot and two-shot use per-peer sequence-number flags, the
+ * LL protocol carries a flag inside every 8-byte store (Sec. IV "LL").
+ *
+ * Every function returns an int status: SYMAR_OK (0) or a negative error.
+ * Nothing throws, aborts or prints.  All device-side waits are bounded; a wait
+ * that gives up records SYMAR_ERR_TIMEOUT in the heap's status word (read it
+ * with symheap_status) and the kernel returns normally.
+ *
+ * Threading: a heap may be used from one host thread and one stream at a time
+ * (the per-CTA epoch counters live in the heap).  Calls on one stream are
+ * ordered by the stream.
+ */
+#ifndef SYMAR_H
+#define SYMAR_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct symheap symheap_t;            /* opaque; owned by the library */
+
+typedef enum { SYMAR_F32 = 0, SYMAR_BF16 = 1 } symar_dtype_t;
+
+typedef enum {
+    SYMAR_AUTO    = 0,   /* per-size selector (Sec. VIII: "select the best-performing
+                            low-latency algorithm based on the collected empirical results") */
+    SYMAR_ONESHOT = 1,   /* Sec. III-A.1, pull form: every rank reads all P inputs           */
+    SYMAR_TWOSHOT = 2,   /* Sec. III-A.2: reduce-scatter, then all-gather with flag handoff  */
+    SYMAR_LL      = 3    /* Sec. IV "LL" + Sec. V example: one-shot push, data+flag stores   */
+} symar_algo_t;
+
+enum {
+    SYMAR_OK              =  0,
+    SYMAR_ERR_INVAL       = -1,   /* bad argument (null, misaligned, out of range, overlap)  */
+    SYMAR_ERR_NOMEM       = -2,   /* device or host allocation failed / caller memory too small */
+    SYMAR_ERR_CUDA        = -3,   /* a CUDA runtime call failed; see symar_last_cuda_error()  */
+    SYMAR_ERR_TIMEOUT     = -4,   /* a bounded device-side wait gave up (via symheap_status)  */
+    SYMAR_ERR_UNSUPPORTED = -5    /* valid request this build cannot serve                    */
+};
+
+/* Compile-time shape of a rank segment (all sizes in bytes unless noted). */
+enum {
+    SYMAR_MAX_RANKS     = 8,      /* P must be 1, 2, 4 or 8                                   */
+    SYMAR_MAX_CTAS      = 160,    /* CTA slots per rank that own flags and an epoch counter   */
+    SYMAR_LL_SLOTS      = 64,     /* CTA slots per rank that own an LL scratch region          */
+    SYMAR_LL_SLOT_VECS  = 1024,   /* 16-byte payload vectors per LL slot, sender and iteration */
+    SYMAR_ALIGN         = 256     /* alignment of every region of a segment                    */
+};
+
+typedef struct {
+    int      P;                   /* ranks                                                     */
+    size_t   bytes_per_rank;      /* user region as requested                                   */
+    size_t   user_bytes;          /* user region as laid out (rounded up to SYMAR_ALIGN)        */
+    size_t   ll_scratch_bytes;    /* per rank: 2 parities x slots x P senders x vecs x 32 B     */
+    size_t   flag_bytes;          /* per rank: ready + done flag arrays + epoch counters        */
+    size_t   stride;              /* bytes from one rank segment to the next                    */
+    size_t   total_bytes;         /* control block + P segments                                 */
+    void    *base;                /* device address of rank 0's segment                         */
+} symheap_info_t;
+
+/* ---- symmetric heap (Sec. II-B symmetric heap; Sec. IV scratch buffer; Sec. V
+ *      ncclLLBuffer layout "address = f(epoch, CTA index)") ------------------- */
+
+/* Bytes of device memory a heap of P ranks with `bytes_per_rank` of user region
+ * needs (control block + P segments of user region, LL scratch, flags).
+ * Returns 0 if P is not 1, 2, 4 or 8.                                          */
+size_t symheap_required_bytes(int P, size_t bytes_per_rank);
+
+/* Create a heap in memory the library allocates with cudaMalloc on the current
+ * device and frees in symheap_destroy.  Scratch and flags are zeroed
+ * (synchronously).  *heap is written only on success.                          */
+int symheap_create(symheap_t **heap, int P, size_t bytes_per_rank);
+
+/* As symheap_create, in caller-owned device memory (e.g. a torch tensor) of at
+ * least symheap_required_bytes() bytes, 256-byte aligned.  The caller keeps the
+ * memory alive until symheap_destroy and frees it afterwards.                  */
+int symheap_create_on(symheap_t **heap, int P, size_t bytes_per_rank,
+                      void *device_mem, size_t device_bytes);
+
+int symheap_destroy(symheap_t *heap);
+
+/* Layout of the heap (host struct filled in). */
+int symheap_info(const symheap_t *heap, symheap_info_t *info);
+
+/* Device address of byte `offset` of rank `rank`'s user region; NULL when out
+ * of range.  symheap_rank_ptr(h, 0, o) is the "symmetric address" that
+ * allreduce() takes for the object at offset o of every rank.                  */
+void *symheap_rank_ptr(const symheap_t *heap, int rank, size_t offset);
+
+/* Zero scratch, flags, epoch counters and the status word (asynchronous on
+ * `cuda_stream`).  Needed only after a SYMAR_ERR_TIMEOUT left them inconsistent. */
+int symheap_reset(symheap_t *heap, void *cuda_stream);
+
+/* Synchronous read of the device status word: *code is SYMAR_OK or
+ * SYMAR_ERR_TIMEOUT; on timeout *rank / *peer / *cta say which emulated rank's
+ * CTA slot gave up waiting for which peer.  Any out pointer may be NULL.       */
+int symheap_status(symheap_t *heap, int *code, int *rank, int *peer, int *cta);
+
+/* ---- the collective ---------------------------------------------------------
+ *
+ * out[r][i] = narrow( ((x_0[i] + x_1[i]) + ... ) + x_{P-1}[i] )   for every rank r,
+ * x_q = widen(in[q]), sum in IEEE binary32 in rank order 0..P-1 (the deterministic
+ * one-/two-shot rows of Table I; accumulator type per Sec. V recvReduce), bf16
+ * narrowed once with round-to-nearest-even.  All three algorithms give the same
+ * bits.
+ *
+ * in, out : symmetric addresses -- device pointers into RANK 0's user region
+ *           (symheap_rank_ptr(heap, 0, off)); rank q's buffer is the same offset
+ *           in its own segment.  16-byte aligned.  Out-of-place only (Sec. VII
+ *           measures out-of-place): the byte ranges must not overlap.
+ * count   : elements PER RANK.  0 is a no-op.  Any count is accepted; a ragged
+ *           tail is handled inside the kernels.
+ * algo    : SYMAR_AUTO picks by table lookup (no timing at call time).  A named
+ *           algorithm is never silently replaced.
+ * cuda_stream : cudaStream_t (NULL = legacy default stream).  The call enqueues
+ *           exactly one kernel and returns; it may be captured in a CUDA graph.
+ * Errors  : SYMAR_ERR_INVAL for a bad pointer/alignment/range/overlap/dtype/algo;
+ *           SYMAR_ERR_CUDA if the launch failed.                                */
+int allreduce(symheap_t *heap, const void *in, void *out, size_t count,
+              symar_dtype_t dtype, symar_algo_t algo, void *cuda_stream);
+
+/* The same collective for HOST buffers (end-to-end path): copies row q of
+ * host_in ([P][count] elements, row-major, host memory, ideally pinned) to rank
+ * q's `in`, runs allreduce(), copies every rank's `out` to row r of host_out
+ * ([P][count]).  All copies and the kernel are enqueued on `cuda_stream`; the
+ * host buffers must stay valid until the stream has drained.                   */
+int allreduce_host(symheap_t *heap, const void *host_in, void *host_out,
+                   const void *in, void *out, size_t count,
+                   symar_dtype_t dtype, symar_algo_t algo, void *cuda_stream);
+
+/* ---- selector (Sec. VIII kernel selection; Sec. IX: selection is empirical) --
+ *
+ * Times every algorithm and launch shape over a power-of-two grid of message
+ * sizes (16 B ... min(bytes_per_rank / 2, 64 MiB) per rank) on an internal
+ * stream, and fills the (P, dtype) table that SYMAR_AUTO and the default launch
+ * shapes consult.  Synchronous; takes seconds.  OVERWRITES the user region of
+ * every rank.  Before it is called, built-in default thresholds apply.         */
+int allreduce_autotune(symheap_t *heap, symar_dtype_t dtype);
+
+/* What the last allreduce() on this heap launched (for reporting). */
+int symar_last_choice(const symheap_t *heap, symar_algo_t *algo,
+                      int *ctas_per_rank, int *threads);
+
+/* What SYMAR_AUTO would launch for a message of `count` elements. */
+int symar_query_choice(symheap_t *heap, size_t count, symar_dtype_t dtype,
+                       symar_algo_t *algo, int *ctas_per_rank, int *threads);
+
+/* One row of the table allreduce_autotune() filled: for messages of 2^log2_bytes
+ * bytes per rank, the best launch shape found for `algo` and its measured time
+ * per call in microseconds (host double).  SYMAR_ERR_INVAL if not tuned.       */
+int symar_tuned_entry(const symheap_t *heap, symar_dtype_t dtype, int log2_bytes,
+                      symar_algo_t algo, int *ctas_per_rank, int *threads, double *host_us);
+
+/* Force the launch shape of one algorithm (0 = back to table/default).  The
+ * library still clamps P * ctas_per_rank to what is co-resident on the device:
+ * CTAs of different ranks wait for one another, so all must be resident.       */
+int symar_set_launch(symheap_t *heap, symar_algo_t algo, int ctas_per_rank, int threads);
+
+/* Upper bound of any device-side wait, in microseconds (default 2 000 000). */
+int symar_set_spin_limit_us(symheap_t *heap, unsigned int microseconds);
+
+/* Test hooks; all off by default and free when off (separate kernel
+ * instantiation).  delay_max_ns > 0: every CTA first idles for a seeded
+ * pseudo-random time below delay_max_ns, to vary the interleaving of ranks.
+ * mute_rank >= 0: that rank sends no data and raises no flags, so that its
+ * peers' bounded waits run out (exercises SYMAR_ERR_TIMEOUT without a fault).  */
+int symar_debug_inject(symheap_t *heap, int mute_rank, unsigned int delay_seed,
+                       unsigned int delay_max_ns);
+
+/* Text of the last CUDA error seen by the library on this thread (host string). */
+const char *symar_last_cuda_error(void);
+
+/* ---- speed-of-light probes (Sec. VI: L_SoL = 2 L_L2_RTT + L_remote_store) ----
+ *
+ * Building blocks of the latency bound, measured on the box:
+ * symar_probe_empty     enqueues an empty kernel of the given shape (its cost
+ *                       in a stream or graph is the launch floor);
+ * symar_probe_fence     ns per __threadfence() over a dependent chain with one
+ *                       outstanding store each (the paper's L_L2_RTT estimate);
+ * symar_probe_pingpong  ns per round trip of one 4-byte flag bounced between
+ *                       two CTAs on different SMs through L2 (the one-GPU
+ *                       analogue of the paper's two-GPU ping-pong).
+ * The last two are synchronous and write host doubles.                         */
+int symar_probe_empty(int grid_x, int grid_y, int block, void *cuda_stream);
+int symar_probe_fence(int iterations, double *host_ns_per_fence);
+int symar_probe_pingpong(int iterations, double *host_ns_per_round_trip);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SYMAR_H */

@@ -1,0 +1,214 @@
+// Thread-level building blocks of the barrier-free AllReduce kernels: scoped
+// memory operations, bounded polling, element widening/narrowing and the
+// data+flag (LL) send/receive on a per-slot, double-buffered scratch region
+// (paper Sec. IV "LL", "Bidirectional Communication & Double Buffering";
+// Sec. V: send, recv, recvUnrolled, recvReduce, bcast, advanceEpoch).
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include "symar_layout.h"
+
+namespace symar {
+
+// ---- memory operations -------------------------------------------------------
+// On one device `.gpu` scope is sufficient; a multi-GPU build of the same
+// protocol would use `.sys`.
+#define SYMAR_SCOPE "gpu"
+
+__device__ __forceinline__ uint32_t ld_acquire_u32(const uint32_t *p)
+{
+    uint32_t v;
+    asm volatile("ld.acquire." SYMAR_SCOPE ".global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_release_u32(uint32_t *p, uint32_t v)
+{
+    asm volatile("st.release." SYMAR_SCOPE ".global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+__device__ __forceinline__ uint64_t ld_relaxed_u64(const uint64_t *p)
+{
+    uint64_t v;
+    asm volatile("ld.relaxed." SYMAR_SCOPE ".global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+    return v;
+}
+
+// 16-byte transfer made of two 8-byte elements.  Each 8-byte element {payload,
+// flag} is a single aligned 64-bit access, hence observed whole; the two
+// elements need not arrive together because each carries its own flag.
+struct __align__(16) U64x2 { uint64_t a, b; };
+
+__device__ __forceinline__ void st_relaxed_v2u64(void *p, uint64_t a, uint64_t b)
+{
+    asm volatile("st.relaxed." SYMAR_SCOPE ".global.v2.u64 [%0], {%1, %2};" ::"l"(p), "l"(a), "l"(b)
+                 : "memory");
+}
+__device__ __forceinline__ U64x2 ld_relaxed_v2u64(const void *p)
+{
+    U64x2 v;
+    asm volatile("ld.relaxed." SYMAR_SCOPE ".global.v2.u64 {%0, %1}, [%2];"
+                 : "=l"(v.a), "=l"(v.b)
+                 : "l"(p)
+                 : "memory");
+    return v;
+}
+
+// A rank's OWN input is written before its kernel starts and never during it:
+// read-only path, no L1 allocation.
+__device__ __forceinline__ uint4 ld_own(const void *p)
+{
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "l"(p));
+    return v;
+}
+// A PEER's input is read only after that peer's "ready" flag was acquired, so it
+// must be an ordinary (coherent) load ordered after the acquire; each byte is
+// used once per reading rank, hence no L1 allocation.
+__device__ __forceinline__ uint4 ld_peer(const void *p)
+{
+    uint4 v;
+    asm volatile("ld.global.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "l"(p)
+                 : "memory");
+    return v;
+}
+// Outputs are written once and not re-read by this kernel.
+__device__ __forceinline__ void st_output(void *p, uint4 v)
+{
+    asm volatile("st.global.cs.v4.u32 [%0], {%1, %2, %3, %4};" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z),
+                 "r"(v.w)
+                 : "memory");
+}
+
+__device__ __forceinline__ uint64_t globaltimer_ns()
+{
+    uint64_t t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
+
+// ---- bounded waiting ------------------------------------------------------------
+// Counts polls in a register; every 256th poll reads the nanosecond timer.  The
+// first reading starts the clock, so the fast path never touches the timer.
+struct Spin {
+    uint32_t n  = 0;
+    uint64_t t0 = 0;
+    __device__ __forceinline__ bool due() { return (++n & 0xffu) == 0; }
+    __device__ __forceinline__ bool expired(uint64_t limit_ns)
+    {
+        uint64_t now = globaltimer_ns();
+        if (t0 == 0) {
+            t0 = now;
+            return false;
+        }
+        return now - t0 > limit_ns;
+    }
+};
+
+// First error wins; the kernel then leaves through its normal exit.
+__device__ __noinline__ void report_timeout(uint32_t *ctl, int rank, int peer, int cta)
+{
+    if (atomicCAS(&ctl[kCtlCode], 0u, (uint32_t)SYMAR_ERR_TIMEOUT) == 0u) {
+        ctl[kCtlRank] = (uint32_t)rank;
+        ctl[kCtlPeer] = (uint32_t)peer;
+        ctl[kCtlCta]  = (uint32_t)cta;
+        __threadfence();
+    }
+}
+
+// ---- per-slot iteration counter ("epoch") ----------------------------------------
+// The counter n is 64-bit and private to one (rank, CTA slot).  The 32-bit flag
+// sent with the data is 1 + n mod (2^32 - 1): never 0 (0 = "never written"),
+// and consecutive iterations always differ in parity n & 1, also across the
+// 32-bit wrap.
+__device__ __forceinline__ uint32_t flag_of(uint64_t n) { return (uint32_t)(n % 0xffffffffull) + 1u; }
+
+// ---- element types ---------------------------------------------------------------
+struct F32 {
+    static constexpr int kEpv = 4;   // elements per 16-byte vector
+    __device__ static __forceinline__ void widen(const uint4 &v, float (&f)[kEpv])
+    {
+        f[0] = __uint_as_float(v.x);
+        f[1] = __uint_as_float(v.y);
+        f[2] = __uint_as_float(v.z);
+        f[3] = __uint_as_float(v.w);
+    }
+    __device__ static __forceinline__ uint4 narrow(const float (&f)[kEpv])
+    {
+        return make_uint4(__float_as_uint(f[0]), __float_as_uint(f[1]), __float_as_uint(f[2]),
+                          __float_as_uint(f[3]));
+    }
+};
+
+struct BF16 {
+    static constexpr int kEpv = 8;
+    __device__ static __forceinline__ void widen(const uint4 &v, float (&f)[kEpv])
+    {
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            f[2 * i]     = __uint_as_float(w[i] << 16);          // low half = even element
+            f[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);  // high half = odd element
+        }
+    }
+    __device__ static __forceinline__ uint4 narrow(const float (&f)[kEpv])
+    {
+        uint32_t w[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            __nv_bfloat162 h = __floats2bfloat162_rn(f[2 * i], f[2 * i + 1]);   // RNE
+            w[i] = *reinterpret_cast<uint32_t *>(&h);
+        }
+        return make_uint4(w[0], w[1], w[2], w[3]);
+    }
+};
+
+// Rank-ordered sum of P vectors with a binary32 accumulator that starts as the
+// rank-0 value; one narrowing at the end (recvReduce's accumulate-and-convert).
+template <typename E, int P>
+__device__ __forceinline__ uint4 reduce_in_rank_order(const uint4 (&x)[P])
+{
+    float acc[E::kEpv];
+    E::widen(x[0], acc);
+#pragma unroll
+    for (int q = 1; q < P; ++q) {
+        float t[E::kEpv];
+        E::widen(x[q], t);
+#pragma unroll
+        for (int j = 0; j < E::kEpv; ++j) acc[j] = __fadd_rn(acc[j], t[j]);
+    }
+    return E::narrow(acc);
+}
+
+// Store of output vector v; the last vector of a message may be partial.
+__device__ __forceinline__ void store_result(char *out, uint64_t v, uint4 val, uint64_t nvec,
+                                             uint32_t tail_bytes)
+{
+    if (tail_bytes != 0 && v == nvec - 1) {
+        const uint16_t *src = reinterpret_cast<const uint16_t *>(&val);
+        uint16_t *dst       = reinterpret_cast<uint16_t *>(out + v * 16);
+        for (uint32_t b = 0; b < tail_bytes / 2; ++b) dst[b] = src[b];
+    } else {
+        st_output(out + v * 16, val);
+    }
+}
+
+// ---- test hook: seeded start delay -------------------------------------------------
+__device__ __forceinline__ void debug_delay(const KArgs &a, int rank, int cta)
+{
+    if (a.dbg_delay_ns == 0) return;
+    uint32_t h = a.dbg_seed ^ (uint32_t)(rank * 0x9E3779B1u) ^ (uint32_t)(cta * 0x85EBCA77u);
+    h ^= h >> 16;
+    h *= 0x7feb352dU;
+    h ^= h >> 15;
+    h *= 0x846ca68bU;
+    h ^= h >> 16;
+    const uint64_t wait = h % a.dbg_delay_ns;
+    const uint64_t t0   = globaltimer_ns();
+    while (globaltimer_ns() - t0 < wait) { /* bounded by dbg_delay_ns */ }
+}
+
+}  // namespace symar

@@ -1,0 +1,566 @@
+// Host side of libsymar: the symmetric heap, argument checking, the per-size
+// selector with its autotuner, and the C ABI declared in include/symar.h.
+// Every step of the collective itself runs in the kernels of symar_kernels.cu;
+// there is no host or library fallback.
+#include <algorithm>
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <map>
+#include <new>
+#include <string>
+#include <tuple>
+#include <vector>
+
+#include "symar_internal.h"
+
+namespace symar {
+
+struct LaunchCfg {
+    int ctas    = 0;   // per rank; 0 = not set
+    int threads = 0;
+};
+
+constexpr int kBuckets = 40;   // bucket b holds messages of (2^(b-1), 2^b] bytes per rank
+constexpr int kAlgos   = 4;    // indexed by symar_algo_t
+
+struct Tuned {
+    bool      valid = false;
+    int       best_algo[kBuckets];
+    LaunchCfg cfg[kAlgos][kBuckets];
+    double    us[kAlgos][kBuckets];
+    int       lo_bucket = 0, hi_bucket = -1;
+};
+
+static thread_local std::string g_last_cuda_error;
+
+static int cuda_fail(cudaError_t e, const char *what)
+{
+    g_last_cuda_error = std::string(what) + ": " + cudaGetErrorString(e);
+    return SYMAR_ERR_CUDA;
+}
+#define CU(call)                                          \
+    do {                                                  \
+        cudaError_t e_ = (call);                          \
+        if (e_ != cudaSuccess) return cuda_fail(e_, #call); \
+    } while (0)
+
+}  // namespace symar
+
+using namespace symar;
+
+struct symheap {
+    int       P              = 0;
+    size_t    bytes_per_rank = 0;
+    Layout    L{};
+    char     *mem   = nullptr;   // heap base (control block)
+    bool      owns  = false;
+    char     *seg0  = nullptr;
+    uint32_t *ctl   = nullptr;
+    int       device  = 0;
+    int       num_sms = 0;
+    uint64_t  spin_ns = 2000000000ull;
+    int       dbg_mute     = -1;
+    unsigned  dbg_seed     = 0;
+    unsigned  dbg_delay_ns = 0;
+    LaunchCfg forced[kAlgos];
+    Tuned     tuned[2];
+    int       last_algo = 0, last_ctas = 0, last_threads = 0;
+    std::map<std::tuple<const void *, int>, int> resident;   // (kernel, threads) -> CTAs co-resident
+};
+
+namespace symar {
+
+static size_t elem_size(int dtype) { return dtype == SYMAR_F32 ? 4 : 2; }
+static bool   valid_P(int P) { return P == 1 || P == 2 || P == 4 || P == 8; }
+static bool   dbg_on(const symheap *h) { return h->dbg_mute >= 0 || h->dbg_delay_ns != 0; }
+
+static int bucket_of(size_t bytes)
+{
+    int b = 0;
+    while (b < kBuckets - 1 && ((size_t)1 << b) < bytes) ++b;
+    return b;
+}
+
+// CTAs of the given kernel and block size that fit on the device at once.  The
+// CTAs of different ranks wait for one another, so a grid larger than this
+// could leave a waiting CTA holding the SM that the CTA it waits for needs.
+static int max_resident(symheap *h, KernelFn fn, int threads)
+{
+    auto key = std::make_tuple((const void *)fn, threads);
+    auto it  = h->resident.find(key);
+    if (it != h->resident.end()) return it->second;
+    int per_sm = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fn, threads, 0) != cudaSuccess) per_sm = 1;
+    int n = std::max(1, per_sm) * h->num_sms;
+    h->resident[key] = n;
+    return n;
+}
+
+static int round_threads(uint64_t want)
+{
+    int t = 32;
+    while (t < (int)kMaxThreads && (uint64_t)t < want) t *= 2;
+    return t;
+}
+
+// Launch shape when neither the caller nor the tuner fixed one.
+static LaunchCfg default_cfg(const symheap *h, int algo, uint64_t nvec)
+{
+    LaunchCfg c;
+    const uint64_t work = algo == SYMAR_TWOSHOT ? (nvec + h->P - 1) / h->P : nvec;   // vectors per rank partition
+    c.threads = work >= 1024 ? 256 : round_threads(std::max<uint64_t>(work / 4, 32));
+    if (work >= (uint64_t)1 << 18) c.threads = 512;
+    uint64_t ctas = (work + c.threads - 1) / c.threads;
+    // bandwidth regime: two CTAs of 512 threads per SM over all ranks
+    const uint64_t fill = std::max(1, 2 * h->num_sms / h->P);
+    const uint64_t cap  = algo == SYMAR_LL ? (uint64_t)kLLSlots : (work >= (uint64_t)1 << 18 ? fill : 16);
+    c.ctas = (int)std::max<uint64_t>(1, std::min(ctas, cap));
+    return c;
+}
+
+static int default_algo(size_t bytes)
+{
+    if (bytes <= (32u << 10)) return SYMAR_LL;
+    if (bytes <= (256u << 10)) return SYMAR_ONESHOT;
+    return SYMAR_TWOSHOT;
+}
+
+struct Plan {
+    int       algo;
+    LaunchCfg cfg;
+    KernelFn  fn;
+    KArgs     args;
+};
+
+// Resolves algorithm and launch shape and fills the kernel arguments.
+static int make_plan(symheap *h, size_t in_off, size_t out_off, size_t count, int dtype, int algo, Plan *p)
+{
+    const size_t es    = elem_size(dtype);
+    const size_t bytes = count * es;
+    const uint64_t nvec = (bytes + 15) / 16;
+    const Tuned &tn    = h->tuned[dtype];
+    const int b        = tn.valid ? std::min(std::max(bucket_of(bytes), tn.lo_bucket), tn.hi_bucket) : 0;
+
+    if (algo == SYMAR_AUTO) algo = tn.valid ? tn.best_algo[b] : default_algo(bytes);
+
+    LaunchCfg cfg = default_cfg(h, algo, nvec);
+    if (tn.valid && tn.cfg[algo][b].ctas > 0) cfg = tn.cfg[algo][b];
+    if (h->forced[algo].ctas > 0) cfg.ctas = h->forced[algo].ctas;
+    if (h->forced[algo].threads > 0) cfg.threads = h->forced[algo].threads;
+
+    cfg.threads = std::min<int>(std::max(32, (cfg.threads + 31) / 32 * 32), (int)kMaxThreads);
+    KernelFn fn = kernel_for(algo, dtype, h->P, dbg_on(h));
+    if (!fn) return SYMAR_ERR_INVAL;
+    const int cap_slots = algo == SYMAR_LL ? kLLSlots : kMaxCtas;
+    const int cap_res   = std::max(1, max_resident(h, fn, cfg.threads) / h->P);
+    cfg.ctas = std::max(1, std::min({cfg.ctas, cap_slots, cap_res}));
+
+    KArgs &a = p->args;
+    std::memset(&a, 0, sizeof a);
+    a.seg0       = h->seg0;
+    a.stride     = h->L.stride;
+    a.in_off     = in_off;
+    a.out_off    = out_off;
+    a.count      = count;
+    a.nvec       = nvec;
+    a.ll_off     = h->L.ll_off;
+    a.ready_off  = h->L.ready_off;
+    a.done_off   = h->L.done_off;
+    a.epoch_off  = h->L.epoch_off;
+    a.ctl        = h->ctl;
+    a.spin_ns    = h->spin_ns;
+    a.tail_bytes = (uint32_t)(bytes % 16);
+    a.dbg_mute   = h->dbg_mute;
+    a.dbg_seed   = h->dbg_seed;
+    a.dbg_delay_ns = h->dbg_delay_ns;
+    if (algo == SYMAR_LL) {
+        // every CTA takes `cv` vectors per iteration; iterations alternate sub-buffers
+        const uint64_t per_cta = (nvec + cfg.ctas - 1) / cfg.ctas;
+        a.cv    = (uint32_t)std::max<uint64_t>(1, std::min<uint64_t>(per_cta, kLLSlotVecs));
+        a.iters = (uint32_t)((nvec + (uint64_t)a.cv * cfg.ctas - 1) / ((uint64_t)a.cv * cfg.ctas));
+    }
+    p->algo = algo;
+    p->cfg  = cfg;
+    p->fn   = fn;
+    return SYMAR_OK;
+}
+
+static int check_buffers(const symheap *h, const void *in, const void *out, size_t count, int dtype,
+                         size_t *in_off, size_t *out_off)
+{
+    if (!h || !in || !out) return SYMAR_ERR_INVAL;
+    if (dtype != SYMAR_F32 && dtype != SYMAR_BF16) return SYMAR_ERR_INVAL;
+    const char *pi = (const char *)in, *po = (const char *)out;
+    if (pi < h->seg0 || po < h->seg0) return SYMAR_ERR_INVAL;
+    const size_t io = pi - h->seg0, oo = po - h->seg0;
+    const size_t bytes = count * elem_size(dtype);
+    if (count != 0 && bytes / count != elem_size(dtype)) return SYMAR_ERR_INVAL;   // overflow
+    if ((io | oo) & 15) return SYMAR_ERR_INVAL;
+    if (io > h->bytes_per_rank || bytes > h->bytes_per_rank - io) return SYMAR_ERR_INVAL;
+    if (oo > h->bytes_per_rank || bytes > h->bytes_per_rank - oo) return SYMAR_ERR_INVAL;
+    if (bytes != 0 && io < oo + bytes && oo < io + bytes) return SYMAR_ERR_INVAL;    // out-of-place only
+    *in_off  = io;
+    *out_off = oo;
+    return SYMAR_OK;
+}
+
+static int run(symheap *h, const void *in, void *out, size_t count, int dtype, int algo, cudaStream_t s)
+{
+    size_t io = 0, oo = 0;
+    int rc = check_buffers(h, in, out, count, dtype, &io, &oo);
+    if (rc != SYMAR_OK) return rc;
+    if (algo < SYMAR_AUTO || algo > SYMAR_LL) return SYMAR_ERR_INVAL;
+    if (count == 0) return SYMAR_OK;
+    Plan p;
+    rc = make_plan(h, io, oo, count, dtype, algo, &p);
+    if (rc != SYMAR_OK) return rc;
+    cudaError_t e = launch_kernel(p.fn, h->P, p.cfg.ctas, p.cfg.threads, p.args, s);
+    if (e != cudaSuccess) return cuda_fail(e, "kernel launch");
+    h->last_algo    = p.algo;
+    h->last_ctas    = p.cfg.ctas;
+    h->last_threads = p.cfg.threads;
+    return SYMAR_OK;
+}
+
+// ---- autotuner ---------------------------------------------------------------------
+
+// Median per-call time (us) of K back-to-back calls captured in one graph.
+static int time_calls(symheap *h, cudaStream_t s, size_t count, int dtype, int algo, int K, int reps,
+                      double *us_out)
+{
+    const size_t bytes = count * elem_size(dtype);
+    const void *in = h->seg0;
+    void *out      = h->seg0 + round_up(bytes, 256);
+    cudaGraph_t graph;
+    cudaGraphExec_t exec;
+    CU(cudaStreamBeginCapture(s, cudaStreamCaptureModeThreadLocal));
+    int rc = SYMAR_OK;
+    for (int k = 0; k < K && rc == SYMAR_OK; ++k) rc = run(h, in, out, count, dtype, algo, s);
+    cudaError_t ce = cudaStreamEndCapture(s, &graph);
+    if (rc != SYMAR_OK) {
+        if (ce == cudaSuccess) cudaGraphDestroy(graph);
+        return rc;
+    }
+    if (ce != cudaSuccess) return cuda_fail(ce, "cudaStreamEndCapture");
+    ce = cudaGraphInstantiate(&exec, graph, 0);
+    if (ce != cudaSuccess) {
+        cudaGraphDestroy(graph);
+        return cuda_fail(ce, "cudaGraphInstantiate");
+    }
+    cudaEvent_t e0, e1;
+    cudaEventCreate(&e0);
+    cudaEventCreate(&e1);
+    std::vector<float> ms(reps);
+    cudaGraphLaunch(exec, s);   // warm
+    for (int i = 0; i < reps; ++i) {
+        cudaEventRecord(e0, s);
+        cudaGraphLaunch(exec, s);
+        cudaEventRecord(e1, s);
+        cudaEventSynchronize(e1);
+        cudaEventElapsedTime(&ms[i], e0, e1);
+    }
+    cudaEventDestroy(e0);
+    cudaEventDestroy(e1);
+    cudaGraphExecDestroy(exec);
+    cudaGraphDestroy(graph);
+    ce = cudaGetLastError();
+    if (ce != cudaSuccess) return cuda_fail(ce, "autotune timing");
+    std::sort(ms.begin(), ms.end());
+    *us_out = (double)ms[reps / 2] * 1000.0 / K;
+    return SYMAR_OK;
+}
+
+static int autotune(symheap *h, int dtype)
+{
+    static const int kThreads[] = {64, 128, 256, 512};
+    static const int kCtas[]    = {1, 2, 4, 8, 12, 16, 18, 24, 32, 37, 48, 64, 74};
+    const size_t es = elem_size(dtype);
+    Tuned tn;
+    size_t max_bytes = std::min<size_t>(h->bytes_per_rank / 2 / 256 * 256, (size_t)64 << 20);
+    if (max_bytes < 16) return SYMAR_ERR_INVAL;
+    tn.lo_bucket = 4;
+    tn.hi_bucket = 4;
+    while (tn.hi_bucket + 1 < kBuckets && ((size_t)1 << (tn.hi_bucket + 1)) <= max_bytes) ++tn.hi_bucket;
+
+    cudaStream_t s;
+    CU(cudaStreamCreateWithFlags(&s, cudaStreamNonBlocking));
+    LaunchCfg saved[kAlgos];
+    for (int a = 0; a < kAlgos; ++a) saved[a] = h->forced[a];
+    const Tuned saved_tuned = h->tuned[dtype];
+    h->tuned[dtype].valid = false;
+
+    int rc = SYMAR_OK;
+    for (int b = tn.lo_bucket; b <= tn.hi_bucket && rc == SYMAR_OK; ++b) {
+        const size_t bytes  = (size_t)1 << b;
+        const size_t count  = bytes / es;
+        const uint64_t nvec = bytes / 16;
+        const int K    = bytes <= (1u << 20) ? 24 : (bytes <= (16u << 20) ? 6 : 2);
+        const int reps = 7;
+        double best_us = 1e30;
+        tn.best_algo[b] = SYMAR_ONESHOT;
+        for (int algo = SYMAR_ONESHOT; algo <= SYMAR_LL && rc == SYMAR_OK; ++algo) {
+            tn.us[algo][b]  = 1e30;
+            tn.cfg[algo][b] = LaunchCfg{};
+            if (algo == SYMAR_LL && bytes > (4u << 20)) continue;      // 2 P M scratch traffic: hopeless there
+            if (algo == SYMAR_ONESHOT && bytes > (32u << 20)) continue;
+            const uint64_t work = algo == SYMAR_TWOSHOT ? (nvec + h->P - 1) / h->P : nvec;
+            for (int T : kThreads) {
+                for (int C : kCtas) {
+                    // skip shapes with far more threads than vectors, except the smallest
+                    if ((uint64_t)C * T > 2 * work && !(C == 1 && T == 64)) continue;
+                    // and shapes that would leave each thread hundreds of vectors
+                    if (work / ((uint64_t)C * T) > 4096) continue;
+                    h->forced[algo] = LaunchCfg{C, T};
+                    Plan p;
+                    if (make_plan(h, 0, round_up(bytes, 256), count, dtype, algo, &p) != SYMAR_OK) continue;
+                    if (p.cfg.ctas != C || p.cfg.threads != T) continue;   // clamped: a duplicate of another shape
+                    double us = 0;
+                    rc = time_calls(h, s, count, dtype, algo, K, reps, &us);
+                    if (rc != SYMAR_OK) break;
+                    if (us < tn.us[algo][b]) {
+                        tn.us[algo][b]  = us;
+                        tn.cfg[algo][b] = LaunchCfg{C, T};
+                    }
+                }
+                if (rc != SYMAR_OK) break;
+            }
+            h->forced[algo] = saved[algo];
+            if (tn.us[algo][b] < best_us) {
+                best_us         = tn.us[algo][b];
+                tn.best_algo[b] = algo;
+            }
+        }
+    }
+    for (int a = 0; a < kAlgos; ++a) h->forced[a] = saved[a];
+    cudaStreamSynchronize(s);
+    cudaStreamDestroy(s);
+    if (rc != SYMAR_OK) {
+        h->tuned[dtype] = saved_tuned;
+        return rc;
+    }
+    tn.valid        = true;
+    h->tuned[dtype] = tn;
+    return SYMAR_OK;
+}
+
+static int create_common(symheap_t **heap, int P, size_t bytes_per_rank, void *mem, size_t mem_bytes, bool owns)
+{
+    Layout L = make_layout(P, bytes_per_rank);
+    if (mem_bytes < L.total) return SYMAR_ERR_NOMEM;
+    if (((uintptr_t)mem & (kAlign - 1)) != 0) return SYMAR_ERR_INVAL;
+    symheap *h = new (std::nothrow) symheap;
+    if (!h) return SYMAR_ERR_NOMEM;
+    h->P = P;
+    h->bytes_per_rank = bytes_per_rank;
+    h->L    = L;
+    h->mem  = (char *)mem;
+    h->owns = owns;
+    h->seg0 = h->mem + kCtlBytes;
+    h->ctl  = (uint32_t *)h->mem;
+    cudaError_t e = cudaGetDevice(&h->device);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&h->num_sms, cudaDevAttrMultiProcessorCount, h->device);
+    if (e == cudaSuccess) e = cudaMemset(h->mem, 0, kCtlBytes);
+    for (int q = 0; q < P && e == cudaSuccess; ++q)
+        e = cudaMemset(h->seg0 + (size_t)q * L.stride + L.ll_off, 0, L.seg_bytes - L.ll_off);
+    // Load every kernel this heap can launch now, so that a first call made
+    // during stream capture does not trigger lazy module loading there.
+    for (int algo = SYMAR_ONESHOT; algo <= SYMAR_LL && e == cudaSuccess; ++algo)
+        for (int dt = SYMAR_F32; dt <= SYMAR_BF16 && e == cudaSuccess; ++dt) {
+            cudaFuncAttributes attr;
+            e = cudaFuncGetAttributes(&attr, kernel_for(algo, dt, P, false));
+        }
+    if (e == cudaSuccess) e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) {
+        delete h;
+        return cuda_fail(e, "heap initialisation");
+    }
+    *heap = h;
+    return SYMAR_OK;
+}
+
+}  // namespace symar
+
+// ---- C ABI ---------------------------------------------------------------------------
+
+extern "C" {
+
+size_t symheap_required_bytes(int P, size_t bytes_per_rank)
+{
+    if (!valid_P(P)) return 0;
+    return make_layout(P, bytes_per_rank).total;
+}
+
+int symheap_create(symheap_t **heap, int P, size_t bytes_per_rank)
+{
+    if (!heap || !valid_P(P) || bytes_per_rank == 0) return SYMAR_ERR_INVAL;
+    const size_t total = make_layout(P, bytes_per_rank).total;
+    void *mem = nullptr;
+    cudaError_t e = cudaMalloc(&mem, total);
+    if (e == cudaErrorMemoryAllocation) {
+        cudaGetLastError();
+        return SYMAR_ERR_NOMEM;
+    }
+    if (e != cudaSuccess) return cuda_fail(e, "cudaMalloc");
+    int rc = create_common(heap, P, bytes_per_rank, mem, total, true);
+    if (rc != SYMAR_OK) cudaFree(mem);
+    return rc;
+}
+
+int symheap_create_on(symheap_t **heap, int P, size_t bytes_per_rank, void *device_mem, size_t device_bytes)
+{
+    if (!heap || !valid_P(P) || bytes_per_rank == 0 || !device_mem) return SYMAR_ERR_INVAL;
+    return create_common(heap, P, bytes_per_rank, device_mem, device_bytes, false);
+}
+
+int symheap_destroy(symheap_t *heap)
+{
+    if (!heap) return SYMAR_ERR_INVAL;
+    int rc = SYMAR_OK;
+    if (heap->owns) {
+        cudaError_t e = cudaFree(heap->mem);
+        if (e != cudaSuccess) rc = cuda_fail(e, "cudaFree");
+    }
+    delete heap;
+    return rc;
+}
+
+int symheap_info(const symheap_t *heap, symheap_info_t *info)
+{
+    if (!heap || !info) return SYMAR_ERR_INVAL;
+    info->P                = heap->P;
+    info->bytes_per_rank   = heap->bytes_per_rank;
+    info->user_bytes       = heap->L.user_bytes;
+    info->ll_scratch_bytes = heap->L.ll_bytes;
+    info->flag_bytes       = heap->L.seg_bytes - heap->L.ready_off;
+    info->stride           = heap->L.stride;
+    info->total_bytes      = heap->L.total;
+    info->base             = heap->seg0;
+    return SYMAR_OK;
+}
+
+void *symheap_rank_ptr(const symheap_t *heap, int rank, size_t offset)
+{
+    if (!heap || rank < 0 || rank >= heap->P || offset >= heap->L.user_bytes) return nullptr;
+    return heap->seg0 + (size_t)rank * heap->L.stride + offset;
+}
+
+int symheap_reset(symheap_t *heap, void *cuda_stream)
+{
+    if (!heap) return SYMAR_ERR_INVAL;
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    CU(cudaMemsetAsync(heap->mem, 0, kCtlBytes, s));
+    for (int q = 0; q < heap->P; ++q)
+        CU(cudaMemsetAsync(heap->seg0 + (size_t)q * heap->L.stride + heap->L.ll_off, 0,
+                           heap->L.seg_bytes - heap->L.ll_off, s));
+    return SYMAR_OK;
+}
+
+int symheap_status(symheap_t *heap, int *code, int *rank, int *peer, int *cta)
+{
+    if (!heap) return SYMAR_ERR_INVAL;
+    uint32_t w[4] = {0, 0, 0, 0};
+    CU(cudaMemcpy(w, heap->ctl, sizeof w, cudaMemcpyDeviceToHost));
+    if (code) *code = (int)w[kCtlCode];
+    if (rank) *rank = (int)w[kCtlRank];
+    if (peer) *peer = (int)w[kCtlPeer];
+    if (cta) *cta = (int)w[kCtlCta];
+    return SYMAR_OK;
+}
+
+int allreduce(symheap_t *heap, const void *in, void *out, size_t count, symar_dtype_t dtype,
+              symar_algo_t algo, void *cuda_stream)
+{
+    return run(heap, in, out, count, (int)dtype, (int)algo, (cudaStream_t)cuda_stream);
+}
+
+int allreduce_host(symheap_t *heap, const void *host_in, void *host_out, const void *in, void *out,
+                   size_t count, symar_dtype_t dtype, symar_algo_t algo, void *cuda_stream)
+{
+    size_t io = 0, oo = 0;
+    int rc = check_buffers(heap, in, out, count, (int)dtype, &io, &oo);
+    if (rc != SYMAR_OK) return rc;
+    if (!host_in || !host_out) return SYMAR_ERR_INVAL;
+    if (count == 0) return SYMAR_OK;
+    cudaStream_t s     = (cudaStream_t)cuda_stream;
+    const size_t bytes = count * elem_size((int)dtype);
+    for (int q = 0; q < heap->P; ++q)
+        CU(cudaMemcpyAsync(heap->seg0 + (size_t)q * heap->L.stride + io, (const char *)host_in + (size_t)q * bytes,
+                           bytes, cudaMemcpyHostToDevice, s));
+    rc = run(heap, in, out, count, (int)dtype, (int)algo, s);
+    if (rc != SYMAR_OK) return rc;
+    for (int r = 0; r < heap->P; ++r)
+        CU(cudaMemcpyAsync((char *)host_out + (size_t)r * bytes, heap->seg0 + (size_t)r * heap->L.stride + oo,
+                           bytes, cudaMemcpyDeviceToHost, s));
+    return SYMAR_OK;
+}
+
+int allreduce_autotune(symheap_t *heap, symar_dtype_t dtype)
+{
+    if (!heap || (dtype != SYMAR_F32 && dtype != SYMAR_BF16)) return SYMAR_ERR_INVAL;
+    return autotune(heap, (int)dtype);
+}
+
+int symar_last_choice(const symheap_t *heap, symar_algo_t *algo, int *ctas_per_rank, int *threads)
+{
+    if (!heap) return SYMAR_ERR_INVAL;
+    if (algo) *algo = (symar_algo_t)heap->last_algo;
+    if (ctas_per_rank) *ctas_per_rank = heap->last_ctas;
+    if (threads) *threads = heap->last_threads;
+    return SYMAR_OK;
+}
+
+int symar_query_choice(symheap_t *heap, size_t count, symar_dtype_t dtype, symar_algo_t *algo,
+                       int *ctas_per_rank, int *threads)
+{
+    if (!heap || (dtype != SYMAR_F32 && dtype != SYMAR_BF16)) return SYMAR_ERR_INVAL;
+    Plan p;
+    int rc = make_plan(heap, 0, 0, count, (int)dtype, algo ? (int)*algo : SYMAR_AUTO, &p);
+    if (rc != SYMAR_OK) return rc;
+    if (algo) *algo = (symar_algo_t)p.algo;
+    if (ctas_per_rank) *ctas_per_rank = p.cfg.ctas;
+    if (threads) *threads = p.cfg.threads;
+    return SYMAR_OK;
+}
+
+int symar_tuned_entry(const symheap_t *heap, symar_dtype_t dtype, int log2_bytes, symar_algo_t algo,
+                      int *ctas_per_rank, int *threads, double *host_us)
+{
+    if (!heap || (dtype != SYMAR_F32 && dtype != SYMAR_BF16)) return SYMAR_ERR_INVAL;
+    const Tuned &tn = heap->tuned[(int)dtype];
+    if (!tn.valid || log2_bytes < tn.lo_bucket || log2_bytes > tn.hi_bucket) return SYMAR_ERR_INVAL;
+    if (algo < SYMAR_ONESHOT || algo > SYMAR_LL) return SYMAR_ERR_INVAL;
+    if (ctas_per_rank) *ctas_per_rank = tn.cfg[algo][log2_bytes].ctas;
+    if (threads) *threads = tn.cfg[algo][log2_bytes].threads;
+    if (host_us) *host_us = tn.us[algo][log2_bytes];
+    return SYMAR_OK;
+}
+
+int symar_set_launch(symheap_t *heap, symar_algo_t algo, int ctas_per_rank, int threads)
+{
+    if (!heap || algo < SYMAR_ONESHOT || algo > SYMAR_LL) return SYMAR_ERR_INVAL;
+    if (ctas_per_rank < 0 || threads < 0 || threads > (int)kMaxThreads) return SYMAR_ERR_INVAL;
+    heap->forced[algo] = LaunchCfg{ctas_per_rank, threads};
+    return SYMAR_OK;
+}
+
+int symar_set_spin_limit_us(symheap_t *heap, unsigned int microseconds)
+{
+    if (!heap || microseconds == 0) return SYMAR_ERR_INVAL;
+    heap->spin_ns = (uint64_t)microseconds * 1000ull;
+    return SYMAR_OK;
+}
+
+int symar_debug_inject(symheap_t *heap, int mute_rank, unsigned int delay_seed, unsigned int delay_max_ns)
+{
+    if (!heap || mute_rank >= heap->P) return SYMAR_ERR_INVAL;
+    if (delay_max_ns > 1000000u) return SYMAR_ERR_INVAL;   // keep test delays below a millisecond
+    heap->dbg_mute     = mute_rank < 0 ? -1 : mute_rank;
+    heap->dbg_seed     = delay_seed;
+    heap->dbg_delay_ns = delay_max_ns;
+    return SYMAR_OK;
+}
+
+const char *symar_last_cuda_error(void) { return g_last_cuda_error.c_str(); }
+
+}  // extern "C"

@@ -1,0 +1,19 @@
+// Declarations shared by the translation units of libsymar (host side).
+#pragma once
+#include <cuda_runtime.h>
+
+#include "symar_layout.h"
+
+namespace symar {
+
+using KernelFn = void (*)(const KArgs);
+
+// Kernel instantiation for (algorithm, element type, ranks); dbg selects the
+// variant that honours the test hooks.  nullptr for unsupported combinations.
+KernelFn kernel_for(int algo, int dtype, int P, bool dbg);
+
+// grid = (ctas_per_rank, P), block = threads; returns the launch status.
+cudaError_t launch_kernel(KernelFn fn, int P, int ctas_per_rank, int threads, const KArgs &args,
+                          cudaStream_t stream);
+
+}  // namespace symar

@@ -1,0 +1,135 @@
+// Speed-of-light probes (paper Sec. VI): the pieces of the latency lower bound,
+// measured on the device the collective runs on.
+//
+//   L_L2_RTT        one __threadfence() with one store outstanding: the SM must
+//                   wait until the store has reached L2, the point of coherence;
+//   flag round trip one 4-byte value bounced between two CTAs on two SMs through
+//                   L2 -- the one-GPU counterpart of the paper's two-GPU
+//                   ping-pong, L_pingpong = 2 L_L2_RTT + 2 L_remote_store;
+//   launch floor    an empty kernel of the same grid and block as the collective.
+//
+// Every spin is bounded; a probe that gives up returns SYMAR_ERR_TIMEOUT.
+#include <cuda_runtime.h>
+
+#include "symar.h"
+
+namespace {
+
+__device__ __forceinline__ unsigned long long timer_ns()
+{
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
+__device__ __forceinline__ unsigned ld_relaxed(const unsigned *p)
+{
+    unsigned v;
+    asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_relaxed(unsigned *p, unsigned v)
+{
+    asm volatile("st.relaxed.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+
+__global__ void empty_kernel() {}
+
+// out[0] = elapsed ns over `iters` store+fence pairs
+__global__ void fence_kernel(unsigned *scratch, int iters, unsigned long long *out)
+{
+    unsigned long long t0 = timer_ns();
+    for (int i = 0; i < iters; ++i) {
+        st_relaxed(scratch, (unsigned)i);
+        __threadfence();
+    }
+    unsigned long long t1 = timer_ns();
+    out[0] = t1 - t0;
+}
+
+constexpr unsigned kSpinLimit = 1u << 22;   // polls; far above any real round trip
+
+// flags[0] is written by block 0 and watched by block 1; flags[32] the reverse
+// (separate 128-byte lines).  out[0] = ns, out[1] = 1 on timeout, out[2..3] = SM ids.
+__global__ void pingpong_kernel(unsigned *flags, int iters, unsigned long long *out)
+{
+    unsigned smid;
+    asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
+    unsigned *mine   = flags + (blockIdx.x == 0 ? 0 : 32);
+    unsigned *theirs = flags + (blockIdx.x == 0 ? 32 : 0);
+    out[2 + blockIdx.x] = smid;
+    bool dead = false;
+    unsigned long long t0 = 0;
+    if (blockIdx.x == 0) {
+        // one untimed exchange first, so that both blocks are known to be running
+        for (int i = 1; i <= iters + 1 && !dead; ++i) {
+            if (i == 2) t0 = timer_ns();
+            st_relaxed(mine, (unsigned)i);
+            unsigned n = 0;
+            while (ld_relaxed(theirs) != (unsigned)i)
+                if (++n > kSpinLimit) { dead = true; break; }
+        }
+        out[0] = timer_ns() - t0;
+    } else {
+        for (int i = 1; i <= iters + 1 && !dead; ++i) {
+            unsigned n = 0;
+            while (ld_relaxed(theirs) != (unsigned)i)
+                if (++n > kSpinLimit) { dead = true; break; }
+            st_relaxed(mine, (unsigned)i);
+        }
+    }
+    if (dead) out[1] = 1;
+}
+
+int sync_and_fetch(unsigned long long *dev, unsigned long long *host, int n)
+{
+    if (cudaDeviceSynchronize() != cudaSuccess) return SYMAR_ERR_CUDA;
+    if (cudaMemcpy(host, dev, n * sizeof(unsigned long long), cudaMemcpyDeviceToHost) != cudaSuccess)
+        return SYMAR_ERR_CUDA;
+    return SYMAR_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int symar_probe_empty(int grid_x, int grid_y, int block, void *cuda_stream)
+{
+    if (grid_x < 1 || grid_y < 1 || block < 1 || block > 1024) return SYMAR_ERR_INVAL;
+    empty_kernel<<<dim3(grid_x, grid_y, 1), block, 0, (cudaStream_t)cuda_stream>>>();
+    return cudaGetLastError() == cudaSuccess ? SYMAR_OK : SYMAR_ERR_CUDA;
+}
+
+int symar_probe_fence(int iterations, double *host_ns_per_fence)
+{
+    if (iterations < 1 || !host_ns_per_fence) return SYMAR_ERR_INVAL;
+    unsigned char *buf = nullptr;
+    if (cudaMalloc(&buf, 512) != cudaSuccess) return SYMAR_ERR_NOMEM;
+    cudaMemset(buf, 0, 512);
+    unsigned long long h[4] = {0, 0, 0, 0};
+    fence_kernel<<<1, 1>>>((unsigned *)buf, 16, (unsigned long long *)(buf + 256));   // warm
+    fence_kernel<<<1, 1>>>((unsigned *)buf, iterations, (unsigned long long *)(buf + 256));
+    int rc = sync_and_fetch((unsigned long long *)(buf + 256), h, 1);
+    cudaFree(buf);
+    if (rc != SYMAR_OK) return rc;
+    *host_ns_per_fence = (double)h[0] / iterations;
+    return SYMAR_OK;
+}
+
+int symar_probe_pingpong(int iterations, double *host_ns_per_round_trip)
+{
+    if (iterations < 1 || !host_ns_per_round_trip) return SYMAR_ERR_INVAL;
+    unsigned char *buf = nullptr;
+    if (cudaMalloc(&buf, 1024) != cudaSuccess) return SYMAR_ERR_NOMEM;
+    cudaMemset(buf, 0, 1024);
+    unsigned long long h[4] = {0, 0, 0, 0};
+    pingpong_kernel<<<2, 1>>>((unsigned *)buf, iterations, (unsigned long long *)(buf + 512));
+    int rc = sync_and_fetch((unsigned long long *)(buf + 512), h, 4);
+    cudaFree(buf);
+    if (rc != SYMAR_OK) return rc;
+    if (h[1] != 0) return SYMAR_ERR_TIMEOUT;
+    if (h[2] == h[3]) return SYMAR_ERR_UNSUPPORTED;   // both blocks landed on one SM: not an L2 round trip
+    *host_ns_per_round_trip = (double)h[0] / iterations;
+    return SYMAR_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,265 @@
+"""ctypes binding of libsymar.so: argument marshalling only.
+
+Function names and argument order follow ``include/symar.h``.  Every step of
+the collective runs in the library's CUDA kernels; if the library is missing
+or fails to load this module raises -- there is no fallback of any kind.
+"""
+from __future__ import annotations
+
+import ctypes
+from ctypes import POINTER, byref, c_char_p, c_double, c_int, c_size_t, c_uint, c_void_p
+from pathlib import Path
+
+_PKG = Path(__file__).resolve().parent
+LIB_PATH = _PKG / "libsymar.so"
+
+F32, BF16 = 0, 1
+AUTO, ONESHOT, TWOSHOT, LL = 0, 1, 2, 3
+ALGO_NAMES = {AUTO: "auto", ONESHOT: "oneshot", TWOSHOT: "twoshot", LL: "ll"}
+DTYPE_NAMES = {F32: "f32", BF16: "bf16"}
+DTYPE_SIZE = {F32: 4, BF16: 2}
+
+OK, ERR_INVAL, ERR_NOMEM, ERR_CUDA, ERR_TIMEOUT, ERR_UNSUPPORTED = 0, -1, -2, -3, -4, -5
+_ERR_NAMES = {
+    ERR_INVAL: "SYMAR_ERR_INVAL", ERR_NOMEM: "SYMAR_ERR_NOMEM", ERR_CUDA: "SYMAR_ERR_CUDA",
+    ERR_TIMEOUT: "SYMAR_ERR_TIMEOUT", ERR_UNSUPPORTED: "SYMAR_ERR_UNSUPPORTED",
+}
+
+MAX_RANKS, MAX_CTAS, LL_SLOTS, LL_SLOT_VECS, ALIGN = 8, 160, 64, 1024, 256
+
+# every symbol include/symar.h declares: (name, restype, argtypes)
+SIGNATURES = [
+    ("symheap_required_bytes", c_size_t, [c_int, c_size_t]),
+    ("symheap_create", c_int, [POINTER(c_void_p), c_int, c_size_t]),
+    ("symheap_create_on", c_int, [POINTER(c_void_p), c_int, c_size_t, c_void_p, c_size_t]),
+    ("symheap_destroy", c_int, [c_void_p]),
+    ("symheap_info", c_int, [c_void_p, c_void_p]),
+    ("symheap_rank_ptr", c_void_p, [c_void_p, c_int, c_size_t]),
+    ("symheap_reset", c_int, [c_void_p, c_void_p]),
+    ("symheap_status", c_int, [c_void_p, POINTER(c_int), POINTER(c_int), POINTER(c_int), POINTER(c_int)]),
+    ("allreduce", c_int, [c_void_p, c_void_p, c_void_p, c_size_t, c_int, c_int, c_void_p]),
+    ("allreduce_host", c_int, [c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, c_int, c_int,
+                               c_void_p]),
+    ("allreduce_autotune", c_int, [c_void_p, c_int]),
+    ("symar_last_choice", c_int, [c_void_p, POINTER(c_int), POINTER(c_int), POINTER(c_int)]),
+    ("symar_query_choice", c_int, [c_void_p, c_size_t, c_int, POINTER(c_int), POINTER(c_int), POINTER(c_int)]),
+    ("symar_tuned_entry", c_int, [c_void_p, c_int, c_int, c_int, POINTER(c_int), POINTER(c_int),
+                                  POINTER(c_double)]),
+    ("symar_set_launch", c_int, [c_void_p, c_int, c_int, c_int]),
+    ("symar_set_spin_limit_us", c_int, [c_void_p, c_uint]),
+    ("symar_debug_inject", c_int, [c_void_p, c_int, c_uint, c_uint]),
+    ("symar_last_cuda_error", c_char_p, []),
+    ("symar_probe_empty", c_int, [c_int, c_int, c_int, c_void_p]),
+    ("symar_probe_fence", c_int, [c_int, POINTER(c_double)]),
+    ("symar_probe_pingpong", c_int, [c_int, POINTER(c_double)]),
+]
+
+
+class SymarError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        detail = ""
+        if code == ERR_CUDA and _lib is not None:
+            detail = ": " + (_lib.symar_last_cuda_error() or b"").decode()
+        super().__init__(f"{where} -> {_ERR_NAMES.get(code, code)}{detail}")
+
+
+class HeapInfo(ctypes.Structure):
+    _fields_ = [
+        ("P", c_int), ("bytes_per_rank", c_size_t), ("user_bytes", c_size_t),
+        ("ll_scratch_bytes", c_size_t), ("flag_bytes", c_size_t), ("stride", c_size_t),
+        ("total_bytes", c_size_t), ("base", c_void_p),
+    ]
+
+
+_lib = None
+
+
+def load() -> ctypes.CDLL:
+    """dlopen the library and declare every signature.  Raises if it is absent."""
+    global _lib
+    if _lib is None:
+        if not LIB_PATH.exists():
+            raise ImportError(
+                f"{LIB_PATH} not found: build it with `python -m paper_2607_16100_b200.build` "
+                "(there is no non-CUDA path)")
+        lib = ctypes.CDLL(str(LIB_PATH))
+        for name, res, args in SIGNATURES:
+            fn = getattr(lib, name)
+            fn.restype = res
+            fn.argtypes = args
+        _lib = lib
+    return _lib
+
+
+def _ck(rc: int, where: str) -> None:
+    if rc != OK:
+        raise SymarError(rc, where)
+
+
+def required_bytes(P: int, bytes_per_rank: int) -> int:
+    return int(load().symheap_required_bytes(P, bytes_per_rank))
+
+
+class SymHeap:
+    """Owner of one ``symheap_t``.  ``device_mem`` (an int address) + ``device_bytes``
+    place the heap in caller memory (``symheap_create_on``); otherwise the library
+    allocates (``symheap_create``)."""
+
+    def __init__(self, P: int, bytes_per_rank: int, device_mem: int | None = None,
+                 device_bytes: int = 0, keepalive=None):
+        self._lib = load()
+        self._h = c_void_p()
+        self._keepalive = keepalive
+        if device_mem is None:
+            _ck(self._lib.symheap_create(byref(self._h), P, bytes_per_rank), "symheap_create")
+        else:
+            _ck(self._lib.symheap_create_on(byref(self._h), P, bytes_per_rank, device_mem, device_bytes),
+                "symheap_create_on")
+        self.P = P
+        self.bytes_per_rank = bytes_per_rank
+        i = self.info()
+        self.base = int(i.base)
+        self.stride = int(i.stride)
+
+    @classmethod
+    def on_torch(cls, P: int, bytes_per_rank: int, device="cuda:0") -> "SymHeap":
+        """Heap in a torch uint8 tensor (PyTorch provides the device memory)."""
+        import torch
+        n = required_bytes(P, bytes_per_rank)
+        buf = torch.empty(n + ALIGN, dtype=torch.uint8, device=device)
+        addr = (buf.data_ptr() + ALIGN - 1) // ALIGN * ALIGN
+        with torch.cuda.device(buf.device):
+            return cls(P, bytes_per_rank, addr, n, keepalive=buf)
+
+    # -- lifetime --
+    def destroy(self) -> None:
+        if self._h:
+            self._lib.symheap_destroy(self._h)
+            self._h = c_void_p()
+            self._keepalive = None
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass
+
+    # -- layout --
+    def info(self) -> HeapInfo:
+        i = HeapInfo()
+        _ck(self._lib.symheap_info(self._h, byref(i)), "symheap_info")
+        return i
+
+    def rank_ptr(self, rank: int, offset: int = 0) -> int:
+        p = self._lib.symheap_rank_ptr(self._h, rank, offset)
+        if not p:
+            raise SymarError(ERR_INVAL, "symheap_rank_ptr")
+        return int(p)
+
+    def reset(self, stream: int = 0) -> None:
+        _ck(self._lib.symheap_reset(self._h, stream), "symheap_reset")
+
+    def status(self):
+        code, rank, peer, cta = c_int(), c_int(), c_int(), c_int()
+        _ck(self._lib.symheap_status(self._h, byref(code), byref(rank), byref(peer), byref(cta)),
+            "symheap_status")
+        return code.value, rank.value, peer.value, cta.value
+
+    # -- the collective --
+    def allreduce_rc(self, in_off: int, out_off: int, count: int, dtype: int, algo: int = AUTO,
+                     stream: int = 0) -> int:
+        """Raw status code; offsets are turned into rank-0 symmetric addresses."""
+        base = self.base
+        return int(self._lib.allreduce(self._h, base + in_off, base + out_off, count, dtype, algo, stream))
+
+    def allreduce(self, in_off: int, out_off: int, count: int, dtype: int, algo: int = AUTO,
+                  stream: int = 0) -> None:
+        _ck(self.allreduce_rc(in_off, out_off, count, dtype, algo, stream), "allreduce")
+
+    def allreduce_ptr(self, in_ptr: int, out_ptr: int, count: int, dtype: int, algo: int = AUTO,
+                      stream: int = 0) -> None:
+        _ck(self._lib.allreduce(self._h, in_ptr, out_ptr, count, dtype, algo, stream), "allreduce")
+
+    def allreduce_host(self, host_in: int, host_out: int, in_off: int, out_off: int, count: int,
+                       dtype: int, algo: int = AUTO, stream: int = 0) -> None:
+        base = self.base
+        _ck(self._lib.allreduce_host(self._h, host_in, host_out, base + in_off, base + out_off, count,
+                                     dtype, algo, stream), "allreduce_host")
+
+    # -- data movement helpers for heaps that live in a torch tensor --
+    def _bytes_view(self, rank: int, offset: int, nbytes: int):
+        if self._keepalive is None:
+            raise RuntimeError("heap does not live in a torch tensor (use SymHeap.on_torch)")
+        if not (0 <= rank < self.P) or offset < 0 or offset + nbytes > self.bytes_per_rank:
+            raise SymarError(ERR_INVAL, "rank/offset/size outside the user region")
+        start = self.base + rank * self.stride + offset - self._keepalive.data_ptr()
+        return self._keepalive[start:start + nbytes]
+
+    def write_rank(self, rank: int, offset: int, array) -> None:
+        """Copy a host numpy array into rank ``rank``'s user region at ``offset``."""
+        import numpy as np
+        import torch
+        a = np.ascontiguousarray(array)
+        src = torch.from_numpy(a.view(np.uint8).reshape(-1))
+        self._bytes_view(rank, offset, a.nbytes).copy_(src, non_blocking=False)
+
+    def read_rank(self, rank: int, offset: int, count: int, np_dtype):
+        """Copy ``count`` elements of ``np_dtype`` from rank ``rank``'s user region to the host."""
+        import numpy as np
+        n = count * np.dtype(np_dtype).itemsize
+        return self._bytes_view(rank, offset, n).cpu().numpy().view(np_dtype).copy()
+
+    def fill_user(self, byte: int) -> None:
+        """Fill every rank's user region with one byte value (poison before a test)."""
+        for q in range(self.P):
+            self._bytes_view(q, 0, self.bytes_per_rank).fill_(byte)
+
+    # -- selector --
+    def autotune(self, dtype: int) -> None:
+        _ck(self._lib.allreduce_autotune(self._h, dtype), "allreduce_autotune")
+
+    def last_choice(self):
+        a, c, t = c_int(), c_int(), c_int()
+        _ck(self._lib.symar_last_choice(self._h, byref(a), byref(c), byref(t)), "symar_last_choice")
+        return a.value, c.value, t.value
+
+    def query_choice(self, count: int, dtype: int, algo: int = AUTO):
+        a, c, t = c_int(algo), c_int(), c_int()
+        _ck(self._lib.symar_query_choice(self._h, count, dtype, byref(a), byref(c), byref(t)),
+            "symar_query_choice")
+        return a.value, c.value, t.value
+
+    def tuned_entry(self, dtype: int, log2_bytes: int, algo: int):
+        c, t, us = c_int(), c_int(), c_double()
+        rc = self._lib.symar_tuned_entry(self._h, dtype, log2_bytes, algo, byref(c), byref(t), byref(us))
+        if rc != OK:
+            return None
+        return c.value, t.value, us.value
+
+    def set_launch(self, algo: int, ctas_per_rank: int, threads: int) -> None:
+        _ck(self._lib.symar_set_launch(self._h, algo, ctas_per_rank, threads), "symar_set_launch")
+
+    def set_spin_limit_us(self, us: int) -> None:
+        _ck(self._lib.symar_set_spin_limit_us(self._h, us), "symar_set_spin_limit_us")
+
+    def debug_inject(self, mute_rank: int = -1, delay_seed: int = 0, delay_max_ns: int = 0) -> None:
+        _ck(self._lib.symar_debug_inject(self._h, mute_rank, delay_seed, delay_max_ns), "symar_debug_inject")
+
+
+# -- probes --
+
+def probe_empty(grid_x: int, grid_y: int, block: int, stream: int = 0) -> None:
+    _ck(load().symar_probe_empty(grid_x, grid_y, block, stream), "symar_probe_empty")
+
+
+def probe_fence(iterations: int = 20000) -> float:
+    v = c_double()
+    _ck(load().symar_probe_fence(iterations, byref(v)), "symar_probe_fence")
+    return v.value
+
+
+def probe_pingpong(iterations: int = 20000) -> float:
+    v = c_double()
+    _ck(load().symar_probe_pingpong(iterations, byref(v)), "symar_probe_pingpong")
+    return v.value

@@ -1,0 +1,311 @@
+"""GPU parity: the CUDA AllReduce (through the C ABI) against the CPU oracle,
+element by element and bit for bit, on the same seeded inputs."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import allreduce_oracle as O
+from paper_2607_16100_b200 import symar, synth
+
+pytestmark = pytest.mark.gpu
+
+ALGOS = [symar.ONESHOT, symar.TWOSHOT, symar.LL]
+NP_DT = {symar.F32: np.float32, symar.BF16: np.uint16}
+DT = {"f32": symar.F32, "bf16": symar.BF16}
+USER = 8 << 20          # user region per rank of the shared test heaps
+
+
+@pytest.fixture(scope="module")
+def heaps():
+    hs = {P: symar.SymHeap.on_torch(P, USER) for P in (1, 2, 4, 8)}
+    yield hs
+    torch.cuda.synchronize()
+    for h in hs.values():
+        h.destroy()
+
+
+def run(h, x, dtype, algo, in_off=0, out_off=None, stream=0, poison=True):
+    """Upload x[P, count], run one allreduce, return out[P, count]."""
+    P, count = x.shape
+    nbytes = x.nbytes // P
+    if out_off is None:
+        out_off = (in_off + nbytes + 255) // 256 * 256
+    if poison:
+        for q in range(P):
+            h.write_rank(q, out_off, np.full(nbytes + 64, 0xA5, dtype=np.uint8))
+    for q in range(P):
+        h.write_rank(q, in_off, x[q])
+    h.allreduce(in_off, out_off, count, dtype, algo, stream)
+    torch.cuda.synchronize()
+    code = h.status()[0]
+    assert code == symar.OK, f"device status {h.status()}"
+    out = np.stack([h.read_rank(q, out_off, count, NP_DT[dtype]) for q in range(P)])
+    if poison:   # nothing may be written past the end of the message
+        for q in range(P):
+            guard = h.read_rank(q, out_off + nbytes, 64, np.uint8)
+            assert np.all(guard == 0xA5), f"rank {q}: wrote past the end of the output"
+    return out
+
+
+def assert_bits(got, want, what=""):
+    if got.dtype == np.float32:
+        got, want = got.view(np.uint32), want.view(np.uint32)
+    bad = np.argwhere(got != want)
+    assert bad.size == 0, f"{what}: {len(bad)} mismatches, first at [rank, i] = {bad[0]}: " \
+                          f"got {got[tuple(bad[0])]:#x} want {want[tuple(bad[0])]:#x}"
+
+
+# ---- tier 1: small shapes, every algorithm x dtype x P x ragged counts -------------
+
+@pytest.mark.parametrize("count", [1, 3, 7, 8, 9, 31, 1023, 1024, 1025, 8191, 70001])
+@pytest.mark.parametrize("P", [1, 2, 4, 8])
+@pytest.mark.parametrize("dtype,dist", [("f32", "uniform"), ("bf16", "normal")])
+@pytest.mark.parametrize("algo", ALGOS)
+def test_small_shapes(heaps, algo, dtype, dist, P, count):
+    x = synth.make_inputs(dist, dtype, P, count, seed=1000 + count)
+    got = run(heaps[P], x, DT[dtype], algo)
+    assert_bits(got, O.allreduce(x), f"algo={algo} {dtype} P={P} count={count}")
+
+
+@pytest.mark.parametrize("algo", ALGOS)
+def test_nonzero_offsets(heaps, algo):
+    h = heaps[4]
+    x = synth.make_inputs("normal", "bf16", 4, 5000, seed=77)
+    got = run(h, x, symar.BF16, algo, in_off=4096 + 16, out_off=1 << 20)
+    assert_bits(got, O.allreduce(x))
+    # output placed BEFORE the input
+    got = run(h, x, symar.BF16, algo, in_off=2 << 20, out_off=48)
+    assert_bits(got, O.allreduce(x))
+
+
+# ---- special values -----------------------------------------------------------------
+
+@pytest.mark.parametrize("algo", ALGOS)
+def test_special_values_f32(heaps, algo):
+    sp = np.array([0.0, -0.0, 1e-45, -1e-45, 1.17549435e-38, np.inf, -np.inf, 3.4e38, -3.4e38, 1.0, 1e8, -1e8],
+                  dtype=np.float32)
+    rng = np.random.default_rng(3)
+    x = sp[rng.integers(0, len(sp), size=(4, 4096))]
+    got = run(heaps[4], x, symar.F32, algo)
+    want = O.allreduce(x)
+    nan = np.isnan(want)
+    assert np.array_equal(np.isnan(got), nan)
+    assert_bits(np.where(nan, np.float32(0), got), np.where(nan, np.float32(0), want))
+
+
+@pytest.mark.parametrize("algo", ALGOS)
+def test_special_values_bf16(heaps, algo):
+    sp = np.array([0x0000, 0x8000, 0x0001, 0x8001, 0x0080, 0x7F80, 0xFF80, 0x7F7F, 0xFF7F, 0x3F80, 0x3B80,
+                   0x4380, 0x7FC0], dtype=np.uint16)
+    rng = np.random.default_rng(4)
+    x = sp[rng.integers(0, len(sp), size=(8, 4096))]
+    got = run(heaps[8], x, symar.BF16, algo)
+    want = O.allreduce(x)
+    is_nan = lambda h: ((h & 0x7F80) == 0x7F80) & ((h & 0x007F) != 0)
+    assert np.array_equal(is_nan(got), is_nan(want))
+    keep = ~is_nan(want)
+    assert_bits(np.where(keep, got, 0), np.where(keep, want, 0))
+
+
+def test_hand_case_order_pin_on_gpu(heaps):
+    # rank order 0..3: (1 + 1e8) - 1e8 + 0 = 0 in binary32; a reordered sum gives 1
+    x = np.array([[1.0] * 8, [1e8] * 8, [-1e8] * 8, [0.0] * 8], dtype=np.float32)
+    for algo in ALGOS:
+        got = run(heaps[4], x, symar.F32, algo)
+        assert np.all(got == 0.0)
+    got = run(heaps[4], x[::-1].copy(), symar.F32, symar.LL)
+    assert np.all(got == 1.0)
+
+
+# ---- launch shapes, multi-iteration LL ----------------------------------------------
+
+@pytest.mark.parametrize("ctas,threads", [(1, 32), (1, 512), (3, 64), (7, 96), (16, 256), (64, 128)])
+@pytest.mark.parametrize("algo", ALGOS)
+def test_forced_launch_shapes(heaps, algo, ctas, threads):
+    h = heaps[8]
+    x = synth.make_inputs("normal", "bf16", 8, 40009, seed=ctas * 1000 + threads)
+    h.set_launch(algo, ctas, threads)
+    try:
+        got = run(h, x, symar.BF16, algo)
+        a, c, t = h.last_choice()
+        assert (a, c, t) == (algo, ctas, threads)
+    finally:
+        h.set_launch(algo, 0, 0)
+    assert_bits(got, O.allreduce(x))
+
+
+def test_ll_many_iterations_alternate_subbuffers(heaps):
+    # one CTA per rank, 1024 vectors per iteration: 300000 fp32 -> 75000 vectors -> 74 iterations
+    h = heaps[4]
+    x = synth.make_inputs("uniform", "f32", 4, 300000, seed=5)
+    h.set_launch(symar.LL, 1, 256)
+    try:
+        got = run(h, x, symar.F32, symar.LL)
+    finally:
+        h.set_launch(symar.LL, 0, 0)
+    assert_bits(got, O.allreduce(x))
+
+
+# ---- determinism, algorithm equality, interleaving stress ---------------------------
+
+def test_algorithms_agree_and_repeat(heaps):
+    h = heaps[8]
+    x = synth.make_inputs("normal", "bf16", 8, 8192, seed=synth.seed_for_config(2))
+    want = O.allreduce(x)
+    for rep in range(40):
+        for algo in ALGOS:
+            assert_bits(run(h, x, symar.BF16, algo, poison=(rep == 0)), want, f"rep {rep} algo {algo}")
+
+
+@pytest.mark.parametrize("algo", ALGOS)
+def test_seeded_start_delays_do_not_change_results(heaps, algo):
+    h = heaps[8]
+    x = synth.make_inputs("uniform", "f32", 8, 20000, seed=31)
+    want = O.allreduce(x)
+    try:
+        for seed in range(12):
+            h.debug_inject(-1, seed + 1, 20000)          # every CTA starts up to 20 us late
+            assert_bits(run(h, x, symar.F32, algo, poison=False), want, f"delay seed {seed}")
+    finally:
+        h.debug_inject(-1, 0, 0)
+
+
+def test_mixed_algorithms_and_shapes_share_flags_safely(heaps):
+    # successive calls with different algorithms, sizes and grids reuse the same
+    # flag words and scratch; per-slot counters must keep every flag value fresh
+    h = heaps[8]
+    rng = np.random.default_rng(12)
+    for i in range(60):
+        algo = ALGOS[int(rng.integers(0, 3))]
+        count = int(rng.integers(1, 30000))
+        dtype = ("f32", "bf16")[int(rng.integers(0, 2))]
+        h.set_launch(algo, int(rng.integers(1, 40)), int(rng.choice([32, 64, 128, 256, 512])))
+        x = synth.make_inputs("normal", dtype, 8, count, seed=500 + i)
+        try:
+            got = run(h, x, DT[dtype], algo, poison=False)
+        finally:
+            h.set_launch(algo, 0, 0)
+        assert_bits(got, O.allreduce(x), f"step {i} algo {algo} count {count}")
+
+
+# ---- CUDA graph capture and replay ----------------------------------------------------
+
+def test_graph_capture_replays(heaps):
+    h = heaps[8]
+    count, calls = 8192 * 4, 6
+    nbytes = count * 2
+    xs = [synth.make_inputs("normal", "bf16", 8, count, seed=synth.seed_for_config(5), call=k)
+          for k in range(calls)]
+    for k, x in enumerate(xs):
+        for q in range(8):
+            h.write_rank(q, k * nbytes, x[q])
+    out0 = 4 << 20
+    s = torch.cuda.Stream()
+    g = torch.cuda.CUDAGraph()
+    torch.cuda.synchronize()
+    with torch.cuda.graph(g, stream=s):
+        for k in range(calls):
+            algo = ALGOS[k % 3]
+            h.allreduce(k * nbytes, out0 + k * nbytes, count, symar.BF16, algo, s.cuda_stream)
+    for rep in range(4):
+        for q in range(8):
+            h.write_rank(q, out0, np.zeros(calls * nbytes, dtype=np.uint8))
+        g.replay()
+        torch.cuda.synchronize()
+        assert h.status()[0] == symar.OK
+        for k, x in enumerate(xs):
+            want = O.allreduce(x)
+            got = np.stack([h.read_rank(q, out0 + k * nbytes, count, np.uint16) for q in range(8)])
+            assert_bits(got, want, f"replay {rep} call {k}")
+
+
+# ---- AUTO, autotune -----------------------------------------------------------------------
+
+def test_auto_default_and_after_autotune():
+    h = symar.SymHeap.on_torch(4, 1 << 20)
+    try:
+        x = synth.make_inputs("int_pm8", "f32", 4, 1024, seed=synth.seed_for_config(1))
+        got = run(h, x, symar.F32, symar.AUTO)
+        assert_bits(got, O.allreduce(x))
+        assert h.last_choice()[0] in ALGOS
+        h.autotune(symar.F32)
+        for count in (4, 1024, 70000, 131072):
+            x = synth.make_inputs("uniform", "f32", 4, count, seed=count)
+            got = run(h, x, symar.F32, symar.AUTO, poison=False)
+            assert_bits(got, O.allreduce(x))
+            a, c, t = h.last_choice()
+            assert (a, c, t) == h.query_choice(count, symar.F32)
+        row = h.tuned_entry(symar.F32, 14, symar.LL)
+        assert row is not None and row[0] >= 1 and row[2] > 0
+    finally:
+        torch.cuda.synchronize()
+        h.destroy()
+
+
+# ---- errors --------------------------------------------------------------------------------
+
+def test_argument_errors(heaps):
+    h = heaps[4]
+    rc = h.allreduce_rc
+    assert rc(0, 4096, 0, symar.F32, symar.LL) == symar.OK                       # count 0: no-op
+    assert rc(8, 4096, 16, symar.F32, symar.LL) == symar.ERR_INVAL               # misaligned in
+    assert rc(0, 4100, 16, symar.F32, symar.LL) == symar.ERR_INVAL               # misaligned out
+    assert rc(0, 32, 16, symar.F32, symar.LL) == symar.ERR_INVAL                 # overlap
+    assert rc(0, 0, 16, symar.F32, symar.LL) == symar.ERR_INVAL                  # in place
+    assert rc(0, USER - 16, 16, symar.F32, symar.LL) == symar.ERR_INVAL          # runs off the region
+    assert rc(USER, 0, 4, symar.F32, symar.LL) == symar.ERR_INVAL
+    assert rc(0, 4096, 16, 7, symar.LL) == symar.ERR_INVAL                       # dtype
+    assert rc(0, 4096, 16, symar.F32, 9) == symar.ERR_INVAL                      # algo
+    assert rc(0, 4096, 1 << 62, symar.F32, symar.LL) == symar.ERR_INVAL          # size overflow
+    assert h.status()[0] == symar.OK
+    with pytest.raises(symar.SymarError):
+        h.rank_ptr(4, 0)
+    with pytest.raises(symar.SymarError):
+        symar.SymHeap(3, 4096)
+
+
+@pytest.mark.parametrize("algo", ALGOS)
+def test_bounded_wait_reports_timeout_and_heap_recovers(algo):
+    # Rank 2 stays silent (host-requested test hook): its peers' waits run out
+    # after the 2 ms limit, the kernel returns, the status word names the peer.
+    h = symar.SymHeap.on_torch(4, 1 << 20)
+    try:
+        x = synth.make_inputs("normal", "bf16", 4, 4096, seed=8)
+        for q in range(4):
+            h.write_rank(q, 0, x[q])
+        h.set_spin_limit_us(2000)
+        h.debug_inject(2, 0, 0)
+        h.allreduce(0, 65536, 4096, symar.BF16, algo)
+        torch.cuda.synchronize()
+        code, rank, peer, cta = h.status()
+        assert code == symar.ERR_TIMEOUT
+        assert peer == 2 and rank != 2
+        # recovery: clear the hook, reset flags/scratch/status, run again
+        h.debug_inject(-1, 0, 0)
+        h.reset()
+        got = run(h, x, symar.BF16, algo)
+        assert_bits(got, O.allreduce(x))
+    finally:
+        torch.cuda.synchronize()
+        h.destroy()
+
+
+def test_host_buffer_entry_point(heaps):
+    h = heaps[8]
+    count = 50000
+    x = synth.make_inputs("uniform", "f32", 8, count, seed=91)
+    hin = torch.from_numpy(x).pin_memory()
+    hout = torch.empty_like(hin).pin_memory()
+    h.allreduce_host(hin.data_ptr(), hout.data_ptr(), 0, 1 << 20, count, symar.F32, symar.AUTO)
+    torch.cuda.synchronize()
+    assert_bits(hout.numpy(), O.allreduce(x))
+
+
+def test_library_owned_heap():
+    h = symar.SymHeap(2, 1 << 16)
+    try:
+        info = h.info()
+        assert info.P == 2 and info.total_bytes == symar.required_bytes(2, 1 << 16)
+        assert h.rank_ptr(1, 0) - h.rank_ptr(0, 0) == info.stride
+    finally:
+        h.destroy()
