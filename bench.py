@@ -1,0 +1,497 @@
+#!/usr/bin/env python
+"""Benchmark of the barrier-free symmetric-memory AllReduce on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+One JSON line on stdout (rank 0).  A "step" is one AllReduce of the bandwidth
+workload: P = 8 emulated ranks, fp32, 64 Mi elements (256 MiB) per rank,
+inputs U(-1, 1), two-shot algorithm.  `value` is algorithmic bytes (every input
+byte read once + every output byte written once = 2 P M) per second with the
+inputs resident in HBM.  The latency half of the metric (P = 8, bf16, 16 KiB per
+rank, p50 against the speed-of-light bound measured in the same process), the
+16 KiB..1 MiB sweep with the selector's choice and the 160-call decode-step
+graph ride along in the same line under `latency_16KB`, `sweep`, `decode_trace`.
+
+N > 1 runs N independent replicas (one process and one heap per GPU; the path
+itself is a single-GPU emulation and has no exchange between GPUs).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+from pathlib import Path
+
+import numpy as np
+
+ROOT = Path(__file__).resolve().parent
+sys.path.insert(0, str(ROOT))
+
+METRIC = "p50 AllReduce latency µs @16KB vs SoL; HBM GB/s @256MB (8 emulated ranks)"
+L2_BYTES = 126 << 20
+
+
+def peaks():
+    p = ROOT / "MEASURED_PEAKS.json"
+    if p.exists():
+        d = json.loads(p.read_text())
+        return float(d["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+    return 6650.0, "fallback (6.65 TB/s, earlier measurement on this pool)"
+
+
+# ---------------------------------------------------------------------------------
+# clocks: nvidia-smi sampled in the background during a timed region
+# ---------------------------------------------------------------------------------
+class ClockSampler:
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", str(self.gpu)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.t = threading.Thread(target=self._pump, daemon=True)
+            self.t.start()
+        except Exception:
+            self.proc = None
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.lines.append((time.time(), line.strip()))
+
+    def stop(self, t_begin: float, t_end: float):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=2)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        rows = [l for (t, l) in self.lines if t_begin <= t <= t_end + 0.2] or [l for (_, l) in self.lines]
+        for l in rows:
+            f = [x.strip() for x in l.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1]))
+                mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"),
+                                 f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None,
+                "sm_max_mhz": float(max(mx)) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ---------------------------------------------------------------------------------
+# reference arm: the CPU oracle on the host cores
+# ---------------------------------------------------------------------------------
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import allreduce_oracle as O
+    from paper_2607_16100_b200 import synth
+    w = synth.WORKLOADS["c4"]
+    P = w["P"]
+    sample = 8 << 20                      # elements per rank per step: 1/8 of the workload
+    x = synth.make_inputs(w["dist"], w["dtype"], P, sample, w["seed"])
+    team = 1
+    for _ in range(max(1, args.warmup)):
+        _, team = O.allreduce_timed_team(x, threads=0)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        O.allreduce_timed_team(x, threads=0)
+    dt = time.perf_counter() - t0
+    algbytes = 2 * P * sample * 4
+    gbs = algbytes * args.steps / dt / 1e9
+    desc = f"{sample} of {w['count']} elements per rank per step (1/8 of the workload), all host cores"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": gbs, "unit": "GB/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": "c4: P=8 emulated ranks, fp32, 64Mi elements (256 MiB) per rank, U(-1,1)",
+                   "sample": desc},
+        "cpu_baseline": {"value": gbs, "unit": "GB/s", "cores": team, "kind": "oracle", "sample": desc},
+        "e2e": {"value": gbs, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+# ---------------------------------------------------------------------------------
+# latency harness: K calls in one CUDA graph, one replay = one sample
+# ---------------------------------------------------------------------------------
+def graph_of(torch, stream, enqueue, K):
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=stream):
+        for k in range(K):
+            enqueue(k, stream.cuda_stream)
+    return g
+
+
+def time_graph(torch, g, stream, K, reps, warm=10):
+    with torch.cuda.stream(stream):
+        for _ in range(warm):
+            g.replay()
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(reps)]
+        for a, b in ev:
+            a.record(stream)
+            g.replay()
+            b.record(stream)
+    stream.synchronize()
+    us = np.array([a.elapsed_time(b) for a, b in ev]) * 1000.0 / K
+    return {"p10": float(np.percentile(us, 10)), "p50": float(np.percentile(us, 50)),
+            "p90": float(np.percentile(us, 90))}
+
+
+def time_stream(torch, stream, enqueue, n, warm=50):
+    """Stream-launched (no graph) per-call p50: events around blocks of 20 calls."""
+    with torch.cuda.stream(stream):
+        for k in range(warm):
+            enqueue(k, stream.cuda_stream)
+        blocks = []
+        for _ in range(n // 20):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            for k in range(20):
+                enqueue(k, stream.cuda_stream)
+            b.record(stream)
+            blocks.append((a, b))
+    stream.synchronize()
+    us = np.array([a.elapsed_time(b) for a, b in blocks]) * 1000.0 / 20
+    return float(np.percentile(us, 50))
+
+
+def latency_suite(torch, symar, synth, hbm_gbs, quick=False):
+    """C2 (16 KiB vs SoL), C3 (sweep + selector), C5 (decode-step graph)."""
+    from oracle import allreduce_oracle as O
+    out = {}
+    stream = torch.cuda.Stream()
+    K, reps = 64, (60 if quick else 300)
+    names = {symar.ONESHOT: "oneshot", symar.TWOSHOT: "twoshot", symar.LL: "ll", symar.AUTO: "auto"}
+
+    # speed-of-light parts (paper Sec. VI), measured here
+    fence_ns = symar.probe_fence(20000)
+    try:
+        rt_ns = symar.probe_pingpong(20000)
+    except symar.SymarError as e:
+        rt_ns = float("nan")
+        out["pingpong_error"] = str(e)
+
+    def empty_floor(cx, py, T):
+        g = graph_of(torch, stream, lambda k, s: symar.probe_empty(cx, py, T, s), K)
+        return time_graph(torch, g, stream, K, reps)
+
+    for P in (8, 4):
+        h = symar.SymHeap.on_torch(P, 24 << 20)
+        t0 = time.time()
+        h.autotune(symar.BF16)
+        tune_s = time.time() - t0
+        out_off = 12 << 20
+        res = {"autotune_seconds": tune_s}
+
+        def bench_size(count, algos, stream_too=False):
+            x = synth.make_inputs("normal", "bf16", P, count, synth.seed_for_config(2))
+            for q in range(P):
+                h.write_rank(q, 0, x[q])
+            want = O.allreduce(x)
+            row = {}
+            for algo in algos:
+                enq = lambda k, s, algo=algo: h.allreduce(0, out_off, count, symar.BF16, algo, s)
+                enq(0, stream.cuda_stream)
+                stream.synchronize()
+                a, c, t = h.last_choice()
+                got = np.stack([h.read_rank(q, out_off, count, np.uint16) for q in range(P)])
+                exact = bool(np.array_equal(got, want)) and h.status()[0] == 0
+                g = graph_of(torch, stream, enq, K)
+                r = time_graph(torch, g, stream, K, reps)
+                r.update({"algo": names[a], "ctas_per_rank": c, "threads": t, "bit_exact": exact})
+                if stream_too:
+                    r["stream_launched_p50"] = time_stream(torch, stream, enq, 400)
+                row[names[algo]] = r
+            return row
+
+        # C2: 16 KiB per rank
+        if P == 8:
+            row = bench_size(8192, (symar.ONESHOT, symar.TWOSHOT, symar.LL, symar.AUTO), stream_too=True)
+            best = min(row.values(), key=lambda r: r["p50"])
+            floor = empty_floor(best["ctas_per_rank"], P, best["threads"])
+            floor11 = empty_floor(1, 1, 1)
+            t_bytes_us = 2 * P * 16384 / (hbm_gbs * 1e9) * 1e6
+            sol = floor["p50"] + rt_ns / 1000.0 + t_bytes_us
+            out["latency_16KB"] = {
+                "workload": "c2: P=8, bf16, 8192 elements (16 KiB) per rank, N(0,1); buffers L2-resident (warm)",
+                "harness": f"{K} back-to-back calls in one CUDA graph, one replay = one sample, {reps} samples; "
+                           "numerator and denominator use the same harness",
+                "p50_us": best["p50"], "best": best, "per_algo": row,
+                "sol_us": sol,
+                "sol_parts_us": {"empty_launch_same_shape": floor["p50"], "empty_launch_1x1": floor11["p50"],
+                                 "flag_round_trip": rt_ns / 1000.0, "bytes_at_peak": t_bytes_us},
+                "ratio_to_sol": best["p50"] / sol,
+                "paper_style_sol_us": (2 * fence_ns + rt_ns / 2) / 1000.0,
+                "fence_us": fence_ns / 1000.0,
+            }
+        # C3: sweep
+        if P == 8:
+            sweep = []
+            for B in synth.WORKLOADS["c3"]["batch"]:
+                row = bench_size(8192 * B, (symar.ONESHOT, symar.TWOSHOT, symar.LL, symar.AUTO))
+                named = {k: v["p50"] for k, v in row.items() if k != "auto"}
+                best_name = min(named, key=named.get)
+                sweep.append({"bytes_per_rank": 16384 * B, "p50_us": {k: v["p50"] for k, v in row.items()},
+                              "selector": row["auto"]["algo"], "selector_shape":
+                                  [row["auto"]["ctas_per_rank"], row["auto"]["threads"]],
+                              "best": best_name,
+                              "selector_within_5pct": bool(row["auto"]["p50"] <= 1.05 * named[best_name]),
+                              "bit_exact": all(v["bit_exact"] for v in row.values())})
+            out["sweep"] = sweep
+        # C5: 160 calls in one graph
+        calls, count = 160, 8192 * 4
+        nb = count * 2
+        xs = [synth.make_inputs("normal", "bf16", P, count, synth.seed_for_config(5), call=k) for k in range(calls)]
+        for k in range(calls):
+            for q in range(P):
+                h.write_rank(q, k * nb, xs[k][q])
+        base_out = 10 << 20 if calls * nb <= (10 << 20) else calls * nb
+        g = graph_of(torch, stream, lambda k, s: h.allreduce(k * nb, base_out + k * nb, count, symar.BF16,
+                                                             symar.AUTO, s), calls)
+        exact = True
+        for rep in range(3):
+            with torch.cuda.stream(stream):
+                g.replay()
+            stream.synchronize()
+            for k in (0, 1, 79, 158, 159) if rep else range(calls):
+                got = np.stack([h.read_rank(q, base_out + k * nb, count, np.uint16) for q in range(P)])
+                exact = exact and bool(np.array_equal(got, O.allreduce(xs[k])))
+        a, c, t = h.last_choice()
+        r = time_graph(torch, g, stream, calls, 60 if quick else 200)
+        floor = empty_floor(c, P, t)
+        t_bytes_us = 2 * P * nb / (hbm_gbs * 1e9) * 1e6
+        sol = floor["p50"] + rt_ns / 1000.0 + t_bytes_us
+        res.update({"step_total_us_p50": r["p50"] * calls, "per_call_us": r, "sol_per_call_us": sol,
+                    "ratio_to_sol": r["p50"] / sol, "algo": names[a], "ctas_per_rank": c, "threads": t,
+                    "bit_exact": exact, "calls": calls, "bytes_per_rank": nb})
+        out.setdefault("decode_trace", {})[f"P{P}"] = res
+        stream.synchronize()
+        h.destroy()
+    return out
+
+
+# ---------------------------------------------------------------------------------
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--count", type=int, default=0, help="elements per rank (default: the 64 Mi workload)")
+    ap.add_argument("--no-latency", action="store_true", help="skip the 16 KiB / sweep / decode-trace section")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--quick", action="store_true", help="fewer latency samples")
+    ap.add_argument("--ctas", type=int, default=0)
+    ap.add_argument("--threads", type=int, default=0)
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    import torch
+    import torch.distributed as dist
+    import __graft_entry__ as ge
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the AllReduce has no CPU path")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    if rank == 0:
+        ge.build()
+    if world > 1:
+        dist.barrier()
+    from paper_2607_16100_b200 import symar, synth
+
+    hbm_gbs, peak_src = peaks()
+    w = dict(synth.WORKLOADS["c4"])
+    if args.count:
+        w["count"] = args.count
+    P, count = w["P"], w["count"]
+    M = count * 4
+    algbytes = 2 * P * M
+
+    # inputs: seeded, generated on the host, then made resident in HBM
+    x = synth.make_inputs(w["dist"], w["dtype"], P, count, w["seed"] + rank)
+    in_off, out_off = 0, (M + 255) // 256 * 256
+    heap = symar.SymHeap.on_torch(P, out_off + M, device=f"cuda:{local}")
+    for q in range(P):
+        heap.write_rank(q, in_off, x[q])
+    if args.ctas or args.threads:
+        heap.set_launch(symar.TWOSHOT, args.ctas, args.threads)
+    stream = torch.cuda.Stream()
+    sh = stream.cuda_stream
+    step = lambda: heap.allreduce(in_off, out_off, count, symar.F32, symar.TWOSHOT, sh)
+
+    for _ in range(args.warmup):
+        step()
+    stream.synchronize()
+    algo, ctas, threads = heap.last_choice()
+
+    sampler = ClockSampler(local)
+    sampler.start()
+    time.sleep(0.3)
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+    t_begin = time.time()
+    with torch.cuda.stream(stream):
+        ev[0].record(stream)
+        for i in range(args.steps):
+            step()
+            ev[i + 1].record(stream)
+    stream.synchronize()
+    torch.cuda.synchronize()
+    t_end = time.time()
+    if world > 1:
+        dist.barrier()
+    total_ms = ev[0].elapsed_time(ev[-1])
+    per_launch_ms = np.array([ev[i].elapsed_time(ev[i + 1]) for i in range(args.steps)])
+    clocks = sampler.stop(t_begin, t_end)
+    assert heap.status()[0] == symar.OK, f"device status {heap.status()}"
+
+    if world > 1:
+        t = torch.tensor([total_ms], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    value = algbytes * world * args.steps / (total_ms * 1e-3) / 1e9
+
+    # parity of what was just timed, on sampled positions (oracle element by element)
+    from oracle import allreduce_oracle as O
+    rng = np.random.default_rng(1)
+    starts = [0, count - 4096, (count // P) - 2048, 3 * (count // P) - 2048] + \
+        [int(s) for s in rng.integers(0, max(1, count - 4096), size=12)]
+    exact = True
+    for s0 in starts:
+        s0 = max(0, min(s0, count - 4096)) // 4 * 4
+        n = min(4096, count - s0)
+        want = O.allreduce(np.ascontiguousarray(x[:, s0:s0 + n]))
+        for r in range(P):
+            got = heap.read_rank(r, out_off + s0 * 4, n, np.float32)
+            exact = exact and bool(np.array_equal(got.view(np.uint32), want[r].view(np.uint32)))
+
+    line = {
+        "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": total_ms / args.steps, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "impl": "ours",
+        "config": {
+            "workload": f"c4: P={P} emulated ranks, fp32, {count} elements ({M >> 20} MiB) per rank, U(-1,1), "
+                        "two-shot reduce-scatter + all-gather; value = 2*P*M bytes / time",
+            "P": P, "elements_per_rank": count, "algo": "twoshot", "ctas_per_rank": ctas, "threads": threads,
+            "l2": f"inputs {P * M >> 20} MiB + outputs {P * M >> 20} MiB per step, far larger than the 126 MB L2; "
+                  "no flush needed",
+            "multi_gpu": "replicas only (independent heaps, no exchange between GPUs)",
+        },
+        "clocks": clocks,
+        "gpu_launches": args.steps,
+        "bit_exact_sampled": exact,
+        "roofline": {
+            "bound": "hbm", "achieved": algbytes / (float(per_launch_ms.mean()) * 1e-3) / 1e9, "peak": hbm_gbs,
+            "unit": "GB/s", "frac": algbytes / (float(per_launch_ms.mean()) * 1e-3) / 1e9 / hbm_gbs,
+            "peak_source": peak_src, "kernel": "twoshot_kernel<F32, 8>",
+            "algorithmic_bytes_per_launch": algbytes,
+            "launch_ms": {"mean": float(per_launch_ms.mean()), "min": float(per_launch_ms.min()),
+                          "max": float(per_launch_ms.max())},
+            "frac_of_nominal_8TBps": algbytes / (float(per_launch_ms.mean()) * 1e-3) / 1e9 / 8000.0,
+            "traffic": None,
+        },
+    }
+    traffic_note = ROOT / "profiles" / "twoshot_f32_p8_traffic.json"
+    if traffic_note.exists():
+        tn = json.loads(traffic_note.read_text())
+        line["roofline"]["traffic"] = tn["dram_bytes_per_launch_at_full_size"]
+        line["roofline"]["traffic_source"] = tn["source"]
+
+    # end to end through the host-buffer entry point
+    if not args.no_e2e:
+        hin = torch.from_numpy(x).pin_memory()
+        hout = torch.empty_like(hin).pin_memory()
+        e2e_steps = min(args.steps, 5)
+        estep = lambda: heap.allreduce_host(hin.data_ptr(), hout.data_ptr(), in_off, out_off, count,
+                                            symar.F32, symar.TWOSHOT, sh)
+        estep()
+        stream.synchronize()
+        if world > 1:
+            dist.barrier()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        with torch.cuda.stream(stream):
+            a.record(stream)
+            for _ in range(e2e_steps):
+                estep()
+            b.record(stream)
+        stream.synchronize()
+        e_ms = a.elapsed_time(b)
+        if world > 1:
+            t = torch.tensor([e_ms], device="cuda", dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e_ms = float(t.item())
+        s0 = count // 2
+        want = O.allreduce(np.ascontiguousarray(x[:, s0:s0 + 4096]))
+        e2e_exact = bool(np.array_equal(hout.numpy()[:, s0:s0 + 4096].view(np.uint32), want.view(np.uint32)))
+        line["e2e"] = {"value": algbytes * world * e2e_steps / (e_ms * 1e-3) / 1e9, "unit": "GB/s",
+                       "h2d_bytes_per_step": P * M, "d2h_bytes_per_step": P * M, "steps": e2e_steps,
+                       "ms_per_step": e_ms / e2e_steps, "bit_exact_sampled": e2e_exact,
+                       "note": "allreduce_host(): pinned host inputs -> HBM, kernel, all P outputs -> pinned host"}
+        del hin, hout
+
+    heap.destroy()
+    del heap
+
+    if rank == 0 and not args.no_cpu:
+        xs = x if count <= (16 << 20) else np.ascontiguousarray(x[:, :16 << 20])
+        best, team = 1e30, 1
+        for _ in range(3):
+            t0 = time.perf_counter()
+            _, team = O.allreduce_timed_team(xs, threads=0)
+            best = min(best, time.perf_counter() - t0)
+        t0 = time.perf_counter()
+        O.allreduce_timed_team(xs, threads=1)
+        one = time.perf_counter() - t0
+        line["cpu_baseline"] = {
+            "value": 2 * P * xs.shape[1] * 4 / best / 1e9, "unit": "GB/s", "cores": team, "kind": "oracle",
+            "sample": f"first {xs.shape[1]} of {count} elements per rank, best of 3 full oracle calls "
+                      f"(OpenMP over elements); single-thread: {2 * P * xs.shape[1] * 4 / one / 1e9:.2f} GB/s",
+        }
+    del x
+
+    if rank == 0 and not args.no_latency:
+        line.update(latency_suite(torch, symar, synth, hbm_gbs, quick=args.quick))
+
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+    if rank == 0:
+        print(json.dumps(line))
+
+
+if __name__ == "__main__":
+    main()
