@@ -340,7 +340,7 @@ def main():
 
     # inputs: seeded, generated on the host, then made resident in HBM
     x = synth.make_inputs(w["dist"], w["dtype"], P, count, w["seed"] + rank)
-    in_off, out_off = 0, (M + 255) // 256 * 256
+    in_off, out_off = 0, (M + 4095) // 4096 * 4096
     heap = symar.SymHeap.on_torch(P, out_off + M, device=f"cuda:{local}")
     for q in range(P):
         heap.write_rank(q, in_off, x[q])

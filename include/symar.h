@@ -61,7 +61,8 @@ enum {
     SYMAR_MAX_CTAS      = 160,    /* CTA slots per rank that own flags and an epoch counter   */
     SYMAR_LL_SLOTS      = 64,     /* CTA slots per rank that own an LL scratch region          */
     SYMAR_LL_SLOT_VECS  = 1024,   /* 16-byte payload vectors per LL slot, sender and iteration */
-    SYMAR_ALIGN         = 256     /* alignment of every region of a segment                    */
+    SYMAR_ALIGN         = 4096    /* alignment of the heap and of every region of a segment:
+                                     streams that start on 1 KiB boundaries use HBM best        */
 };
 
 typedef struct {
@@ -89,7 +90,7 @@ size_t symheap_required_bytes(int P, size_t bytes_per_rank);
 int symheap_create(symheap_t **heap, int P, size_t bytes_per_rank);
 
 /* As symheap_create, in caller-owned device memory (e.g. a torch tensor) of at
- * least symheap_required_bytes() bytes, 256-byte aligned.  The caller keeps the
+ * least symheap_required_bytes() bytes, SYMAR_ALIGN-byte aligned.  The caller keeps the
  * memory alive until symheap_destroy and frees it afterwards.                  */
 int symheap_create_on(symheap_t **heap, int P, size_t bytes_per_rank,
                       void *device_mem, size_t device_bytes);
@@ -123,7 +124,8 @@ int symheap_status(symheap_t *heap, int *code, int *rank, int *peer, int *cta);
  *
  * in, out : symmetric addresses -- device pointers into RANK 0's user region
  *           (symheap_rank_ptr(heap, 0, off)); rank q's buffer is the same offset
- *           in its own segment.  16-byte aligned.  Out-of-place only (Sec. VII
+ *           in its own segment.  16-byte aligned (1 KiB-aligned buffers stream
+ *           fastest for large messages).  Out-of-place only (Sec. VII
  *           measures out-of-place): the byte ranges must not overlap.
  * count   : elements PER RANK.  0 is a no-op.  Any count is accepted; a ragged
  *           tail is handled inside the kernels.
@@ -158,6 +160,10 @@ int allreduce_autotune(symheap_t *heap, symar_dtype_t dtype);
 int symar_last_choice(const symheap_t *heap, symar_algo_t *algo,
                       int *ctas_per_rank, int *threads);
 
+/* Kernel variant bits (see symar_set_variant) and dynamic shared memory of the
+ * last launch; shared_bytes > 0 means the bulk-copy two-shot kernel ran.          */
+int symar_last_kernel(const symheap_t *heap, unsigned int *variant, size_t *shared_bytes);
+
 /* What SYMAR_AUTO would launch for a message of `count` elements. */
 int symar_query_choice(symheap_t *heap, size_t count, symar_dtype_t dtype,
                        symar_algo_t *algo, int *ctas_per_rank, int *threads);
@@ -172,6 +178,15 @@ int symar_tuned_entry(const symheap_t *heap, symar_dtype_t dtype, int log2_bytes
  * library still clamps P * ctas_per_rank to what is co-resident on the device:
  * CTAs of different ranks wait for one another, so all must be resident.       */
 int symar_set_launch(symheap_t *heap, symar_algo_t algo, int ctas_per_rank, int threads);
+
+/* Implementation variant of one algorithm's kernel, for performance experiments;
+ * every variant computes the same bits.  0 = default.  One-shot: bit 0 = publish
+ * the exchange count at kernel exit instead of right after the exchange;
+ * two-shot: bit 0 = contiguous chunks also for large messages (no block-cyclic
+ * ownership), bit 1 = 16-byte instead of 32-byte accesses for large messages,
+ * bit 2 = never use the bulk-copy kernel, bits 8-10 = its pipeline depth (0:
+ * default), bits 12-13 = log2 of its tile size over 4 KiB.                        */
+int symar_set_variant(symheap_t *heap, symar_algo_t algo, unsigned int variant);
 
 /* Upper bound of any device-side wait, in microseconds (default 2 000 000). */
 int symar_set_spin_limit_us(symheap_t *heap, unsigned int microseconds);

@@ -26,6 +26,26 @@ __device__ __forceinline__ void st_release_u32(uint32_t *p, uint32_t v)
 {
     asm volatile("st.release." SYMAR_SCOPE ".global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
+__device__ __forceinline__ uint32_t ld_relaxed_u32(const uint32_t *p)
+{
+    uint32_t v;
+    asm volatile("ld.relaxed." SYMAR_SCOPE ".global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+// Signal: add 1 to a peer's flag word; release orders every earlier write of
+// this thread (and, through the preceding CTA barrier, of its CTA) before it.
+__device__ __forceinline__ void red_release_inc_u32(uint32_t *p)
+{
+    asm volatile("red.release." SYMAR_SCOPE ".global.add.u32 [%0], 1;" ::"l"(p) : "memory");
+}
+__device__ __forceinline__ void red_relaxed_inc_u32(uint32_t *p)
+{
+    asm volatile("red.relaxed." SYMAR_SCOPE ".global.add.u32 [%0], 1;" ::"l"(p) : "memory");
+}
+__device__ __forceinline__ void fence_acq_rel()
+{
+    asm volatile("fence.acq_rel." SYMAR_SCOPE ";" ::: "memory");
+}
 __device__ __forceinline__ uint64_t ld_relaxed_u64(const uint64_t *p)
 {
     uint64_t v;
@@ -63,13 +83,13 @@ __device__ __forceinline__ uint4 ld_own(const void *p)
                  : "l"(p));
     return v;
 }
-// A PEER's input is read only after that peer's "ready" flag was acquired, so it
-// must be an ordinary (coherent) load ordered after the acquire; each byte is
-// used once per reading rank, hence no L1 allocation.
+// A PEER's input is read only after that peer's "ready" signal was observed: a
+// strong (L1-bypassing) load issued after the poll, so it cannot return a line
+// cached before the signal.
 __device__ __forceinline__ uint4 ld_peer(const void *p)
 {
     uint4 v;
-    asm volatile("ld.global.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];"
+    asm volatile("ld.relaxed." SYMAR_SCOPE ".global.v4.u32 {%0, %1, %2, %3}, [%4];"
                  : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
                  : "l"(p)
                  : "memory");
@@ -80,6 +100,27 @@ __device__ __forceinline__ void st_output(void *p, uint4 v)
 {
     asm volatile("st.global.cs.v4.u32 [%0], {%1, %2, %3, %4};" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z),
                  "r"(v.w)
+                 : "memory");
+}
+
+// 32-byte accesses (two adjacent 16-byte vectors), 32-byte aligned.  Issued
+// after this warp's acquire poll, which already dropped any stale L1 line, so
+// an ordinary load is enough.
+struct U32B { uint4 lo, hi; };
+__device__ __forceinline__ U32B ld_peer_32B(const void *p)
+{
+    U32B v;
+    asm volatile("ld.global.L1::no_allocate.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                 : "=r"(v.lo.x), "=r"(v.lo.y), "=r"(v.lo.z), "=r"(v.lo.w), "=r"(v.hi.x), "=r"(v.hi.y),
+                   "=r"(v.hi.z), "=r"(v.hi.w)
+                 : "l"(p)
+                 : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_output_32B(void *p, const U32B &v)
+{
+    asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(p), "r"(v.lo.x), "r"(v.lo.y),
+                 "r"(v.lo.z), "r"(v.lo.w), "r"(v.hi.x), "r"(v.hi.y), "r"(v.hi.z), "r"(v.hi.w)
                  : "memory");
 }
 
@@ -109,7 +150,7 @@ struct Spin {
 };
 
 // First error wins; the kernel then leaves through its normal exit.
-__device__ __noinline__ void report_timeout(uint32_t *ctl, int rank, int peer, int cta)
+static __device__ __noinline__ void report_timeout(uint32_t *ctl, int rank, int peer, int cta)
 {
     if (atomicCAS(&ctl[kCtlCode], 0u, (uint32_t)SYMAR_ERR_TIMEOUT) == 0u) {
         ctl[kCtlRank] = (uint32_t)rank;
@@ -183,14 +224,18 @@ __device__ __forceinline__ uint4 reduce_in_rank_order(const uint4 (&x)[P])
     return E::narrow(acc);
 }
 
-// Store of output vector v; the last vector of a message may be partial.
-__device__ __forceinline__ void store_result(char *out, uint64_t v, uint4 val, uint64_t nvec,
+// Store of output vector v; the last vector of a message may be partial.  The
+// partial store peels 2-byte pieces out of registers with compile-time indices
+// (no address of `val` is taken, so it never lives in local memory).
+__device__ __forceinline__ void store_result(char *out, uint64_t v, const uint4 &val, uint64_t nvec,
                                              uint32_t tail_bytes)
 {
     if (tail_bytes != 0 && v == nvec - 1) {
-        const uint16_t *src = reinterpret_cast<const uint16_t *>(&val);
-        uint16_t *dst       = reinterpret_cast<uint16_t *>(out + v * 16);
-        for (uint32_t b = 0; b < tail_bytes / 2; ++b) dst[b] = src[b];
+        uint16_t *dst = reinterpret_cast<uint16_t *>(out + v * 16);
+        const uint32_t w[4] = {val.x, val.y, val.z, val.w};
+#pragma unroll
+        for (int b = 0; b < 8; ++b)
+            if ((uint32_t)b < tail_bytes / 2) dst[b] = (uint16_t)(w[b >> 1] >> ((b & 1) * 16));
     } else {
         st_output(out + v * 16, val);
     }
@@ -210,5 +255,71 @@ __device__ __forceinline__ void debug_delay(const KArgs &a, int rank, int cta)
     const uint64_t t0   = globaltimer_ns();
     while (globaltimer_ns() - t0 < wait) { /* bounded by dbg_delay_ns */ }
 }
+
+// ---- one synchronisation of Table I ---------------------------------------------------
+// Slot c of rank r signals slot c of every peer and waits for every peer's
+// signal.
+//
+// A signal is an atomic increment of the receiver's flag word for this sender,
+// so the sender needs no sequence number.  The receiver compares against its
+// own count of exchanges on this slot (a word private to (rank, slot) that the
+// caller advances), whose load travels together with the first poll.  Lane q
+// polls peer q's flag with an acquire load, so all P polls are in flight
+// together and one round trip observes them all.
+//
+// RELEASE says whether the signal must order this CTA's earlier writes (the
+// "chunk done" handoff: yes, after a CTA barrier).  The "input ready" signal
+// orders nothing written by this kernel -- the input was complete before the
+// kernel started, and a kernel boundary makes it visible to every later reader
+// -- so it is a relaxed increment and costs no fence on the critical path.
+// `want` receives the count to publish.  Returns false if the wait ran out.
+template <int P, bool RELEASE>
+__device__ __forceinline__ bool flag_exchange(const KArgs &a, uint64_t flags_off, const uint32_t *count,
+                                              int r, int c, bool silent, bool all_warps, uint32_t &want)
+{
+    const uint32_t t    = threadIdx.x;
+    const uint32_t lane = t & 31u;
+    if (t < P && !silent) {
+        uint32_t *dst =
+            reinterpret_cast<uint32_t *>(a.seg0 + t * a.stride + flags_off + (size_t)c * kFlagGroup) + r;
+        if (RELEASE) red_release_inc_u32(dst);
+        else red_relaxed_inc_u32(dst);
+    }
+    const uint32_t *mine =
+        reinterpret_cast<const uint32_t *>(a.seg0 + (size_t)r * a.stride + flags_off + (size_t)c * kFlagGroup) +
+        (lane < P ? lane : 0);
+    const uint32_t n = ld_relaxed_u32(count);
+    if (!all_warps && t >= 32) {
+        want = n + 1;
+        return true;
+    }
+    Spin spin;
+    for (;;) {
+        const uint32_t f = ld_acquire_u32(mine);
+        want = n + 1;
+        // ">= want": a peer may already have signalled its next call
+        const unsigned late = __ballot_sync(0xffffffffu, lane < P && (int32_t)(f - want) < 0);
+        if (late == 0) return true;
+        if (spin.due() && __any_sync(0xffffffffu, spin.expired(a.spin_ns))) {
+            if (lane == 0) report_timeout(a.ctl, r, __ffs(late) - 1, c);
+            return false;
+        }
+    }
+}
+
+// Reduce-scatter + all-gather of one 16-byte vector: P loads, the rank-ordered
+// sum, then the result goes straight from registers into every rank's output.
+template <typename E, int P>
+__device__ __forceinline__ void twoshot_vector(const KArgs &a, uint64_t v)
+{
+    uint4 x[P];
+#pragma unroll
+    for (int q = 0; q < P; ++q) x[q] = ld_peer(a.seg0 + (size_t)q * a.stride + a.in_off + v * 16);
+    const uint4 res = reduce_in_rank_order<E, P>(x);
+#pragma unroll
+    for (int q = 0; q < P; ++q)
+        store_result(a.seg0 + (size_t)q * a.stride + a.out_off, v, res, a.nvec, a.tail_bytes);
+}
+
 
 }  // namespace symar

@@ -19,6 +19,7 @@ namespace symar {
 struct LaunchCfg {
     int ctas    = 0;   // per rank; 0 = not set
     int threads = 0;
+    int variant = -1;  // kernel variant bits; -1 = not set
 };
 
 constexpr int kBuckets = 40;   // bucket b holds messages of (2^(b-1), 2^b] bytes per rank
@@ -59,13 +60,18 @@ struct symheap {
     uint32_t *ctl   = nullptr;
     int       device  = 0;
     int       num_sms = 0;
+    int       max_smem = 48 * 1024;   // opt-in dynamic shared memory per CTA
     uint64_t  spin_ns = 2000000000ull;
     int       dbg_mute     = -1;
     unsigned  dbg_seed     = 0;
     unsigned  dbg_delay_ns = 0;
     LaunchCfg forced[kAlgos];
+    unsigned  variant[kAlgos] = {0, 0, 0, 0};
+    bool      variant_forced[kAlgos] = {false, false, false, false};
     Tuned     tuned[2];
     int       last_algo = 0, last_ctas = 0, last_threads = 0;
+    unsigned  last_variant = 0;
+    size_t    last_smem = 0;
     std::map<std::tuple<const void *, int>, int> resident;   // (kernel, threads) -> CTAs co-resident
 };
 
@@ -85,13 +91,13 @@ static int bucket_of(size_t bytes)
 // CTAs of the given kernel and block size that fit on the device at once.  The
 // CTAs of different ranks wait for one another, so a grid larger than this
 // could leave a waiting CTA holding the SM that the CTA it waits for needs.
-static int max_resident(symheap *h, KernelFn fn, int threads)
+static int max_resident(symheap *h, KernelFn fn, int threads, size_t smem = 0)
 {
-    auto key = std::make_tuple((const void *)fn, threads);
+    auto key = std::make_tuple((const void *)fn, threads + (int)(smem << 4));
     auto it  = h->resident.find(key);
     if (it != h->resident.end()) return it->second;
     int per_sm = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fn, threads, 0) != cudaSuccess) per_sm = 1;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fn, threads, smem) != cudaSuccess) per_sm = 1;
     int n = std::max(1, per_sm) * h->num_sms;
     h->resident[key] = n;
     return n;
@@ -104,17 +110,31 @@ static int round_threads(uint64_t want)
     return t;
 }
 
+// Variant bits of the bulk two-shot kernel: pipeline depth and tile size.
+static int bulk_variant(int stages, int tile_log2_over_4k) { return (stages << 8) | (tile_log2_over_4k << 12); }
+
 // Launch shape when neither the caller nor the tuner fixed one.
 static LaunchCfg default_cfg(const symheap *h, int algo, uint64_t nvec)
 {
     LaunchCfg c;
+    c.variant = 0;
     const uint64_t work = algo == SYMAR_TWOSHOT ? (nvec + h->P - 1) / h->P : nvec;   // vectors per rank partition
-    c.threads = work >= 1024 ? 256 : round_threads(std::max<uint64_t>(work / 4, 32));
-    if (work >= (uint64_t)1 << 18) c.threads = 512;
+    if (algo == SYMAR_TWOSHOT && nvec >= kBulkMinVec) {
+        // Bandwidth regime.  HBM3e delivers most when few, long streams are in
+        // flight: about 100 CTAs in total, each with one 64 KiB stage (P tiles)
+        // ahead of the one it reduces (measured on B200; more CTAs, more stages or
+        // shorter tiles all lose several percent to DRAM page conflicts).
+        int tile_log2 = 0;
+        while ((4096u << tile_log2) * (unsigned)h->P < 65536u && tile_log2 < 3) ++tile_log2;
+        c.threads = 256;
+        c.ctas    = std::max(1, std::min(100 / h->P, (int)kMaxCtas));
+        c.variant = bulk_variant(2, tile_log2);
+        return c;
+    }
+    // Latency regime: about one vector per thread, small blocks, few CTAs.
+    c.threads = work >= 2048 ? 128 : round_threads(std::max<uint64_t>(work / 16, 32));
     uint64_t ctas = (work + c.threads - 1) / c.threads;
-    // bandwidth regime: two CTAs of 512 threads per SM over all ranks
-    const uint64_t fill = std::max(1, 2 * h->num_sms / h->P);
-    const uint64_t cap  = algo == SYMAR_LL ? (uint64_t)kLLSlots : (work >= (uint64_t)1 << 18 ? fill : 16);
+    const uint64_t cap = algo == SYMAR_LL ? (uint64_t)kLLSlots : (uint64_t)std::max(1, 2 * h->num_sms / h->P);
     c.ctas = (int)std::max<uint64_t>(1, std::min(ctas, cap));
     return c;
 }
@@ -130,6 +150,7 @@ struct Plan {
     int       algo;
     LaunchCfg cfg;
     KernelFn  fn;
+    size_t    smem = 0;     // dynamic shared memory of the launch
     KArgs     args;
 };
 
@@ -148,16 +169,32 @@ static int make_plan(symheap *h, size_t in_off, size_t out_off, size_t count, in
     if (tn.valid && tn.cfg[algo][b].ctas > 0) cfg = tn.cfg[algo][b];
     if (h->forced[algo].ctas > 0) cfg.ctas = h->forced[algo].ctas;
     if (h->forced[algo].threads > 0) cfg.threads = h->forced[algo].threads;
+    if (h->variant_forced[algo]) cfg.variant = (int)h->variant[algo];
+    if (cfg.variant < 0) cfg.variant = 0;
+    const unsigned var = (unsigned)cfg.variant;
 
     cfg.threads = std::min<int>(std::max(32, (cfg.threads + 31) / 32 * 32), (int)kMaxThreads);
-    KernelFn fn = kernel_for(algo, dtype, h->P, dbg_on(h));
-    if (!fn) return SYMAR_ERR_INVAL;
-    const int cap_slots = algo == SYMAR_LL ? kLLSlots : kMaxCtas;
-    const int cap_res   = std::max(1, max_resident(h, fn, cfg.threads) / h->P);
-    cfg.ctas = std::max(1, std::min({cfg.ctas, cap_slots, cap_res}));
-
     KArgs &a = p->args;
     std::memset(&a, 0, sizeof a);
+    KernelFn fn = kernel_for(algo, dtype, h->P, dbg_on(h));
+    p->smem     = 0;
+    // bandwidth regime of two-shot: the bulk-copy kernel (the test hooks live in
+    // the register kernel only)
+    if (algo == SYMAR_TWOSHOT && nvec >= kBulkMinVec && !dbg_on(h) && !(var & 4u)) {
+        fn          = bulk_kernel_for(dtype, h->P);
+        const unsigned v = var;
+        a.tile_vecs = 256u << ((v >> 12) & 3u);                       // 4, 8, 16 or 32 KiB tiles
+        a.stages    = ((v >> 8) & 7u) ? ((v >> 8) & 7u) : 2u;
+        while (a.stages > 2 && bulk_smem_bytes(h->P, a.tile_vecs, a.stages) > (size_t)h->max_smem) --a.stages;
+        while (a.tile_vecs > 256 && bulk_smem_bytes(h->P, a.tile_vecs, a.stages) > (size_t)h->max_smem)
+            a.tile_vecs /= 2;
+        p->smem     = bulk_smem_bytes(h->P, a.tile_vecs, a.stages);
+    }
+    if (!fn) return SYMAR_ERR_INVAL;
+    const int cap_slots = algo == SYMAR_LL ? kLLSlots : kMaxCtas;
+    const int cap_res   = std::max(1, max_resident(h, fn, cfg.threads, p->smem) / h->P);
+    cfg.ctas = std::max(1, std::min({cfg.ctas, cap_slots, cap_res}));
+
     a.seg0       = h->seg0;
     a.stride     = h->L.stride;
     a.in_off     = in_off;
@@ -171,9 +208,15 @@ static int make_plan(symheap *h, size_t in_off, size_t out_off, size_t count, in
     a.ctl        = h->ctl;
     a.spin_ns    = h->spin_ns;
     a.tail_bytes = (uint32_t)(bytes % 16);
+    a.variant    = var;
     a.dbg_mute   = h->dbg_mute;
     a.dbg_seed   = h->dbg_seed;
     a.dbg_delay_ns = h->dbg_delay_ns;
+    if (algo == SYMAR_TWOSHOT) {
+        const bool cyclic = nvec >= kCyclicMinVec && !(var & 1u);
+        a.blk_log2 = cyclic ? kCyclicLog2 : kOneChunk;
+        a.wide     = cyclic && ((in_off | out_off) % 32 == 0) && !(var & 2u);
+    }
     if (algo == SYMAR_LL) {
         // every CTA takes `cv` vectors per iteration; iterations alternate sub-buffers
         const uint64_t per_cta = (nvec + cfg.ctas - 1) / cfg.ctas;
@@ -215,11 +258,13 @@ static int run(symheap *h, const void *in, void *out, size_t count, int dtype, i
     Plan p;
     rc = make_plan(h, io, oo, count, dtype, algo, &p);
     if (rc != SYMAR_OK) return rc;
-    cudaError_t e = launch_kernel(p.fn, h->P, p.cfg.ctas, p.cfg.threads, p.args, s);
+    cudaError_t e = launch_kernel(p.fn, h->P, p.cfg.ctas, p.cfg.threads, p.smem, p.args, s);
     if (e != cudaSuccess) return cuda_fail(e, "kernel launch");
     h->last_algo    = p.algo;
     h->last_ctas    = p.cfg.ctas;
     h->last_threads = p.cfg.threads;
+    h->last_variant = p.args.variant;
+    h->last_smem    = p.smem;
     return SYMAR_OK;
 }
 
@@ -231,7 +276,7 @@ static int time_calls(symheap *h, cudaStream_t s, size_t count, int dtype, int a
 {
     const size_t bytes = count * elem_size(dtype);
     const void *in = h->seg0;
-    void *out      = h->seg0 + round_up(bytes, 256);
+    void *out      = h->seg0 + round_up(bytes, kAlign);
     cudaGraph_t graph;
     cudaGraphExec_t exec;
     CU(cudaStreamBeginCapture(s, cudaStreamCaptureModeThreadLocal));
@@ -274,10 +319,10 @@ static int time_calls(symheap *h, cudaStream_t s, size_t count, int dtype, int a
 static int autotune(symheap *h, int dtype)
 {
     static const int kThreads[] = {64, 128, 256, 512};
-    static const int kCtas[]    = {1, 2, 4, 8, 12, 16, 18, 24, 32, 37, 48, 64, 74};
+    static const int kCtas[]    = {1, 2, 4, 8, 10, 12, 15, 16, 18, 24, 32, 37, 48, 64, 74};
     const size_t es = elem_size(dtype);
     Tuned tn;
-    size_t max_bytes = std::min<size_t>(h->bytes_per_rank / 2 / 256 * 256, (size_t)64 << 20);
+    size_t max_bytes = std::min<size_t>(h->bytes_per_rank / 2 / kAlign * kAlign, (size_t)64 << 20);
     if (max_bytes < 16) return SYMAR_ERR_INVAL;
     tn.lo_bucket = 4;
     tn.hi_bucket = 4;
@@ -286,7 +331,13 @@ static int autotune(symheap *h, int dtype)
     cudaStream_t s;
     CU(cudaStreamCreateWithFlags(&s, cudaStreamNonBlocking));
     LaunchCfg saved[kAlgos];
-    for (int a = 0; a < kAlgos; ++a) saved[a] = h->forced[a];
+    unsigned saved_variant[kAlgos];
+    bool saved_forced[kAlgos];
+    for (int a = 0; a < kAlgos; ++a) {
+        saved[a]         = h->forced[a];
+        saved_variant[a] = h->variant[a];
+        saved_forced[a]  = h->variant_forced[a];
+    }
     const Tuned saved_tuned = h->tuned[dtype];
     h->tuned[dtype].valid = false;
 
@@ -305,34 +356,54 @@ static int autotune(symheap *h, int dtype)
             if (algo == SYMAR_LL && bytes > (4u << 20)) continue;      // 2 P M scratch traffic: hopeless there
             if (algo == SYMAR_ONESHOT && bytes > (32u << 20)) continue;
             const uint64_t work = algo == SYMAR_TWOSHOT ? (nvec + h->P - 1) / h->P : nvec;
-            for (int T : kThreads) {
-                for (int C : kCtas) {
-                    // skip shapes with far more threads than vectors, except the smallest
-                    if ((uint64_t)C * T > 2 * work && !(C == 1 && T == 64)) continue;
-                    // and shapes that would leave each thread hundreds of vectors
-                    if (work / ((uint64_t)C * T) > 4096) continue;
-                    h->forced[algo] = LaunchCfg{C, T};
-                    Plan p;
-                    if (make_plan(h, 0, round_up(bytes, 256), count, dtype, algo, &p) != SYMAR_OK) continue;
-                    if (p.cfg.ctas != C || p.cfg.threads != T) continue;   // clamped: a duplicate of another shape
-                    double us = 0;
-                    rc = time_calls(h, s, count, dtype, algo, K, reps, &us);
-                    if (rc != SYMAR_OK) break;
-                    if (us < tn.us[algo][b]) {
-                        tn.us[algo][b]  = us;
-                        tn.cfg[algo][b] = LaunchCfg{C, T};
+            // kernel variants worth timing: the default; for two-shot in the bandwidth
+            // regime the bulk kernel's tile sizes and depths, and the register kernel
+            std::vector<int> variants = {0};
+            const bool bulk = algo == SYMAR_TWOSHOT && nvec >= kBulkMinVec;
+            if (bulk)
+                variants = {bulk_variant(2, 1), bulk_variant(3, 1), bulk_variant(2, 2), bulk_variant(3, 0),
+                            bulk_variant(4, 0), 4};
+            for (int var : variants) {
+                for (int T : kThreads) {
+                    if (bulk && var != 4 && T != 128 && T != 256) continue;
+                    for (int C : kCtas) {
+                        // skip shapes with far more threads than vectors, except the smallest
+                        if ((uint64_t)C * T > 2 * work && !(C == 1 && T == 64)) continue;
+                        // and shapes that would leave each thread hundreds of vectors
+                        if (!bulk && work / ((uint64_t)C * T) > 4096) continue;
+                        if (bulk && (C * h->P < 48)) continue;
+                        h->forced[algo]         = LaunchCfg{C, T, var};
+                        h->variant[algo]        = (unsigned)var;
+                        h->variant_forced[algo] = true;
+                        Plan p;
+                        if (make_plan(h, 0, round_up(bytes, kAlign), count, dtype, algo, &p) != SYMAR_OK) continue;
+                        if (p.cfg.ctas != C || p.cfg.threads != T) continue;   // clamped: a duplicate of another shape
+                        double us = 0;
+                        rc = time_calls(h, s, count, dtype, algo, K, reps, &us);
+                        if (rc != SYMAR_OK) break;
+                        if (us < tn.us[algo][b]) {
+                            tn.us[algo][b]  = us;
+                            tn.cfg[algo][b] = LaunchCfg{C, T, var};
+                        }
                     }
+                    if (rc != SYMAR_OK) break;
                 }
                 if (rc != SYMAR_OK) break;
             }
-            h->forced[algo] = saved[algo];
+            h->forced[algo]         = saved[algo];
+            h->variant[algo]        = saved_variant[algo];
+            h->variant_forced[algo] = saved_forced[algo];
             if (tn.us[algo][b] < best_us) {
                 best_us         = tn.us[algo][b];
                 tn.best_algo[b] = algo;
             }
         }
     }
-    for (int a = 0; a < kAlgos; ++a) h->forced[a] = saved[a];
+    for (int a = 0; a < kAlgos; ++a) {
+        h->forced[a]         = saved[a];
+        h->variant[a]        = saved_variant[a];
+        h->variant_forced[a] = saved_forced[a];
+    }
     cudaStreamSynchronize(s);
     cudaStreamDestroy(s);
     if (rc != SYMAR_OK) {
@@ -360,6 +431,7 @@ static int create_common(symheap_t **heap, int P, size_t bytes_per_rank, void *m
     h->ctl  = (uint32_t *)h->mem;
     cudaError_t e = cudaGetDevice(&h->device);
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&h->num_sms, cudaDevAttrMultiProcessorCount, h->device);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&h->max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, h->device);
     if (e == cudaSuccess) e = cudaMemset(h->mem, 0, kCtlBytes);
     for (int q = 0; q < P && e == cudaSuccess; ++q)
         e = cudaMemset(h->seg0 + (size_t)q * L.stride + L.ll_off, 0, L.seg_bytes - L.ll_off);
@@ -369,6 +441,13 @@ static int create_common(symheap_t **heap, int P, size_t bytes_per_rank, void *m
         for (int dt = SYMAR_F32; dt <= SYMAR_BF16 && e == cudaSuccess; ++dt) {
             cudaFuncAttributes attr;
             e = cudaFuncGetAttributes(&attr, kernel_for(algo, dt, P, false));
+            if (e == cudaSuccess && algo == SYMAR_TWOSHOT) {
+                KernelFn bk = bulk_kernel_for(dt, P);
+                e = cudaFuncGetAttributes(&attr, bk);
+                // opt in to the large dynamic shared memory now (not during a capture)
+                if (e == cudaSuccess)
+                    e = cudaFuncSetAttribute(bk, cudaFuncAttributeMaxDynamicSharedMemorySize, h->max_smem);
+            }
         }
     if (e == cudaSuccess) e = cudaDeviceSynchronize();
     if (e != cudaSuccess) {
@@ -510,6 +589,14 @@ int symar_last_choice(const symheap_t *heap, symar_algo_t *algo, int *ctas_per_r
     return SYMAR_OK;
 }
 
+int symar_last_kernel(const symheap_t *heap, unsigned int *variant, size_t *shared_bytes)
+{
+    if (!heap) return SYMAR_ERR_INVAL;
+    if (variant) *variant = heap->last_variant;
+    if (shared_bytes) *shared_bytes = heap->last_smem;
+    return SYMAR_OK;
+}
+
 int symar_query_choice(symheap_t *heap, size_t count, symar_dtype_t dtype, symar_algo_t *algo,
                        int *ctas_per_rank, int *threads)
 {
@@ -541,6 +628,14 @@ int symar_set_launch(symheap_t *heap, symar_algo_t algo, int ctas_per_rank, int 
     if (!heap || algo < SYMAR_ONESHOT || algo > SYMAR_LL) return SYMAR_ERR_INVAL;
     if (ctas_per_rank < 0 || threads < 0 || threads > (int)kMaxThreads) return SYMAR_ERR_INVAL;
     heap->forced[algo] = LaunchCfg{ctas_per_rank, threads};
+    return SYMAR_OK;
+}
+
+int symar_set_variant(symheap_t *heap, symar_algo_t algo, unsigned int variant)
+{
+    if (!heap || algo < SYMAR_ONESHOT || algo > SYMAR_LL) return SYMAR_ERR_INVAL;
+    heap->variant[algo]        = variant;
+    heap->variant_forced[algo] = variant != 0;
     return SYMAR_OK;
 }
 

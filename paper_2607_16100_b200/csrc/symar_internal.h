@@ -12,8 +12,12 @@ using KernelFn = void (*)(const KArgs);
 // variant that honours the test hooks.  nullptr for unsupported combinations.
 KernelFn kernel_for(int algo, int dtype, int P, bool dbg);
 
+// Two-shot kernel of the bandwidth regime (bulk asynchronous copies through
+// shared memory); needs bulk_smem_bytes() of dynamic shared memory.
+KernelFn bulk_kernel_for(int dtype, int P);
+
 // grid = (ctas_per_rank, P), block = threads; returns the launch status.
-cudaError_t launch_kernel(KernelFn fn, int P, int ctas_per_rank, int threads, const KArgs &args,
-                          cudaStream_t stream);
+cudaError_t launch_kernel(KernelFn fn, int P, int ctas_per_rank, int threads, size_t smem_bytes,
+                          const KArgs &args, cudaStream_t stream);
 
 }  // namespace symar

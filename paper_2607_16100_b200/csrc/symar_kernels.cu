@@ -1,71 +1,44 @@
-// The three AllReduce kernels.  One launch emulates all P ranks: blockIdx.y is
-// the rank, blockIdx.x the CTA slot of that rank.  CTAs of different ranks meet
-// only through the symmetric heap, as GPUs of one NVLink domain would.
+// The AllReduce kernels built from per-thread loads and stores.  One launch
+// emulates all P ranks: blockIdx.y is the rank, blockIdx.x the CTA slot of that
+// rank.  CTAs of different ranks meet only through the symmetric heap, as GPUs
+// of one NVLink domain would.
 //
-//   oneshot_kernel  Sec. III-A.1 (pull): exchange "input ready" flags with every
-//                   peer, read all P inputs, reduce, write the own output.
-//   twoshot_kernel  Sec. III-A.2: the same exchange, reduce only the own chunk,
-//                   store it into every rank's output (all-gather from
-//                   registers), then hand off with "chunk done" flags.
+//   oneshot_kernel  Sec. III-A.1 (pull): exchange "input ready" signals with
+//                   every peer, read all P inputs, reduce, write the own output.
+//   twoshot_kernel  Sec. III-A.2: the same exchange, reduce only the owned
+//                   vectors, store them into every rank's output (all-gather
+//                   from registers), then hand off with "done" signals.
 //   ll_kernel       Sec. IV "LL" + Sec. V example kernel: push every input word
 //                   to every peer's scratch as {payload, flag} 8-byte stores,
 //                   poll the own scratch, reduce, write the own output; scratch
 //                   is double-buffered by iteration parity.
 //
+// (The two-shot kernel for the bandwidth regime, built on bulk asynchronous
+// copies, lives in symar_bulk.cu.)
+//
 // No kernel contains a grid-wide barrier; every wait is one-directional (a CTA
-// waits for data or a flag FROM each peer) and bounded.
+// waits for data or a signal FROM each peer) and bounded.
 #include "symar_device.cuh"
 #include "symar_internal.h"
 
 namespace symar {
-
-// "Input ready" exchange shared by one-shot and two-shot (one synchronisation,
-// Table I).  Lane q of warp 0 raises this rank's flag at peer q; then every
-// warp polls the P flags of its own rank with lane q watching peer q, so all P
-// polls are in flight together.  Returns false if the wait ran out.
-template <int P, bool DBG>
-__device__ __forceinline__ bool exchange_flags(const KArgs &a, uint64_t flags_off, int r, int c,
-                                               uint32_t e, bool muted, bool all_warps)
-{
-    const uint32_t t    = threadIdx.x;
-    const uint32_t lane = t & 31u;
-    if (t < P && !muted) {
-        uint32_t *dst =
-            reinterpret_cast<uint32_t *>(a.seg0 + t * a.stride + flags_off + (size_t)c * kFlagGroup) + r;
-        st_release_u32(dst, e);
-    }
-    if (P == 1) return true;
-    if (!all_warps && t >= 32) return true;
-    const uint32_t *mine =
-        reinterpret_cast<const uint32_t *>(a.seg0 + (size_t)r * a.stride + flags_off + (size_t)c * kFlagGroup) +
-        (lane < P ? lane : 0);
-    Spin spin;
-    for (;;) {
-        const uint32_t f = ld_acquire_u32(mine);
-        const unsigned late = __ballot_sync(0xffffffffu, lane < P && f != e);
-        if (late == 0) return true;
-        if (spin.due()) {
-            if (__any_sync(0xffffffffu, spin.expired(a.spin_ns))) {
-                if (lane == 0) report_timeout(a.ctl, r, __ffs(late) - 1, c);
-                return false;
-            }
-        }
-    }
-}
 
 template <typename E, int P, bool DBG>
 __global__ void __launch_bounds__(kMaxThreads) oneshot_kernel(const KArgs a)
 {
     const int c = blockIdx.x, r = blockIdx.y, C = gridDim.x;
     const uint32_t t = threadIdx.x, T = blockDim.x;
-    char *seg_r  = a.seg0 + (size_t)r * a.stride;
-    uint64_t *ep = reinterpret_cast<uint64_t *>(seg_r + a.epoch_off) + c;
-    const uint64_t n = ld_relaxed_u64(ep) + 1;   // this call's iteration number of slot c
+    char *seg_r = a.seg0 + (size_t)r * a.stride;
+    uint32_t *count = reinterpret_cast<uint32_t *>(seg_r + a.epoch_off + ready_count_off(c));
     if (DBG) debug_delay(a, r, c);
-    const bool muted = DBG && a.dbg_mute == r;
+    if (DBG && a.dbg_mute == r) return;       // test hook: this rank never joins
 
-    const bool ok = exchange_flags<P, DBG>(a, a.ready_off, r, c, flag_of(n), muted, true);
-
+    uint32_t want;
+    const bool ok = flag_exchange<P, false>(a, a.ready_off, count, r, c, false, true, want);
+    // Every warp has consumed the count; publish the next one now so that its
+    // store drains while the data is in flight.
+    __syncthreads();
+    if (t == 0) *count = want;
     if (ok) {
         char *out = seg_r + a.out_off;
         for (uint64_t v = (uint64_t)c * T + t; v < a.nvec; v += (uint64_t)C * T) {
@@ -75,8 +48,26 @@ __global__ void __launch_bounds__(kMaxThreads) oneshot_kernel(const KArgs a)
             store_result(out, v, reduce_in_rank_order<E, P>(x), a.nvec, a.tail_bytes);
         }
     }
-    __syncthreads();          // every thread has read the counter before it moves
-    if (t == 0) *ep = n;
+}
+
+// The same for two adjacent vectors moved as one 32-byte access per peer.
+template <typename E, int P>
+__device__ __forceinline__ void twoshot_vector_pair(const KArgs &a, uint64_t v)
+{
+    U32B x[P];
+#pragma unroll
+    for (int q = 0; q < P; ++q) x[q] = ld_peer_32B(a.seg0 + (size_t)q * a.stride + a.in_off + v * 16);
+    uint4 lo[P], hi[P];
+#pragma unroll
+    for (int q = 0; q < P; ++q) {
+        lo[q] = x[q].lo;
+        hi[q] = x[q].hi;
+    }
+    U32B res;
+    res.lo = reduce_in_rank_order<E, P>(lo);
+    res.hi = reduce_in_rank_order<E, P>(hi);
+#pragma unroll
+    for (int q = 0; q < P; ++q) st_output_32B(a.seg0 + (size_t)q * a.stride + a.out_off + v * 16, res);
 }
 
 template <typename E, int P, bool DBG>
@@ -84,35 +75,60 @@ __global__ void __launch_bounds__(kMaxThreads) twoshot_kernel(const KArgs a)
 {
     const int c = blockIdx.x, r = blockIdx.y, C = gridDim.x;
     const uint32_t t = threadIdx.x, T = blockDim.x;
-    char *seg_r  = a.seg0 + (size_t)r * a.stride;
-    uint64_t *ep = reinterpret_cast<uint64_t *>(seg_r + a.epoch_off) + c;
-    const uint64_t n = ld_relaxed_u64(ep) + 1;
+    char *seg_r = a.seg0 + (size_t)r * a.stride;
+    uint32_t *rcount = reinterpret_cast<uint32_t *>(seg_r + a.epoch_off + ready_count_off(c));
+    uint32_t *dcount = reinterpret_cast<uint32_t *>(seg_r + a.epoch_off + done_count_off(c));
     if (DBG) debug_delay(a, r, c);
-    const bool muted  = DBG && a.dbg_mute == r;
-    const uint32_t e  = flag_of(n);
+    if (DBG && a.dbg_mute == r) return;       // test hook: this rank never joins
 
-    // reduce-scatter: rank r owns chunk r = vectors [lo, hi)
-    bool ok = exchange_flags<P, DBG>(a, a.ready_off, r, c, e, muted, true);
+    // reduce-scatter: which vectors rank r owns
+    uint32_t rwant, dwant;
+    bool ok = flag_exchange<P, false>(a, a.ready_off, rcount, r, c, false, true, rwant);
     if (ok) {
-        const uint64_t chv = (a.nvec + P - 1) / P;
-        const uint64_t lo  = (uint64_t)r * chv;
-        const uint64_t hi  = (lo + chv < a.nvec) ? lo + chv : a.nvec;
-        for (uint64_t v = lo + (uint64_t)c * T + t; v < hi; v += (uint64_t)C * T) {
-            uint4 x[P];
-#pragma unroll
-            for (int q = 0; q < P; ++q) x[q] = ld_peer(a.seg0 + (size_t)q * a.stride + a.in_off + v * 16);
-            const uint4 res = reduce_in_rank_order<E, P>(x);
-            // all-gather straight from registers into every rank's output
-#pragma unroll
-            for (int q = 0; q < P; ++q)
-                store_result(a.seg0 + (size_t)q * a.stride + a.out_off, v, res, a.nvec, a.tail_bytes);
+        const uint64_t step = (uint64_t)C * T;
+        if (a.blk_log2 == kOneChunk) {
+            // small and medium messages: rank r owns the contiguous chunk r
+            const uint64_t chv = (a.nvec + P - 1) / P;
+            const uint64_t lo  = (uint64_t)r * chv;
+            const uint64_t hi  = (lo + chv < a.nvec) ? lo + chv : a.nvec;
+            for (uint64_t v = lo + (uint64_t)c * T + t; v < hi; v += step) twoshot_vector<E, P>(a, v);
+        } else {
+            // large messages: blocks of 2^blk_log2 vectors are dealt to the ranks
+            // round-robin, so that at any moment all P * C CTAs stream through the
+            // same neighbourhood of each buffer (fewer open DRAM pages than P
+            // far-apart chunks).  Rank r owns blocks r, r + P, r + 2P, ...
+            const uint32_t sh   = a.blk_log2;
+            const uint64_t nblk = (a.nvec + (1ull << sh) - 1) >> sh;
+            const uint64_t mine = (nblk + P - 1 - r) / P;
+            if (a.wide) {
+                const uint64_t total = mine << (sh - 1);            // 32-byte steps
+                const uint64_t mask  = (1ull << (sh - 1)) - 1;
+                for (uint64_t w = (uint64_t)c * T + t; w < total; w += step) {
+                    const uint64_t v = (((w >> (sh - 1)) * P + r) << sh) + 2 * (w & mask);
+                    if (v + 2 < a.nvec) twoshot_vector_pair<E, P>(a, v);   // never the (maybe partial) last vector
+                    else {
+                        if (v < a.nvec) twoshot_vector<E, P>(a, v);
+                        if (v + 1 < a.nvec) twoshot_vector<E, P>(a, v + 1);
+                    }
+                }
+            } else {
+                const uint64_t total = mine << sh;
+                const uint64_t mask  = (1ull << sh) - 1;
+                for (uint64_t w = (uint64_t)c * T + t; w < total; w += step) {
+                    const uint64_t v = (((w >> sh) * P + r) << sh) + (w & mask);
+                    if (v < a.nvec) twoshot_vector<E, P>(a, v);
+                }
+            }
         }
     }
-    // handoff: this CTA's part of chunk r has landed everywhere -> tell every
-    // peer; then wait until every peer's CTA c has delivered its part here.
+    // handoff: this CTA's part of rank r's vectors has landed everywhere -> tell
+    // every peer; then wait until every peer's CTA c has delivered its part here.
     __syncthreads();
-    if (ok) ok = exchange_flags<P, DBG>(a, a.done_off, r, c, e, muted, false);
-    if (t == 0) *ep = n;
+    flag_exchange<P, true>(a, a.done_off, dcount, r, c, !ok, false, dwant);
+    if (t == 0) {
+        *rcount = rwant;
+        *dcount = dwant;
+    }
 }
 
 template <typename E, int P, bool DBG>
@@ -124,11 +140,12 @@ __global__ void __launch_bounds__(kMaxThreads) ll_kernel(const KArgs a)
     uint64_t *ep = reinterpret_cast<uint64_t *>(seg_r + a.epoch_off) + c;
     const uint64_t n0 = ld_relaxed_u64(ep);
     if (DBG) debug_delay(a, r, c);
-    const bool muted = DBG && a.dbg_mute == r;
+    if (DBG && a.dbg_mute == r) return;       // test hook: this rank never joins
 
     const char *in = seg_r + a.in_off;
     char *out      = seg_r + a.out_off;
     bool failed    = false;
+    uint4 kept     = make_uint4(0u, 0u, 0u, 0u);   // own vector of the first trip stays in registers
 
     for (uint32_t it = 0; it < a.iters && !failed; ++it) {
         const uint64_t n   = n0 + 1 + it;            // advanceEpoch: flag value and sub-buffer
@@ -138,51 +155,60 @@ __global__ void __launch_bounds__(kMaxThreads) ll_kernel(const KArgs a)
         const uint64_t region = a.ll_off + ((uint64_t)(n & 1) * kLLSlots + c) * P * kLLSenderBytes;
         const uint64_t hi_e   = (uint64_t)e << 32;
 
-        // bcast: {payload word, flag} pairs into every rank's scratch, sender row r
-        if (!muted) {
-            for (uint32_t k = t; k < cnt; k += T) {
-                const uint4 x = ld_own(in + (v0 + k) * 16);
-                const uint64_t d0 = hi_e | x.x, d1 = hi_e | x.y, d2 = hi_e | x.z, d3 = hi_e | x.w;
+        // bcast: {payload word, flag} pairs into every PEER's scratch, sender row r.
+        // The own contribution stays in registers (same bits as a round trip
+        // through the own scratch row would return).
+        for (uint32_t k = t; k < cnt; k += T) {
+            const uint4 x = ld_own(in + (v0 + k) * 16);
+            if (k == t) kept = x;
+            const uint64_t d0 = hi_e | x.x, d1 = hi_e | x.y, d2 = hi_e | x.z, d3 = hi_e | x.w;
 #pragma unroll
-                for (int q = 0; q < P; ++q) {
-                    char *dst = a.seg0 + (size_t)q * a.stride + region + (size_t)r * kLLSenderBytes + (size_t)k * 16;
-                    st_relaxed_v2u64(dst, d0, d1);
-                    st_relaxed_v2u64(dst + (size_t)kLLSlotVecs * 16, d2, d3);
-                }
+            for (int q = 0; q < P; ++q) {
+                if (q == r) continue;
+                char *dst = a.seg0 + (size_t)q * a.stride + region + (size_t)r * kLLSenderBytes + (size_t)k * 16;
+                st_relaxed_v2u64(dst, d0, d1);
+                st_relaxed_v2u64(dst + (size_t)kLLSlotVecs * 16, d2, d3);
             }
         }
-        // recvReduce: poll all P sender rows together until every flag matches
+        // recvReduce: poll the P-1 peer rows together; a row that has arrived is
+        // not polled again
         for (uint32_t k = t; k < cnt && !failed; k += T) {
             const char *src = seg_r + region + (size_t)k * 16;
-            U64x2 lo[P], hi[P];
+            uint4 x[P];
+            const uint4 own = (k == t) ? kept : ld_own(in + (v0 + k) * 16);
+            unsigned need   = ((1u << P) - 1u) & ~(1u << r);
             Spin spin;
-            for (;;) {
-                bool ready = true;
+            while (need != 0) {
+                U64x2 lo[P], hi[P];
 #pragma unroll
                 for (int q = 0; q < P; ++q) {
-                    lo[q] = ld_relaxed_v2u64(src + (size_t)q * kLLSenderBytes);
-                    hi[q] = ld_relaxed_v2u64(src + (size_t)q * kLLSenderBytes + (size_t)kLLSlotVecs * 16);
+                    if (need >> q & 1u) {
+                        lo[q] = ld_relaxed_v2u64(src + (size_t)q * kLLSenderBytes);
+                        hi[q] = ld_relaxed_v2u64(src + (size_t)q * kLLSenderBytes + (size_t)kLLSlotVecs * 16);
+                    }
                 }
 #pragma unroll
-                for (int q = 0; q < P; ++q)
-                    ready = ready && (uint32_t)(lo[q].a >> 32) == e && (uint32_t)(lo[q].b >> 32) == e &&
-                            (uint32_t)(hi[q].a >> 32) == e && (uint32_t)(hi[q].b >> 32) == e;
-                if (ready) break;
-                if (spin.due() && spin.expired(a.spin_ns)) {
-                    int late = 0;
-#pragma unroll
-                    for (int q = P - 1; q >= 0; --q)
-                        if ((uint32_t)(lo[q].a >> 32) != e || (uint32_t)(hi[q].b >> 32) != e) late = q;
-                    report_timeout(a.ctl, r, late, c);
+                for (int q = 0; q < P; ++q) {
+                    if (need >> q & 1u) {
+                        const bool here = (uint32_t)(lo[q].a >> 32) == e && (uint32_t)(lo[q].b >> 32) == e &&
+                                          (uint32_t)(hi[q].a >> 32) == e && (uint32_t)(hi[q].b >> 32) == e;
+                        if (here) {
+                            x[q] = make_uint4((uint32_t)lo[q].a, (uint32_t)lo[q].b, (uint32_t)hi[q].a,
+                                              (uint32_t)hi[q].b);
+                            need &= ~(1u << q);
+                        }
+                    }
+                }
+                if (need != 0 && spin.due() && spin.expired(a.spin_ns)) {
+                    report_timeout(a.ctl, r, __ffs(need) - 1, c);
                     failed = true;
                     break;
                 }
             }
             if (failed) break;
-            uint4 x[P];
 #pragma unroll
             for (int q = 0; q < P; ++q)
-                x[q] = make_uint4((uint32_t)lo[q].a, (uint32_t)lo[q].b, (uint32_t)hi[q].a, (uint32_t)hi[q].b);
+                if (q == r) x[q] = own;
             store_result(out, v0 + k, reduce_in_rank_order<E, P>(x), a.nvec, a.tail_bytes);
         }
         // No CTA barrier between iterations: position k is sent and received by
@@ -191,7 +217,7 @@ __global__ void __launch_bounds__(kMaxThreads) ll_kernel(const KArgs a)
         // thread's send of iteration i, issued after that thread's receive of
         // iteration i-1 -- so the sub-buffer of parity (i+1)&1 is free.
     }
-    __syncthreads();
+    __syncthreads();          // every thread has read the counter before it moves
     if (t == 0) *ep = n0 + a.iters;
 }
 
@@ -227,10 +253,10 @@ KernelFn kernel_for(int algo, int dtype, int P, bool dbg)
     return nullptr;
 }
 
-cudaError_t launch_kernel(KernelFn fn, int P, int ctas_per_rank, int threads, const KArgs &args,
-                          cudaStream_t stream)
+cudaError_t launch_kernel(KernelFn fn, int P, int ctas_per_rank, int threads, size_t smem_bytes,
+                          const KArgs &args, cudaStream_t stream)
 {
-    fn<<<dim3((unsigned)ctas_per_rank, (unsigned)P, 1), dim3((unsigned)threads, 1, 1), 0, stream>>>(args);
+    fn<<<dim3((unsigned)ctas_per_rank, (unsigned)P, 1), dim3((unsigned)threads, 1, 1), smem_bytes, stream>>>(args);
     return cudaGetLastError();
 }
 

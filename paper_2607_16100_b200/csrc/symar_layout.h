@@ -5,7 +5,7 @@
 // segment q  :  [ user region | LL scratch | ready flags | done flags | epochs | pad ]
 //
 // Every rank segment has the same layout (symmetric objects: same offset + rank
-// id addresses a peer's copy), every region starts on a 256-byte boundary.
+// id addresses a peer's copy), every region starts on a 4 KiB boundary.
 //
 // LL scratch of the RECEIVING rank, indexed [parity][slot c][sender q][half][k]:
 //   parity  alternates with the slot's iteration counter (double buffering: a
@@ -28,9 +28,32 @@ constexpr int      kMaxCtas     = SYMAR_MAX_CTAS;
 constexpr int      kLLSlots     = SYMAR_LL_SLOTS;
 constexpr uint32_t kLLSlotVecs  = SYMAR_LL_SLOT_VECS;
 constexpr size_t   kAlign       = SYMAR_ALIGN;
-constexpr size_t   kCtlBytes    = 256;              // control block at the heap base
+constexpr size_t   kCtlBytes    = SYMAR_ALIGN;      // control block at the heap base
 constexpr size_t   kFlagGroup   = 32;               // kMaxRanks x u32: one L2 sector per (rank, slot)
 constexpr size_t   kMaxThreads  = 512;
+
+// byte offsets of the two u32 exchange counters of slot c, relative to epoch_off
+__host__ __device__ constexpr size_t ready_count_off(int c) { return (size_t)kMaxCtas * 8 + (size_t)c * 4; }
+__host__ __device__ constexpr size_t done_count_off(int c) { return (size_t)kMaxCtas * 12 + (size_t)c * 4; }
+
+// variant bits (performance experiments; same results)
+enum : uint32_t {
+    kVarLateCount = 1u,    // one-shot: publish the exchange count at kernel exit instead of
+                           // right after the exchange
+};
+
+constexpr uint32_t kOneChunk     = 0xffu;   // KArgs::blk_log2: rank r owns one contiguous chunk
+constexpr uint32_t kCyclicLog2   = 9;       // block-cyclic block: 512 vectors = 8 KiB
+constexpr uint64_t kCyclicMinVec = 1u << 16;   // vectors per rank (1 MiB) from which blocks are dealt round-robin
+
+// bulk two-shot (bandwidth regime)
+constexpr uint64_t kBulkMinVec   = 1u << 18;   // vectors per rank (4 MiB) from which it is used
+constexpr uint32_t kBulkOutBufs  = 3;          // output tiles cycling through shared memory
+constexpr size_t   kBulkBarBytes = 128;        // mbarriers at the start of dynamic shared memory
+__host__ __device__ constexpr size_t bulk_smem_bytes(int P, uint32_t tile_vecs, uint32_t stages)
+{
+    return kBulkBarBytes + ((size_t)stages * P + kBulkOutBufs) * tile_vecs * 16;
+}
 
 // control block words (u32)
 enum : int { kCtlCode = 0, kCtlRank = 1, kCtlPeer = 2, kCtlCta = 3 };
@@ -44,7 +67,8 @@ struct Layout {
     size_t   ll_bytes;
     size_t   ready_off;      // kMaxCtas groups of kFlagGroup bytes
     size_t   done_off;
-    size_t   epoch_off;      // kMaxCtas x u64 iteration counters
+    size_t   epoch_off;      // kMaxCtas x u64 LL iteration counters, then kMaxCtas x u32
+                             // "ready" exchange counters, then kMaxCtas x u32 "done" counters
     size_t   seg_bytes;      // used bytes of a segment
     size_t   stride;         // segment pitch
     size_t   total;          // control block + P * stride
@@ -63,10 +87,10 @@ inline Layout make_layout(int P, size_t bytes_per_rank)
     L.ready_off  = L.ll_off + L.ll_bytes;
     L.done_off   = L.ready_off + (size_t)kMaxCtas * kFlagGroup;
     L.epoch_off  = L.done_off + (size_t)kMaxCtas * kFlagGroup;
-    L.seg_bytes  = round_up(L.epoch_off + (size_t)kMaxCtas * sizeof(uint64_t), kAlign);
-    // Pitch: pad by an odd number of 256-byte units so that equal offsets of
-    // different ranks do not all start on the same DRAM channel/bank set.
-    L.stride     = L.seg_bytes + 9 * kAlign;
+    L.seg_bytes  = round_up(L.epoch_off + (size_t)kMaxCtas * (sizeof(uint64_t) + 2 * sizeof(uint32_t)), kAlign);
+    // Pitch: two spare pages, so that the pitch is not a large power of two while
+    // every segment still starts on a page boundary.
+    L.stride     = L.seg_bytes + 2 * kAlign;
     L.total      = kCtlBytes + (size_t)P * L.stride;
     return L;
 }
@@ -88,6 +112,11 @@ struct KArgs {
     uint32_t  tail_bytes;    // valid bytes of the last vector, 0 = the last vector is full
     uint32_t  cv;            // LL: vectors per CTA per iteration (<= kLLSlotVecs)
     uint32_t  iters;         // LL: iterations
+    uint32_t  blk_log2;      // two-shot: log2 of the block-cyclic block in vectors, or kOneChunk
+    uint32_t  wide;          // two-shot: 1 = 32-byte accesses (buffers 32-byte aligned)
+    uint32_t  tile_vecs;     // bulk two-shot: vectors per tile
+    uint32_t  stages;        // bulk two-shot: input tiles in flight per CTA
+    uint32_t  variant;       // implementation variant bits of the kernel (same results)
     int32_t   dbg_mute;      // test hook: rank that stays silent, -1 = none
     uint32_t  dbg_seed;
     uint32_t  dbg_delay_ns;

@@ -25,7 +25,7 @@ _ERR_NAMES = {
     ERR_TIMEOUT: "SYMAR_ERR_TIMEOUT", ERR_UNSUPPORTED: "SYMAR_ERR_UNSUPPORTED",
 }
 
-MAX_RANKS, MAX_CTAS, LL_SLOTS, LL_SLOT_VECS, ALIGN = 8, 160, 64, 1024, 256
+MAX_RANKS, MAX_CTAS, LL_SLOTS, LL_SLOT_VECS, ALIGN = 8, 160, 64, 1024, 4096
 
 # every symbol include/symar.h declares: (name, restype, argtypes)
 SIGNATURES = [
@@ -42,10 +42,12 @@ SIGNATURES = [
                                c_void_p]),
     ("allreduce_autotune", c_int, [c_void_p, c_int]),
     ("symar_last_choice", c_int, [c_void_p, POINTER(c_int), POINTER(c_int), POINTER(c_int)]),
+    ("symar_last_kernel", c_int, [c_void_p, POINTER(c_uint), POINTER(c_size_t)]),
     ("symar_query_choice", c_int, [c_void_p, c_size_t, c_int, POINTER(c_int), POINTER(c_int), POINTER(c_int)]),
     ("symar_tuned_entry", c_int, [c_void_p, c_int, c_int, c_int, POINTER(c_int), POINTER(c_int),
                                   POINTER(c_double)]),
     ("symar_set_launch", c_int, [c_void_p, c_int, c_int, c_int]),
+    ("symar_set_variant", c_int, [c_void_p, c_int, c_uint]),
     ("symar_set_spin_limit_us", c_int, [c_void_p, c_uint]),
     ("symar_debug_inject", c_int, [c_void_p, c_int, c_uint, c_uint]),
     ("symar_last_cuda_error", c_char_p, []),
@@ -224,6 +226,11 @@ class SymHeap:
         _ck(self._lib.symar_last_choice(self._h, byref(a), byref(c), byref(t)), "symar_last_choice")
         return a.value, c.value, t.value
 
+    def last_kernel(self):
+        v, sm = c_uint(), c_size_t()
+        _ck(self._lib.symar_last_kernel(self._h, byref(v), byref(sm)), "symar_last_kernel")
+        return v.value, sm.value
+
     def query_choice(self, count: int, dtype: int, algo: int = AUTO):
         a, c, t = c_int(algo), c_int(), c_int()
         _ck(self._lib.symar_query_choice(self._h, count, dtype, byref(a), byref(c), byref(t)),
@@ -239,6 +246,9 @@ class SymHeap:
 
     def set_launch(self, algo: int, ctas_per_rank: int, threads: int) -> None:
         _ck(self._lib.symar_set_launch(self._h, algo, ctas_per_rank, threads), "symar_set_launch")
+
+    def set_variant(self, algo: int, variant: int) -> None:
+        _ck(self._lib.symar_set_variant(self._h, algo, variant), "symar_set_variant")
 
     def set_spin_limit_us(self, us: int) -> None:
         _ck(self._lib.symar_set_spin_limit_us(self._h, us), "symar_set_spin_limit_us")

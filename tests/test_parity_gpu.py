@@ -146,6 +146,71 @@ def test_ll_many_iterations_alternate_subbuffers(heaps):
     assert_bits(got, O.allreduce(x))
 
 
+# ---- bandwidth regime: block-cyclic ownership, 32-byte accesses, bulk-copy pipeline ----
+
+@pytest.fixture(scope="module")
+def big_heaps():
+    hs = {P: symar.SymHeap.on_torch(P, 40 << 20) for P in (2, 4, 8)}
+    yield hs
+    torch.cuda.synchronize()
+    for h in hs.values():
+        h.destroy()
+
+
+def bulk_var(stages, tile_log2):
+    return (stages << 8) | (tile_log2 << 12)
+
+
+@pytest.mark.parametrize("P,dtype,count", [
+    (8, "f32", 1 << 20), (8, "f32", (1 << 20) + 1), (8, "f32", (1 << 20) + 2051), (8, "bf16", (1 << 21) + 5),
+    (8, "bf16", 3 * (1 << 20) + 4099), (4, "f32", (1 << 20) + 7), (2, "bf16", (1 << 21) + 8193),
+    (8, "f32", 4 * (1 << 20) + 3),
+])
+@pytest.mark.parametrize("variant,ctas,threads", [
+    (0, 0, 0),                       # defaults: bulk kernel, 64 KiB stage
+    (bulk_var(3, 0), 37, 256),       # 4 KiB tiles, three stages, two CTAs per SM
+    (bulk_var(2, 1), 7, 128),        # 8 KiB tiles, odd CTA count
+    (bulk_var(4, 0), 13, 512),
+    (bulk_var(2, 3), 3, 64),         # tile larger than shared memory allows: library shrinks it
+    (4, 37, 256),                    # register kernel: block-cyclic + 32-byte accesses
+    (4 | 2, 18, 512),                # register kernel: block-cyclic, 16-byte accesses
+    (4 | 1, 5, 96),                  # register kernel: one contiguous chunk per rank
+])
+def test_bandwidth_regime_paths(big_heaps, P, dtype, count, variant, ctas, threads):
+    h = big_heaps[P]
+    dist = "uniform" if dtype == "f32" else "normal"
+    x = synth.make_inputs(dist, dtype, P, count, seed=count + P)
+    out_off = 20 << 20
+    h.set_variant(symar.TWOSHOT, variant)
+    h.set_launch(symar.TWOSHOT, ctas, threads)
+    try:
+        got = run(h, x, DT[dtype], symar.TWOSHOT, in_off=0, out_off=out_off)
+        var, smem = h.last_kernel()
+        if not (variant & 4):
+            assert smem > 0, "the bulk-copy kernel should have been used"
+        else:
+            assert smem == 0
+    finally:
+        h.set_variant(symar.TWOSHOT, 0)
+        h.set_launch(symar.TWOSHOT, 0, 0)
+    assert_bits(got, O.allreduce(x), f"P={P} {dtype} count={count} variant={variant:#x}")
+
+
+def test_bandwidth_regime_unaligned_buffers(big_heaps):
+    # 16-byte (not 32-byte) aligned input and output: bulk copies still legal, the
+    # register kernel must fall back to 16-byte accesses
+    h = big_heaps[8]
+    count = (1 << 20) + 37
+    x = synth.make_inputs("uniform", "f32", 8, count, seed=4242)
+    for variant in (0, 4):
+        h.set_variant(symar.TWOSHOT, variant)
+        try:
+            got = run(h, x, symar.F32, symar.TWOSHOT, in_off=16, out_off=(20 << 20) + 48)
+        finally:
+            h.set_variant(symar.TWOSHOT, 0)
+        assert_bits(got, O.allreduce(x), f"variant {variant}")
+
+
 # ---- determinism, algorithm equality, interleaving stress ---------------------------
 
 def test_algorithms_agree_and_repeat(heaps):
