@@ -199,6 +199,44 @@ int symar_set_spin_limit_us(symheap_t *heap, unsigned int microseconds);
 int symar_debug_inject(symheap_t *heap, int mute_rank, unsigned int delay_seed,
                        unsigned int delay_max_ns);
 
+/* ---- AllReduce without any allocation ------------------------------------------
+ *
+ * (The paper has no counterpart of this entry point: its kernels take their
+ * scratch from NCCL's symmetric-memory allocator.)
+ *
+ * For callers that cannot allocate device memory -- code running with a frozen
+ * memory pool inside a serving loop, a plugin that was handed no allocator, code
+ * that may run while another thread captures a CUDA graph (an allocation would
+ * break the capture), or a deployment that fixes all device memory at start-up --
+ * and therefore cannot create a symmetric heap.  The caller passes plain device
+ * buffers; the LL protocol's scratch and its counters live in one file-scope
+ * __device__ array of about 8 MiB that every GPU which loads the library holds
+ * until the process exits.  This function and everything it calls allocate and
+ * free nothing (no cudaMalloc/cudaFree, no allocating library routine).
+ *
+ * in, out : device buffers of P rows; rank q's input is at in + q * rank_pitch_bytes,
+ *           rank r's output at out + r * rank_pitch_bytes.  16-byte aligned, as is
+ *           the pitch; the input rows and the output rows must not overlap.
+ * count   : elements per rank; count * element size may not exceed
+ *           SYMAR_STATIC_MAX_BYTES (else SYMAR_ERR_UNSUPPORTED -- use a heap).
+ *           0 is a no-op.  The result is the same bits as allreduce() gives.
+ * device_status : optional device word (may be NULL), owned by the caller; it is
+ *           cleared on the stream before the launch and set to SYMAR_ERR_TIMEOUT
+ *           if a bounded wait inside the kernel gave up.
+ * cuda_stream : the copy-free call enqueues one small memset (only if
+ *           device_status is given) and one kernel.
+ *
+ * Set-up: the first call on each device looks up the device address of the
+ * scratch array (with that device current) and loads the kernel; make that first
+ * call outside any stream capture.  Sharing: all calls on a device use the same
+ * array.  Its flags and counters are sequence numbers that are meant to persist
+ * from call to call, so nothing needs clearing between calls, but two calls
+ * that overlap on the GPU (different streams or host threads) race on it --
+ * serialise them.                                                               */
+enum { SYMAR_STATIC_MAX_BYTES = 32768 };
+int allreduce_static(const void *in, void *out, size_t rank_pitch_bytes, int P, size_t count,
+                     symar_dtype_t dtype, unsigned int *device_status, void *cuda_stream);
+
 /* Text of the last CUDA error seen by the library on this thread (host string). */
 const char *symar_last_cuda_error(void);
 

@@ -50,6 +50,7 @@ SIGNATURES = [
     ("symar_set_variant", c_int, [c_void_p, c_int, c_uint]),
     ("symar_set_spin_limit_us", c_int, [c_void_p, c_uint]),
     ("symar_debug_inject", c_int, [c_void_p, c_int, c_uint, c_uint]),
+    ("allreduce_static", c_int, [c_void_p, c_void_p, c_size_t, c_int, c_size_t, c_int, c_void_p, c_void_p]),
     ("symar_last_cuda_error", c_char_p, []),
     ("symar_probe_empty", c_int, [c_int, c_int, c_int, c_void_p]),
     ("symar_probe_fence", c_int, [c_int, POINTER(c_double)]),
@@ -255,6 +256,17 @@ class SymHeap:
 
     def debug_inject(self, mute_rank: int = -1, delay_seed: int = 0, delay_max_ns: int = 0) -> None:
         _ck(self._lib.symar_debug_inject(self._h, mute_rank, delay_seed, delay_max_ns), "symar_debug_inject")
+
+
+STATIC_MAX_BYTES = 32768
+
+
+def allreduce_static(in_ptr: int, out_ptr: int, rank_pitch_bytes: int, P: int, count: int, dtype: int,
+                     status_ptr: int = 0, stream: int = 0) -> int:
+    """AllReduce on plain device buffers with library-internal static scratch; the
+    library allocates nothing.  Returns the raw status code."""
+    return int(load().allreduce_static(in_ptr, out_ptr, rank_pitch_bytes, P, count, dtype,
+                                       status_ptr or None, stream))
 
 
 # -- probes --
