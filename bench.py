@@ -100,6 +100,24 @@ class ClockSampler:
 
 
 # ---------------------------------------------------------------------------------
+# multi-process plumbing (replicas only: no data-path collective)
+# ---------------------------------------------------------------------------------
+def max_over_ranks(dist, ms: float, device) -> float:
+    """Slowest rank's time: the job is as slow as its slowest replica."""
+    import torch
+    if dist is None or not dist.is_initialized() or dist.get_world_size() == 1:
+        return ms
+    t = torch.tensor([ms], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(units_per_rank_step: float, world: int, steps: int, total_ms: float) -> float:
+    """Aggregate throughput: every replica processed the same units in `total_ms`."""
+    return units_per_rank_step * world * steps / (total_ms * 1e-3)
+
+
+# ---------------------------------------------------------------------------------
 # reference arm: the CPU oracle on the host cores
 # ---------------------------------------------------------------------------------
 def run_reference(args):
@@ -187,11 +205,20 @@ def latency_suite(torch, symar, synth, hbm_gbs, quick=False):
 
     # speed-of-light parts (paper Sec. VI), measured here
     fence_ns = symar.probe_fence(20000)
-    try:
-        rt_ns = symar.probe_pingpong(20000)
-    except symar.SymarError as e:
-        rt_ns = float("nan")
-        out["pingpong_error"] = str(e)
+    # The flag round trip depends on where the two SMs sit on the two-die chip; the
+    # ranks of the AllReduce are spread over all of it.  Sample SM pairs at growing
+    # distance and use the median pair for the bound (min and max are reported).
+    pairs = []
+    for partner in (1, 2, 3, 5, 9, 17, 33, 49, 65, 73, 74, 81, 97, 113, 129, 147):
+        try:
+            ns, sm = symar.probe_pingpong_pair(partner, 10000)
+            pairs.append({"partner_block": partner, "smids": list(sm), "round_trip_us": ns / 1000.0})
+        except symar.SymarError:
+            pass
+    rts = sorted(p["round_trip_us"] for p in pairs)
+    rt_ns = 1000.0 * (rts[len(rts) // 2] if rts else float("nan"))
+    out["flag_round_trip_pairs"] = {"min_us": rts[0] if rts else None, "median_us": rt_ns / 1000.0,
+                                    "max_us": rts[-1] if rts else None, "pairs": pairs}
 
     def empty_floor(cx, py, T):
         g = graph_of(torch, stream, lambda k, s: symar.probe_empty(cx, py, T, s), K)
@@ -306,6 +333,7 @@ def main():
     ap.add_argument("--quick", action="store_true", help="fewer latency samples")
     ap.add_argument("--ctas", type=int, default=0)
     ap.add_argument("--threads", type=int, default=0)
+    ap.add_argument("--variant", type=lambda v: int(v, 0), default=0, help="two-shot kernel variant bits")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -346,6 +374,8 @@ def main():
         heap.write_rank(q, in_off, x[q])
     if args.ctas or args.threads:
         heap.set_launch(symar.TWOSHOT, args.ctas, args.threads)
+    if args.variant:
+        heap.set_variant(symar.TWOSHOT, args.variant)
     stream = torch.cuda.Stream()
     sh = stream.cuda_stream
     step = lambda: heap.allreduce(in_off, out_off, count, symar.F32, symar.TWOSHOT, sh)
@@ -354,6 +384,9 @@ def main():
         step()
     stream.synchronize()
     algo, ctas, threads = heap.last_choice()
+    variant, smem = heap.last_kernel()
+    kernel = "twoshot_bulk_kernel<F32, 8>" if smem else "twoshot_kernel<F32, 8>"
+    tile_kib = (4 << ((variant >> 12) & 3)) if smem else None
 
     sampler = ClockSampler(local)
     sampler.start()
@@ -378,11 +411,8 @@ def main():
     clocks = sampler.stop(t_begin, t_end)
     assert heap.status()[0] == symar.OK, f"device status {heap.status()}"
 
-    if world > 1:
-        t = torch.tensor([total_ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
-    value = algbytes * world * args.steps / (total_ms * 1e-3) / 1e9
+    total_ms = max_over_ranks(dist if world > 1 else None, total_ms, "cuda")
+    value = whole_job_value(algbytes, world, args.steps, total_ms) / 1e9
 
     # parity of what was just timed, on sampled positions (oracle element by element)
     from oracle import allreduce_oracle as O
@@ -407,6 +437,8 @@ def main():
             "workload": f"c4: P={P} emulated ranks, fp32, {count} elements ({M >> 20} MiB) per rank, U(-1,1), "
                         "two-shot reduce-scatter + all-gather; value = 2*P*M bytes / time",
             "P": P, "elements_per_rank": count, "algo": "twoshot", "ctas_per_rank": ctas, "threads": threads,
+            "kernel": kernel, "bulk_tile_KiB": tile_kib, "bulk_stages": ((variant >> 8) & 7) or None,
+            "dynamic_smem_bytes": smem,
             "l2": f"inputs {P * M >> 20} MiB + outputs {P * M >> 20} MiB per step, far larger than the 126 MB L2; "
                   "no flush needed",
             "multi_gpu": "replicas only (independent heaps, no exchange between GPUs)",
@@ -417,7 +449,7 @@ def main():
         "roofline": {
             "bound": "hbm", "achieved": algbytes / (float(per_launch_ms.mean()) * 1e-3) / 1e9, "peak": hbm_gbs,
             "unit": "GB/s", "frac": algbytes / (float(per_launch_ms.mean()) * 1e-3) / 1e9 / hbm_gbs,
-            "peak_source": peak_src, "kernel": "twoshot_kernel<F32, 8>",
+            "peak_source": peak_src, "kernel": kernel,
             "algorithmic_bytes_per_launch": algbytes,
             "launch_ms": {"mean": float(per_launch_ms.mean()), "min": float(per_launch_ms.min()),
                           "max": float(per_launch_ms.max())},
@@ -425,11 +457,11 @@ def main():
             "traffic": None,
         },
     }
-    traffic_note = ROOT / "profiles" / "twoshot_f32_p8_traffic.json"
-    if traffic_note.exists():
-        tn = json.loads(traffic_note.read_text())
-        line["roofline"]["traffic"] = tn["dram_bytes_per_launch_at_full_size"]
-        line["roofline"]["traffic_source"] = tn["source"]
+    traffic_note = ROOT / "profiles" / "twoshot_bulk_f32_p8_traffic.txt"
+    if traffic_note.exists() and smem and count == synth.WORKLOADS["c4"]["count"]:
+        kv = dict(l.split("=", 1) for l in traffic_note.read_text().splitlines() if "=" in l and not l.startswith("#"))
+        line["roofline"]["traffic"] = int(kv["dram_bytes_per_launch_at_full_size "].strip())
+        line["roofline"]["traffic_source"] = kv["source "].strip()
 
     # end to end through the host-buffer entry point
     if not args.no_e2e:
@@ -450,14 +482,11 @@ def main():
             b.record(stream)
         stream.synchronize()
         e_ms = a.elapsed_time(b)
-        if world > 1:
-            t = torch.tensor([e_ms], device="cuda", dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e_ms = float(t.item())
+        e_ms = max_over_ranks(dist if world > 1 else None, e_ms, "cuda")
         s0 = count // 2
         want = O.allreduce(np.ascontiguousarray(x[:, s0:s0 + 4096]))
         e2e_exact = bool(np.array_equal(hout.numpy()[:, s0:s0 + 4096].view(np.uint32), want.view(np.uint32)))
-        line["e2e"] = {"value": algbytes * world * e2e_steps / (e_ms * 1e-3) / 1e9, "unit": "GB/s",
+        line["e2e"] = {"value": whole_job_value(algbytes, world, e2e_steps, e_ms) / 1e9, "unit": "GB/s",
                        "h2d_bytes_per_step": P * M, "d2h_bytes_per_step": P * M, "steps": e2e_steps,
                        "ms_per_step": e_ms / e2e_steps, "bit_exact_sampled": e2e_exact,
                        "note": "allreduce_host(): pinned host inputs -> HBM, kernel, all P outputs -> pinned host"}

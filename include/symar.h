@@ -249,11 +249,18 @@ const char *symar_last_cuda_error(void);
  *                       outstanding store each (the paper's L_L2_RTT estimate);
  * symar_probe_pingpong  ns per round trip of one 4-byte flag bounced between
  *                       two CTAs on different SMs through L2 (the one-GPU
- *                       analogue of the paper's two-GPU ping-pong).
+ *                       analogue of the paper's two-GPU ping-pong); blocks 0
+ *                       and 1 of a 2-block launch, usually neighbouring SMs.
  * The last two are synchronous and write host doubles.                         */
 int symar_probe_empty(int grid_x, int grid_y, int block, void *cuda_stream);
 int symar_probe_fence(int iterations, double *host_ns_per_fence);
 int symar_probe_pingpong(int iterations, double *host_ns_per_round_trip);
+/* The same between block 0 and block `partner_block` of a (partner_block + 1)-block
+ * launch, i.e. between SMs that are farther apart the larger the partner index;
+ * host_smids (2 ints, may be NULL) receives the two SM ids.  The round trip
+ * depends on where the two SMs and the flag's L2 slice sit on the chip.        */
+int symar_probe_pingpong_pair(int iterations, int partner_block, double *host_ns_per_round_trip,
+                              int *host_smids);
 
 #ifdef __cplusplus
 }

@@ -50,13 +50,15 @@ constexpr unsigned kSpinLimit = 1u << 22;   // polls; far above any real round t
 
 // flags[0] is written by block 0 and watched by block 1; flags[32] the reverse
 // (separate 128-byte lines).  out[0] = ns, out[1] = 1 on timeout, out[2..3] = SM ids.
-__global__ void pingpong_kernel(unsigned *flags, int iters, unsigned long long *out)
+__global__ void pingpong_kernel(unsigned *flags, int iters, unsigned long long *out, int partner)
 {
+    // blocks other than 0 and `partner` only fill the SMs in between
+    if (blockIdx.x != 0 && (int)blockIdx.x != partner) return;
     unsigned smid;
     asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
     unsigned *mine   = flags + (blockIdx.x == 0 ? 0 : 32);
     unsigned *theirs = flags + (blockIdx.x == 0 ? 32 : 0);
-    out[2 + blockIdx.x] = smid;
+    out[2 + (blockIdx.x == 0 ? 0 : 1)] = smid;
     bool dead = false;
     unsigned long long t0 = 0;
     if (blockIdx.x == 0) {
@@ -115,21 +117,33 @@ int symar_probe_fence(int iterations, double *host_ns_per_fence)
     return SYMAR_OK;
 }
 
-int symar_probe_pingpong(int iterations, double *host_ns_per_round_trip)
+int symar_probe_pingpong_pair(int iterations, int partner_block, double *host_ns_per_round_trip,
+                              int *host_smids)
 {
-    if (iterations < 1 || !host_ns_per_round_trip) return SYMAR_ERR_INVAL;
+    if (iterations < 1 || partner_block < 1 || partner_block > 1023 || !host_ns_per_round_trip)
+        return SYMAR_ERR_INVAL;
     unsigned char *buf = nullptr;
     if (cudaMalloc(&buf, 1024) != cudaSuccess) return SYMAR_ERR_NOMEM;
     cudaMemset(buf, 0, 1024);
     unsigned long long h[4] = {0, 0, 0, 0};
-    pingpong_kernel<<<2, 1>>>((unsigned *)buf, iterations, (unsigned long long *)(buf + 512));
+    pingpong_kernel<<<partner_block + 1, 1>>>((unsigned *)buf, iterations, (unsigned long long *)(buf + 512),
+                                              partner_block);
     int rc = sync_and_fetch((unsigned long long *)(buf + 512), h, 4);
     cudaFree(buf);
     if (rc != SYMAR_OK) return rc;
     if (h[1] != 0) return SYMAR_ERR_TIMEOUT;
+    if (host_smids) {
+        host_smids[0] = (int)h[2];
+        host_smids[1] = (int)h[3];
+    }
     if (h[2] == h[3]) return SYMAR_ERR_UNSUPPORTED;   // both blocks landed on one SM: not an L2 round trip
     *host_ns_per_round_trip = (double)h[0] / iterations;
     return SYMAR_OK;
+}
+
+int symar_probe_pingpong(int iterations, double *host_ns_per_round_trip)
+{
+    return symar_probe_pingpong_pair(iterations, 1, host_ns_per_round_trip, nullptr);
 }
 
 }  // extern "C"

@@ -55,6 +55,7 @@ SIGNATURES = [
     ("symar_probe_empty", c_int, [c_int, c_int, c_int, c_void_p]),
     ("symar_probe_fence", c_int, [c_int, POINTER(c_double)]),
     ("symar_probe_pingpong", c_int, [c_int, POINTER(c_double)]),
+    ("symar_probe_pingpong_pair", c_int, [c_int, c_int, POINTER(c_double), POINTER(c_int)]),
 ]
 
 
@@ -285,3 +286,11 @@ def probe_pingpong(iterations: int = 20000) -> float:
     v = c_double()
     _ck(load().symar_probe_pingpong(iterations, byref(v)), "symar_probe_pingpong")
     return v.value
+
+
+def probe_pingpong_pair(partner_block: int, iterations: int = 20000):
+    """(ns per round trip, (smid0, smid1)) between block 0 and block `partner_block`."""
+    v = c_double()
+    sm = (c_int * 2)()
+    _ck(load().symar_probe_pingpong_pair(iterations, partner_block, byref(v), sm), "symar_probe_pingpong_pair")
+    return v.value, (sm[0], sm[1])
