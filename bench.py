@@ -195,7 +195,7 @@ def time_stream(torch, stream, enqueue, n, warm=50):
     return float(np.percentile(us, 50))
 
 
-def latency_suite(torch, symar, synth, hbm_gbs, quick=False):
+def latency_suite(torch, symar, synth, hbm_gbs, quick=False, autotune=True):
     """C2 (16 KiB vs SoL), C3 (sweep + selector), C5 (decode-step graph)."""
     from oracle import allreduce_oracle as O
     out = {}
@@ -220,14 +220,16 @@ def latency_suite(torch, symar, synth, hbm_gbs, quick=False):
     out["flag_round_trip_pairs"] = {"min_us": rts[0] if rts else None, "median_us": rt_ns / 1000.0,
                                     "max_us": rts[-1] if rts else None, "pairs": pairs}
 
-    def empty_floor(cx, py, T):
-        g = graph_of(torch, stream, lambda k, s: symar.probe_empty(cx, py, T, s), K)
+    def empty_floor(cx, py, T, pdl=False):
+        probe = symar.probe_empty_pdl if pdl else symar.probe_empty
+        g = graph_of(torch, stream, lambda k, s: probe(cx, py, T, s), K)
         return time_graph(torch, g, stream, K, reps)
 
     for P in (8, 4):
         h = symar.SymHeap.on_torch(P, 24 << 20)
         t0 = time.time()
-        h.autotune(symar.BF16)
+        if autotune:
+            h.autotune(symar.BF16)
         tune_s = time.time() - t0
         out_off = 12 << 20
         res = {"autotune_seconds": tune_s}
@@ -273,6 +275,43 @@ def latency_suite(torch, symar, synth, hbm_gbs, quick=False):
                 "paper_style_sol_us": (2 * fence_ns + rt_ns / 2) / 1000.0,
                 "fence_us": fence_ns / 1000.0,
             }
+            # the same with programmatic dependent launch, floor measured with the same attribute
+            h.set_pdl(True)
+            prow = bench_size(8192, (symar.AUTO,))["auto"]
+            h.set_pdl(False)
+            pfloor = empty_floor(prow["ctas_per_rank"], P, prow["threads"], pdl=True)
+            psol = pfloor["p50"] + rt_ns / 1000.0 + t_bytes_us
+            out["latency_16KB"]["with_programmatic_dependent_launch"] = {
+                "p50_us": prow["p50"], "algo": prow["algo"], "bit_exact": prow["bit_exact"],
+                "empty_launch_same_shape_us": pfloor["p50"], "sol_us": psol, "ratio_to_sol": prow["p50"] / psol}
+        # below the metric's sizes: where the data+flag protocol is meant to win (the
+        # paper's own zoom is at one 128-byte line per rank), and one cold-cache number
+        if P == 8:
+            small = []
+            for nbytes in (128, 1024, 4096):
+                row = bench_size(nbytes // 2, (symar.ONESHOT, symar.TWOSHOT, symar.LL, symar.AUTO))
+                fl = empty_floor(row["auto"]["ctas_per_rank"], P, row["auto"]["threads"])
+                s_ol = fl["p50"] + rt_ns / 1000.0 + 2 * P * nbytes / (hbm_gbs * 1e9) * 1e6
+                small.append({"bytes_per_rank": nbytes, "p50_us": {k: v["p50"] for k, v in row.items()},
+                              "selector": row["auto"]["algo"],
+                              "selector_shape": [row["auto"]["ctas_per_rank"], row["auto"]["threads"]],
+                              "sol_us": s_ol, "ratio_to_sol": row["auto"]["p50"] / s_ol,
+                              "bit_exact": all(v["bit_exact"] for v in row.values())})
+            out["small_messages"] = small
+            scrub = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+            cold = []
+            with torch.cuda.stream(stream):
+                for i in range(30):
+                    scrub.fill_(i & 0xFF)                      # evicts heap lines from L2
+                    a_, b_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    a_.record(stream)
+                    h.allreduce(0, out_off, 8192, symar.BF16, symar.AUTO, stream.cuda_stream)
+                    b_.record(stream)
+                    cold.append((a_, b_))
+            stream.synchronize()
+            out["latency_16KB"]["cold_l2_single_call_us_p50"] = float(np.percentile(
+                [a_.elapsed_time(b_) * 1000.0 for a_, b_ in cold], 50))
+            del scrub
         # C3: sweep
         if P == 8:
             sweep = []
@@ -312,7 +351,19 @@ def latency_suite(torch, symar, synth, hbm_gbs, quick=False):
         sol = floor["p50"] + rt_ns / 1000.0 + t_bytes_us
         res.update({"step_total_us_p50": r["p50"] * calls, "per_call_us": r, "sol_per_call_us": sol,
                     "ratio_to_sol": r["p50"] / sol, "algo": names[a], "ctas_per_rank": c, "threads": t,
-                    "bit_exact": exact, "calls": calls, "bytes_per_rank": nb})
+                    "bit_exact": exact, "calls": calls, "bytes_per_rank": nb,
+                    "cache_state": "every call has its own input and output (%d MiB touched per step): "
+                                   "mostly HBM-cold, unlike the warm 16 KiB number" % (2 * P * calls * nb >> 20)})
+        h.set_pdl(True)
+        gp = graph_of(torch, stream, lambda k, s: h.allreduce(k * nb, base_out + k * nb, count, symar.BF16,
+                                                              symar.AUTO, s), calls)
+        rp = time_graph(torch, gp, stream, calls, 60 if quick else 200)
+        h.set_pdl(False)
+        kchk = calls - 1
+        gotp = np.stack([h.read_rank(q, base_out + kchk * nb, count, np.uint16) for q in range(P)])
+        res["with_programmatic_dependent_launch"] = {
+            "step_total_us_p50": rp["p50"] * calls, "per_call_us": rp["p50"],
+            "bit_exact": bool(np.array_equal(gotp, O.allreduce(xs[kchk])))}
         out.setdefault("decode_trace", {})[f"P{P}"] = res
         stream.synchronize()
         h.destroy()
@@ -331,6 +382,8 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--quick", action="store_true", help="fewer latency samples")
+    ap.add_argument("--latency-only", action="store_true", help="skip the bandwidth workload (no `value`)")
+    ap.add_argument("--no-autotune", action="store_true", help="latency section with the built-in launch shapes")
     ap.add_argument("--ctas", type=int, default=0)
     ap.add_argument("--threads", type=int, default=0)
     ap.add_argument("--variant", type=lambda v: int(v, 0), default=0, help="two-shot kernel variant bits")
@@ -359,6 +412,17 @@ def main():
     from paper_2607_16100_b200 import symar, synth
 
     hbm_gbs, peak_src = peaks()
+    if args.latency_only:
+        if rank == 0:
+            line = {"metric": METRIC, "impl": "ours", "n_gpus": world, "data": "synthetic", "dtype": "bf16",
+                    "note": "latency section only"}
+            line.update(latency_suite(torch, symar, synth, hbm_gbs, quick=args.quick,
+                                      autotune=not args.no_autotune))
+            print(json.dumps(line))
+        if world > 1:
+            dist.barrier()
+            dist.destroy_process_group()
+        return
     w = dict(synth.WORKLOADS["c4"])
     if args.count:
         w["count"] = args.count
@@ -513,7 +577,7 @@ def main():
     del x
 
     if rank == 0 and not args.no_latency:
-        line.update(latency_suite(torch, symar, synth, hbm_gbs, quick=args.quick))
+        line.update(latency_suite(torch, symar, synth, hbm_gbs, quick=args.quick, autotune=not args.no_autotune))
 
     if world > 1:
         dist.barrier()

@@ -180,13 +180,21 @@ int symar_tuned_entry(const symheap_t *heap, symar_dtype_t dtype, int log2_bytes
 int symar_set_launch(symheap_t *heap, symar_algo_t algo, int ctas_per_rank, int threads);
 
 /* Implementation variant of one algorithm's kernel, for performance experiments;
- * every variant computes the same bits.  0 = default.  One-shot: bit 0 = publish
- * the exchange count at kernel exit instead of right after the exchange;
+ * every variant computes the same bits.  0 = back to the table/default choice;
+ * bit 31 alone forces the plain variant (all other bits 0).  One-shot: bits 8-9 = bytes
+ * per thread (0: 16, 1: 8, 2: 4); LL: bit 8 = 8 instead of 16 payload bytes per thread;
  * two-shot: bit 0 = contiguous chunks also for large messages (no block-cyclic
  * ownership), bit 1 = 16-byte instead of 32-byte accesses for large messages,
  * bit 2 = never use the bulk-copy kernel, bits 8-10 = its pipeline depth (0:
  * default), bits 12-13 = log2 of its tile size over 4 KiB.                        */
 int symar_set_variant(symheap_t *heap, symar_algo_t algo, unsigned int variant);
+
+/* Programmatic dependent launch (off by default).  When on, every allreduce() is
+ * launched so that the NEXT kernel of the stream may become resident while it
+ * still runs; each AllReduce kernel first waits until the previous grid of the
+ * stream has completed and its writes are visible, so results and ordering are
+ * unchanged -- only launch latency of back-to-back calls is hidden.            */
+int symar_set_pdl(symheap_t *heap, int enabled);
 
 /* Upper bound of any device-side wait, in microseconds (default 2 000 000). */
 int symar_set_spin_limit_us(symheap_t *heap, unsigned int microseconds);
@@ -253,6 +261,8 @@ const char *symar_last_cuda_error(void);
  *                       and 1 of a 2-block launch, usually neighbouring SMs.
  * The last two are synchronous and write host doubles.                         */
 int symar_probe_empty(int grid_x, int grid_y, int block, void *cuda_stream);
+/* the launch floor with programmatic dependent launch (see symar_set_pdl) */
+int symar_probe_empty_pdl(int grid_x, int grid_y, int block, void *cuda_stream);
 int symar_probe_fence(int iterations, double *host_ns_per_fence);
 int symar_probe_pingpong(int iterations, double *host_ns_per_round_trip);
 /* The same between block 0 and block `partner_block` of a (partner_block + 1)-block

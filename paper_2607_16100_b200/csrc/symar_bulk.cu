@@ -96,6 +96,7 @@ __global__ void __launch_bounds__(kMaxThreads) twoshot_bulk_kernel(const KArgs a
     }
     __syncthreads();
 
+    if (a.pdl) pdl_wait();                  // the previous call has left the heap
     uint32_t rwant, dwant;
     bool ok = flag_exchange<P, false>(a, a.ready_off, rcount, r, c, false, true, rwant);
     ok = __syncthreads_and(ok);            // the whole CTA enters the pipeline, or none of it

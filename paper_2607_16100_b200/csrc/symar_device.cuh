@@ -131,6 +131,14 @@ __device__ __forceinline__ uint64_t globaltimer_ns()
     return t;
 }
 
+// ---- programmatic dependent launch ------------------------------------------------
+// With the launch attribute set, the next kernel of the stream may be made
+// resident while this one still runs; it blocks in pdl_wait() until this grid
+// has completed and its writes are visible.  Without the attribute both calls
+// do nothing.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;"); }
+
 // ---- bounded waiting ------------------------------------------------------------
 // Counts polls in a register; every 256th poll reads the nanosecond timer.  The
 // first reading starts the clock, so the fast path never touches the timer.
@@ -165,7 +173,15 @@ static __device__ __noinline__ void report_timeout(uint32_t *ctl, int rank, int 
 // sent with the data is 1 + n mod (2^32 - 1): never 0 (0 = "never written"),
 // and consecutive iterations always differ in parity n & 1, also across the
 // 32-bit wrap.
-__device__ __forceinline__ uint32_t flag_of(uint64_t n) { return (uint32_t)(n % 0xffffffffull) + 1u; }
+// (2^32 = 1 mod 2^32 - 1, so the remainder is the folded sum of the two halves;
+// no 64-bit division on the critical path.)
+__device__ __forceinline__ uint32_t flag_of(uint64_t n)
+{
+    uint64_t x = (n & 0xffffffffull) + (n >> 32);      // < 2^33
+    x = (x & 0xffffffffull) + (x >> 32);               // <= 2^32
+    if (x >= 0xffffffffull) x -= 0xffffffffull;        // n mod (2^32 - 1)
+    return (uint32_t)x + 1u;
+}
 
 // ---- element types ---------------------------------------------------------------
 struct F32 {
@@ -222,6 +238,80 @@ __device__ __forceinline__ uint4 reduce_in_rank_order(const uint4 (&x)[P])
         for (int j = 0; j < E::kEpv; ++j) acc[j] = __fadd_rn(acc[j], t[j]);
     }
     return E::narrow(acc);
+}
+
+// ---- narrow units: W 32-bit words per thread (W = 1, 2 or 4) --------------------------
+// For small messages the per-thread instruction count, not bandwidth, sets the
+// latency; giving a thread 4 or 8 bytes instead of 16 shortens its unpack/add
+// chain and spreads the message over more warps.
+template <int W> struct Words { uint32_t w[W]; };
+
+template <int W>
+__device__ __forceinline__ Words<W> ld_peer_words(const void *p)
+{
+    Words<W> v;
+    if (W == 1)
+        asm volatile("ld.relaxed." SYMAR_SCOPE ".global.u32 %0, [%1];" : "=r"(v.w[0]) : "l"(p) : "memory");
+    else if (W == 2)
+        asm volatile("ld.relaxed." SYMAR_SCOPE ".global.v2.u32 {%0, %1}, [%2];"
+                     : "=r"(v.w[0]), "=r"(v.w[W > 1 ? 1 : 0])
+                     : "l"(p)
+                     : "memory");
+    else
+        asm volatile("ld.relaxed." SYMAR_SCOPE ".global.v4.u32 {%0, %1, %2, %3}, [%4];"
+                     : "=r"(v.w[0]), "=r"(v.w[W > 1 ? 1 : 0]), "=r"(v.w[W > 2 ? 2 : 0]), "=r"(v.w[W > 3 ? 3 : 0])
+                     : "l"(p)
+                     : "memory");
+    return v;
+}
+
+// rank-ordered binary32 sum of P units, one narrowing at the end
+template <typename E, int P, int W>
+__device__ __forceinline__ Words<W> reduce_words_in_rank_order(const Words<W> (&x)[P])
+{
+    Words<W> out;
+    if (E::kEpv == 4) {          // fp32: one element per word
+#pragma unroll
+        for (int i = 0; i < W; ++i) {
+            float acc = __uint_as_float(x[0].w[i]);
+#pragma unroll
+            for (int q = 1; q < P; ++q) acc = __fadd_rn(acc, __uint_as_float(x[q].w[i]));
+            out.w[i] = __float_as_uint(acc);
+        }
+    } else {                     // bf16: two elements per word, low half first
+#pragma unroll
+        for (int i = 0; i < W; ++i) {
+            float lo = __uint_as_float(x[0].w[i] << 16), hi = __uint_as_float(x[0].w[i] & 0xffff0000u);
+#pragma unroll
+            for (int q = 1; q < P; ++q) {
+                lo = __fadd_rn(lo, __uint_as_float(x[q].w[i] << 16));
+                hi = __fadd_rn(hi, __uint_as_float(x[q].w[i] & 0xffff0000u));
+            }
+            __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
+            out.w[i] = *reinterpret_cast<uint32_t *>(&h);
+        }
+    }
+    return out;
+}
+
+// store of a unit of which only `valid` bytes (a multiple of 2, 1..4W) belong to the message
+template <int W>
+__device__ __forceinline__ void store_words(char *dst, const Words<W> &v, uint32_t valid)
+{
+    if (valid >= 4u * W) {
+        if (W == 1) asm volatile("st.global.u32 [%0], %1;" ::"l"(dst), "r"(v.w[0]) : "memory");
+        else if (W == 2)
+            asm volatile("st.global.v2.u32 [%0], {%1, %2};" ::"l"(dst), "r"(v.w[0]), "r"(v.w[W > 1 ? 1 : 0]) : "memory");
+        else
+            asm volatile("st.global.v4.u32 [%0], {%1, %2, %3, %4};" ::"l"(dst), "r"(v.w[0]), "r"(v.w[W > 1 ? 1 : 0]),
+                         "r"(v.w[W > 2 ? 2 : 0]), "r"(v.w[W > 3 ? 3 : 0])
+                         : "memory");
+    } else {
+        uint16_t *d = reinterpret_cast<uint16_t *>(dst);
+#pragma unroll
+        for (int b = 0; b < 2 * W; ++b)
+            if ((uint32_t)(2 * b) < valid) d[b] = (uint16_t)(v.w[b >> 1] >> ((b & 1) * 16));
+    }
 }
 
 // Store of output vector v; the last vector of a message may be partial.  The

@@ -23,6 +23,23 @@
 
 namespace symar {
 
+// One-shot data phase with W words per thread: unit u covers bytes [4W u, 4W u + 4W).
+template <typename E, int P, int W>
+__device__ __forceinline__ void oneshot_units(const KArgs &a, char *out, uint64_t first, uint64_t step)
+{
+    const uint64_t bytes  = a.tail_bytes ? (a.nvec - 1) * 16 + a.tail_bytes : a.nvec * 16;
+    const uint64_t nunits = (bytes + 4 * W - 1) / (4 * W);
+    for (uint64_t u = first; u < nunits; u += step) {
+        Words<W> x[P];
+#pragma unroll
+        for (int q = 0; q < P; ++q)
+            x[q] = ld_peer_words<W>(a.seg0 + (size_t)q * a.stride + a.in_off + u * (4 * W));
+        const uint64_t left = bytes - u * (4 * W);
+        store_words<W>(out + u * (4 * W), reduce_words_in_rank_order<E, P, W>(x),
+                       left < 4u * W ? (uint32_t)left : 4u * W);
+    }
+}
+
 template <typename E, int P, bool DBG>
 __global__ void __launch_bounds__(kMaxThreads) oneshot_kernel(const KArgs a)
 {
@@ -30,6 +47,7 @@ __global__ void __launch_bounds__(kMaxThreads) oneshot_kernel(const KArgs a)
     const uint32_t t = threadIdx.x, T = blockDim.x;
     char *seg_r = a.seg0 + (size_t)r * a.stride;
     uint32_t *count = reinterpret_cast<uint32_t *>(seg_r + a.epoch_off + ready_count_off(c));
+    if (a.pdl) pdl_wait();                    // the previous call has left the heap
     if (DBG) debug_delay(a, r, c);
     if (DBG && a.dbg_mute == r) return;       // test hook: this rank never joins
 
@@ -39,13 +57,20 @@ __global__ void __launch_bounds__(kMaxThreads) oneshot_kernel(const KArgs a)
     // store drains while the data is in flight.
     __syncthreads();
     if (t == 0) *count = want;
+    if (a.pdl) pdl_launch_dependents();       // the next call may take its seats now
     if (ok) {
         char *out = seg_r + a.out_off;
-        for (uint64_t v = (uint64_t)c * T + t; v < a.nvec; v += (uint64_t)C * T) {
-            uint4 x[P];
+        const uint64_t first = (uint64_t)c * T + t, step = (uint64_t)C * T;
+        const uint32_t narrow = (a.variant >> 8) & 3u;     // bytes per thread: 16, 8 or 4
+        if (narrow == 2) oneshot_units<E, P, 1>(a, out, first, step);
+        else if (narrow == 1) oneshot_units<E, P, 2>(a, out, first, step);
+        else {
+            for (uint64_t v = first; v < a.nvec; v += step) {
+                uint4 x[P];
 #pragma unroll
-            for (int q = 0; q < P; ++q) x[q] = ld_peer(a.seg0 + (size_t)q * a.stride + a.in_off + v * 16);
-            store_result(out, v, reduce_in_rank_order<E, P>(x), a.nvec, a.tail_bytes);
+                for (int q = 0; q < P; ++q) x[q] = ld_peer(a.seg0 + (size_t)q * a.stride + a.in_off + v * 16);
+                store_result(out, v, reduce_in_rank_order<E, P>(x), a.nvec, a.tail_bytes);
+            }
         }
     }
 }
@@ -78,12 +103,14 @@ __global__ void __launch_bounds__(kMaxThreads) twoshot_kernel(const KArgs a)
     char *seg_r = a.seg0 + (size_t)r * a.stride;
     uint32_t *rcount = reinterpret_cast<uint32_t *>(seg_r + a.epoch_off + ready_count_off(c));
     uint32_t *dcount = reinterpret_cast<uint32_t *>(seg_r + a.epoch_off + done_count_off(c));
+    if (a.pdl) pdl_wait();                    // the previous call has left the heap
     if (DBG) debug_delay(a, r, c);
     if (DBG && a.dbg_mute == r) return;       // test hook: this rank never joins
 
     // reduce-scatter: which vectors rank r owns
     uint32_t rwant, dwant;
     bool ok = flag_exchange<P, false>(a, a.ready_off, rcount, r, c, false, true, rwant);
+    if (a.pdl) pdl_launch_dependents();
     if (ok) {
         const uint64_t step = (uint64_t)C * T;
         if (a.blk_log2 == kOneChunk) {
@@ -131,6 +158,83 @@ __global__ void __launch_bounds__(kMaxThreads) twoshot_kernel(const KArgs a)
     }
 }
 
+// LL with 8 bytes of payload per thread: one 16-byte {w0,f,w1,f} store per peer and
+// one 16-byte poll per peer and round.  Half the instructions per thread of the
+// 16-byte form and twice the threads; same scratch layout (unit u = half u&1 of
+// vector u>>1), so both forms can alternate on one heap.
+template <typename E, int P>
+__device__ __forceinline__ bool ll_iteration_narrow(const KArgs &a, int r, int c, uint32_t e, uint64_t region,
+                                                    uint64_t v0, uint32_t cnt, Words<2> &kept)
+{
+    const uint32_t t = threadIdx.x, T = blockDim.x;
+    char *seg_r       = a.seg0 + (size_t)r * a.stride;
+    const char *in    = seg_r + a.in_off;
+    char *out         = seg_r + a.out_off;
+    const uint64_t hi_e = (uint64_t)e << 32;
+    const uint32_t units = 2 * cnt;
+    // bytes of unit u that belong to the message (0 = the unit lies past its end)
+    auto valid_of = [&](uint32_t u) -> uint32_t {
+        const uint64_t v = v0 + (u >> 1);
+        const uint32_t vb = (a.tail_bytes != 0 && v == a.nvec - 1) ? a.tail_bytes : 16u;
+        const uint32_t lo = (u & 1u) * 8u;
+        return vb > lo ? (vb - lo < 8u ? vb - lo : 8u) : 0u;
+    };
+    for (uint32_t u = t; u < units; u += T) {
+        if (valid_of(u) == 0) continue;
+        const size_t off = (size_t)(u & 1u) * kLLSlotVecs * 16 + (size_t)(u >> 1) * 16;
+        Words<2> x;
+        asm volatile("ld.global.nc.L1::no_allocate.v2.u32 {%0, %1}, [%2];"
+                     : "=r"(x.w[0]), "=r"(x.w[1])
+                     : "l"(in + (v0 + (u >> 1)) * 16 + (u & 1u) * 8));
+        if (u == t) kept = x;
+        const uint64_t d0 = hi_e | x.w[0], d1 = hi_e | x.w[1];
+        char *dst = a.seg0 + region + (size_t)r * kLLSenderBytes + off;
+#pragma unroll
+        for (int q = 0; q < P; ++q) {
+            if (q != r) st_relaxed_v2u64(dst, d0, d1);
+            dst += a.stride;
+        }
+    }
+    for (uint32_t u = t; u < units; u += T) {
+        const uint32_t valid = valid_of(u);
+        if (valid == 0) continue;
+        const size_t off = (size_t)(u & 1u) * kLLSlotVecs * 16 + (size_t)(u >> 1) * 16;
+        const char *src  = seg_r + region + off;
+        Words<2> x[P];
+        unsigned need = ((1u << P) - 1u) & ~(1u << r);
+        Spin spin;
+        while (need != 0) {
+            U64x2 d[P];
+#pragma unroll
+            for (int q = 0; q < P; ++q)
+                if (need >> q & 1u) d[q] = ld_relaxed_v2u64(src + (size_t)q * kLLSenderBytes);
+#pragma unroll
+            for (int q = 0; q < P; ++q) {
+                if ((need >> q & 1u) && (uint32_t)(d[q].a >> 32) == e && (uint32_t)(d[q].b >> 32) == e) {
+                    x[q].w[0] = (uint32_t)d[q].a;
+                    x[q].w[1] = (uint32_t)d[q].b;
+                    need &= ~(1u << q);
+                }
+            }
+            if (need != 0 && spin.due() && spin.expired(a.spin_ns)) {
+                report_timeout(a.ctl, r, __ffs(need) - 1, c);
+                return false;
+            }
+        }
+        Words<2> own;
+        if (u == t) own = kept;
+        else
+            asm volatile("ld.global.nc.L1::no_allocate.v2.u32 {%0, %1}, [%2];"
+                         : "=r"(own.w[0]), "=r"(own.w[1])
+                         : "l"(in + (v0 + (u >> 1)) * 16 + (u & 1u) * 8));
+#pragma unroll
+        for (int q = 0; q < P; ++q)
+            if (q == r) x[q] = own;
+        store_words<2>(out + (v0 + (u >> 1)) * 16 + (u & 1u) * 8, reduce_words_in_rank_order<E, P, 2>(x), valid);
+    }
+    return true;
+}
+
 template <typename E, int P, bool DBG>
 __global__ void __launch_bounds__(kMaxThreads) ll_kernel(const KArgs a)
 {
@@ -138,6 +242,10 @@ __global__ void __launch_bounds__(kMaxThreads) ll_kernel(const KArgs a)
     const uint32_t t = threadIdx.x, T = blockDim.x;
     char *seg_r  = a.seg0 + (size_t)r * a.stride;
     uint64_t *ep = reinterpret_cast<uint64_t *>(seg_r + a.epoch_off) + c;
+    if (a.pdl) {
+        pdl_wait();                           // the previous call has left the heap
+        pdl_launch_dependents();
+    }
     const uint64_t n0 = ld_relaxed_u64(ep);
     if (DBG) debug_delay(a, r, c);
     if (DBG && a.dbg_mute == r) return;       // test hook: this rank never joins
@@ -146,6 +254,7 @@ __global__ void __launch_bounds__(kMaxThreads) ll_kernel(const KArgs a)
     char *out      = seg_r + a.out_off;
     bool failed    = false;
     uint4 kept     = make_uint4(0u, 0u, 0u, 0u);   // own vector of the first trip stays in registers
+    Words<2> kept2 = {{0u, 0u}};
 
     for (uint32_t it = 0; it < a.iters && !failed; ++it) {
         const uint64_t n   = n0 + 1 + it;            // advanceEpoch: flag value and sub-buffer
@@ -155,6 +264,10 @@ __global__ void __launch_bounds__(kMaxThreads) ll_kernel(const KArgs a)
         const uint64_t region = a.ll_off + ((uint64_t)(n & 1) * kLLSlots + c) * P * kLLSenderBytes;
         const uint64_t hi_e   = (uint64_t)e << 32;
 
+        if (a.variant & 0x100u) {            // 8 bytes of payload per thread
+            failed = !ll_iteration_narrow<E, P>(a, r, c, e, region, v0, cnt, kept2);
+            continue;
+        }
         // bcast: {payload word, flag} pairs into every PEER's scratch, sender row r.
         // The own contribution stays in registers (same bits as a round trip
         // through the own scratch row would return).
@@ -256,8 +369,21 @@ KernelFn kernel_for(int algo, int dtype, int P, bool dbg)
 cudaError_t launch_kernel(KernelFn fn, int P, int ctas_per_rank, int threads, size_t smem_bytes,
                           const KArgs &args, cudaStream_t stream)
 {
-    fn<<<dim3((unsigned)ctas_per_rank, (unsigned)P, 1), dim3((unsigned)threads, 1, 1), smem_bytes, stream>>>(args);
-    return cudaGetLastError();
+    if (!args.pdl) {
+        fn<<<dim3((unsigned)ctas_per_rank, (unsigned)P, 1), dim3((unsigned)threads, 1, 1), smem_bytes, stream>>>(args);
+        return cudaGetLastError();
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim          = dim3((unsigned)ctas_per_rank, (unsigned)P, 1);
+    cfg.blockDim         = dim3((unsigned)threads, 1, 1);
+    cfg.dynamicSmemBytes = smem_bytes;
+    cfg.stream           = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs    = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, fn, args);
 }
 
 }  // namespace symar

@@ -117,6 +117,7 @@ struct KArgs {
     uint32_t  tile_vecs;     // bulk two-shot: vectors per tile
     uint32_t  stages;        // bulk two-shot: input tiles in flight per CTA
     uint32_t  variant;       // implementation variant bits of the kernel (same results)
+    uint32_t  pdl;           // 1 = launched with programmatic dependent launch
     int32_t   dbg_mute;      // test hook: rank that stays silent, -1 = none
     uint32_t  dbg_seed;
     uint32_t  dbg_delay_ns;

@@ -33,6 +33,11 @@ __device__ __forceinline__ void st_relaxed(unsigned *p, unsigned v)
 }
 
 __global__ void empty_kernel() {}
+__global__ void empty_pdl_kernel()
+{
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;");
+}
 
 // out[0] = elapsed ns over `iters` store+fence pairs
 __global__ void fence_kernel(unsigned *scratch, int iters, unsigned long long *out)
@@ -99,6 +104,21 @@ int symar_probe_empty(int grid_x, int grid_y, int block, void *cuda_stream)
     if (grid_x < 1 || grid_y < 1 || block < 1 || block > 1024) return SYMAR_ERR_INVAL;
     empty_kernel<<<dim3(grid_x, grid_y, 1), block, 0, (cudaStream_t)cuda_stream>>>();
     return cudaGetLastError() == cudaSuccess ? SYMAR_OK : SYMAR_ERR_CUDA;
+}
+
+int symar_probe_empty_pdl(int grid_x, int grid_y, int block, void *cuda_stream)
+{
+    if (grid_x < 1 || grid_y < 1 || block < 1 || block > 1024) return SYMAR_ERR_INVAL;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim  = dim3(grid_x, grid_y, 1);
+    cfg.blockDim = dim3(block, 1, 1);
+    cfg.stream   = (cudaStream_t)cuda_stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs    = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, empty_pdl_kernel) == cudaSuccess ? SYMAR_OK : SYMAR_ERR_CUDA;
 }
 
 int symar_probe_fence(int iterations, double *host_ns_per_fence)

@@ -48,11 +48,13 @@ SIGNATURES = [
                                   POINTER(c_double)]),
     ("symar_set_launch", c_int, [c_void_p, c_int, c_int, c_int]),
     ("symar_set_variant", c_int, [c_void_p, c_int, c_uint]),
+    ("symar_set_pdl", c_int, [c_void_p, c_int]),
     ("symar_set_spin_limit_us", c_int, [c_void_p, c_uint]),
     ("symar_debug_inject", c_int, [c_void_p, c_int, c_uint, c_uint]),
     ("allreduce_static", c_int, [c_void_p, c_void_p, c_size_t, c_int, c_size_t, c_int, c_void_p, c_void_p]),
     ("symar_last_cuda_error", c_char_p, []),
     ("symar_probe_empty", c_int, [c_int, c_int, c_int, c_void_p]),
+    ("symar_probe_empty_pdl", c_int, [c_int, c_int, c_int, c_void_p]),
     ("symar_probe_fence", c_int, [c_int, POINTER(c_double)]),
     ("symar_probe_pingpong", c_int, [c_int, POINTER(c_double)]),
     ("symar_probe_pingpong_pair", c_int, [c_int, c_int, POINTER(c_double), POINTER(c_int)]),
@@ -252,6 +254,9 @@ class SymHeap:
     def set_variant(self, algo: int, variant: int) -> None:
         _ck(self._lib.symar_set_variant(self._h, algo, variant), "symar_set_variant")
 
+    def set_pdl(self, enabled: bool) -> None:
+        _ck(self._lib.symar_set_pdl(self._h, 1 if enabled else 0), "symar_set_pdl")
+
     def set_spin_limit_us(self, us: int) -> None:
         _ck(self._lib.symar_set_spin_limit_us(self._h, us), "symar_set_spin_limit_us")
 
@@ -274,6 +279,10 @@ def allreduce_static(in_ptr: int, out_ptr: int, rank_pitch_bytes: int, P: int, c
 
 def probe_empty(grid_x: int, grid_y: int, block: int, stream: int = 0) -> None:
     _ck(load().symar_probe_empty(grid_x, grid_y, block, stream), "symar_probe_empty")
+
+
+def probe_empty_pdl(grid_x: int, grid_y: int, block: int, stream: int = 0) -> None:
+    _ck(load().symar_probe_empty_pdl(grid_x, grid_y, block, stream), "symar_probe_empty_pdl")
 
 
 def probe_fence(iterations: int = 20000) -> float:

@@ -146,6 +146,42 @@ def test_ll_many_iterations_alternate_subbuffers(heaps):
     assert_bits(got, O.allreduce(x))
 
 
+FORCE_PLAIN = 1 << 31
+
+
+@pytest.mark.parametrize("count", [1, 2, 3, 5, 8, 9, 63, 64, 1023, 4099, 40001])
+@pytest.mark.parametrize("P,dtype,dist", [(8, "bf16", "normal"), (4, "f32", "uniform"), (2, "bf16", "normal"),
+                                          (1, "f32", "uniform")])
+@pytest.mark.parametrize("algo,variant", [(symar.ONESHOT, FORCE_PLAIN), (symar.ONESHOT, 0x100),
+                                          (symar.ONESHOT, 0x200), (symar.LL, FORCE_PLAIN), (symar.LL, 0x100)])
+def test_unit_width_variants(heaps, algo, variant, P, dtype, dist, count):
+    # 16, 8 or 4 bytes per thread: same bits, whatever the ragged tail
+    h = heaps[P]
+    x = synth.make_inputs(dist, dtype, P, count, seed=31 * count + P)
+    h.set_variant(algo, variant)
+    try:
+        got = run(h, x, DT[dtype], algo)
+        assert h.last_kernel()[0] == variant & 0x7FFFFFFF
+    finally:
+        h.set_variant(algo, 0)
+    assert_bits(got, O.allreduce(x), f"algo={algo} variant={variant:#x} P={P} {dtype} count={count}")
+
+
+def test_ll_narrow_many_iterations_and_mixed_widths(heaps):
+    # narrow and wide LL calls alternate on the same scratch; one CTA forces many iterations
+    h = heaps[8]
+    x = synth.make_inputs("normal", "bf16", 8, 100003, seed=77)
+    want = O.allreduce(x)
+    try:
+        for variant, ctas, threads in ((0x100, 1, 128), (FORCE_PLAIN, 2, 64), (0x100, 3, 512), (0x100, 64, 32)):
+            h.set_variant(symar.LL, variant)
+            h.set_launch(symar.LL, ctas, threads)
+            assert_bits(run(h, x, symar.BF16, symar.LL, poison=False), want, f"variant {variant:#x}")
+    finally:
+        h.set_variant(symar.LL, 0)
+        h.set_launch(symar.LL, 0, 0)
+
+
 # ---- bandwidth regime: block-cyclic ownership, 32-byte accesses, bulk-copy pipeline ----
 
 @pytest.fixture(scope="module")
@@ -282,6 +318,41 @@ def test_graph_capture_replays(heaps):
             want = O.allreduce(x)
             got = np.stack([h.read_rank(q, out0 + k * nbytes, count, np.uint16) for q in range(8)])
             assert_bits(got, want, f"replay {rep} call {k}")
+
+
+def test_programmatic_dependent_launch_keeps_results_and_order(heaps):
+    # back-to-back calls whose input is the previous call's output: with the
+    # launch attribute on, each kernel may become resident early but must not
+    # touch the heap before its predecessor has finished
+    h = heaps[8]
+    count = 8192
+    nb = count * 2
+    x = synth.make_inputs("normal", "bf16", 8, count, seed=606)
+    for q in range(8):
+        h.write_rank(q, 0, x[q])
+    h.set_pdl(True)
+    try:
+        s = torch.cuda.Stream()
+        chain = [ALGOS[k % 3] for k in range(9)]
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=s):
+            for k, algo in enumerate(chain):
+                h.allreduce(k * nb, (k + 1) * nb, count, symar.BF16, algo, s.cuda_stream)
+        for rep in range(3):
+            g.replay()
+        torch.cuda.synchronize()
+        assert h.status()[0] == symar.OK
+        want = x
+        for k in range(len(chain)):
+            want = O.allreduce(want)            # every rank's next input is the previous result
+            got = np.stack([h.read_rank(q, (k + 1) * nb, count, np.uint16) for q in range(8)])
+            assert_bits(got, want, f"link {k}")
+        # stream-launched as well
+        for algo in ALGOS:
+            got = run(h, x, symar.BF16, algo, in_off=0, out_off=1 << 20, poison=False)
+            assert_bits(got, O.allreduce(x))
+    finally:
+        h.set_pdl(False)
 
 
 # ---- AUTO, autotune -----------------------------------------------------------------------
