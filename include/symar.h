@@ -20,6 +20,10 @@
  * that gives up records SYMAR_ERR_TIMEOUT in the heap's status word (read it
  * with symheap_status) and the kernel returns normally.
  *
+ * Environment (read when a heap is created): SYMAR_ALGO = oneshot | twoshot | ll
+ * replaces SYMAR_AUTO's choice; SYMAR_SPIN_LIMIT_US bounds device-side waits;
+ * SYMAR_PDL = 1 enables programmatic dependent launch.
+ *
  * Threading: a heap may be used from one host thread and one stream at a time
  * (the per-CTA epoch counters live in the heap).  Calls on one stream are
  * ordered by the stream.

@@ -5,6 +5,7 @@
 #include <algorithm>
 #include <cmath>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <map>
 #include <new>
@@ -63,6 +64,7 @@ struct symheap {
     int       max_smem = 48 * 1024;   // opt-in dynamic shared memory per CTA
     uint64_t  spin_ns = 2000000000ull;
     bool      pdl          = false;
+    int       env_algo     = 0;       // SYMAR_ALGO override of SYMAR_AUTO, 0 = none
     int       dbg_mute     = -1;
     unsigned  dbg_seed     = 0;
     unsigned  dbg_delay_ns = 0;
@@ -180,7 +182,7 @@ static int make_plan(symheap *h, size_t in_off, size_t out_off, size_t count, in
     const Tuned &tn    = h->tuned[dtype];
     const int b        = tn.valid ? std::min(std::max(bucket_of(bytes), tn.lo_bucket), tn.hi_bucket) : 0;
 
-    if (algo == SYMAR_AUTO) algo = tn.valid ? tn.best_algo[b] : default_algo(bytes);
+    if (algo == SYMAR_AUTO) algo = h->env_algo ? h->env_algo : (tn.valid ? tn.best_algo[b] : default_algo(bytes));
 
     LaunchCfg cfg = default_cfg(h, algo, nvec);
     if (tn.valid && tn.cfg[algo][b].ctas > 0) cfg = tn.cfg[algo][b];
@@ -478,6 +480,18 @@ static int create_common(symheap_t **heap, int P, size_t bytes_per_rank, void *m
         delete h;
         return cuda_fail(e, "heap initialisation");
     }
+    // Environment overrides (read once per heap): SYMAR_SPIN_LIMIT_US bounds every
+    // device-side wait; SYMAR_ALGO = oneshot | twoshot | ll replaces SYMAR_AUTO's choice;
+    // SYMAR_PDL = 1 turns programmatic dependent launch on.
+    if (const char *v = std::getenv("SYMAR_SPIN_LIMIT_US")) {
+        const long us = std::atol(v);
+        if (us > 0) h->spin_ns = (uint64_t)us * 1000ull;
+    }
+    if (const char *v = std::getenv("SYMAR_ALGO")) {
+        const std::string a(v);
+        h->env_algo = a == "oneshot" ? SYMAR_ONESHOT : a == "twoshot" ? SYMAR_TWOSHOT : a == "ll" ? SYMAR_LL : 0;
+    }
+    if (const char *v = std::getenv("SYMAR_PDL")) h->pdl = std::atoi(v) != 0;
     *heap = h;
     return SYMAR_OK;
 }

@@ -1,0 +1,120 @@
+"""The five benchmark workloads at their full sizes, in the launch configuration
+bench.py times, bit for bit against the CPU oracle."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import allreduce_oracle as O
+from paper_2607_16100_b200 import symar, synth
+
+pytestmark = pytest.mark.gpu
+
+ALGOS = [symar.ONESHOT, symar.TWOSHOT, symar.LL, symar.AUTO]
+DT = {"f32": symar.F32, "bf16": symar.BF16}
+NP = {"f32": np.float32, "bf16": np.uint16}
+
+
+def bits(a):
+    return np.ascontiguousarray(a).view(np.uint8)
+
+
+def one_call(h, x, dtype, algo, in_off, out_off):
+    P, count = x.shape
+    for q in range(P):
+        h.write_rank(q, in_off, x[q])
+    h.allreduce(in_off, out_off, count, DT[dtype], algo)
+    torch.cuda.synchronize()
+    assert h.status()[0] == symar.OK
+    return np.stack([h.read_rank(q, out_off, count, NP[dtype]) for q in range(P)])
+
+
+def test_c1_exact_integer_sums_p4_fp32():
+    w = synth.WORKLOADS["c1"]
+    x = synth.make_inputs(w["dist"], w["dtype"], w["P"], w["count"], w["seed"])
+    want = O.allreduce(x)
+    assert np.array_equal(want[0], x.astype(np.int64).sum(axis=0).astype(np.float32))   # the config's own point
+    h = symar.SymHeap.on_torch(w["P"], 1 << 20)
+    try:
+        for algo in ALGOS:
+            got = one_call(h, x, "f32", algo, 0, 1 << 19)
+            assert np.array_equal(bits(got), bits(want)), algo
+    finally:
+        h.destroy()
+
+
+def test_c2_and_c3_message_sweep_p8_bf16():
+    w = synth.WORKLOADS["c3"]
+    h = symar.SymHeap.on_torch(8, 4 << 20)
+    try:
+        for tuned in (False, True):
+            if tuned:
+                h.autotune(symar.BF16)
+            for B in w["batch"]:
+                count = w["count"] * B
+                x = synth.make_inputs(w["dist"], "bf16", 8, count, w["seed"] + B)
+                want = O.allreduce(x)
+                for algo in ALGOS:
+                    got = one_call(h, x, "bf16", algo, 0, 2 << 20)
+                    assert np.array_equal(bits(got), bits(want)), (tuned, B, algo)
+    finally:
+        torch.cuda.synchronize()
+        h.destroy()
+
+
+def test_c4_full_size_p8_fp32_256MiB():
+    w = synth.WORKLOADS["c4"]
+    P, count = w["P"], w["count"]
+    M = count * 4
+    x = synth.make_inputs(w["dist"], "f32", P, count, w["seed"])
+    want = O.allreduce_timed_team(x, threads=0)[0][0]          # all rows of the oracle's output are equal
+    h = symar.SymHeap.on_torch(P, 2 * M)
+    try:
+        for q in range(P):
+            h.write_rank(q, 0, x[q])
+        del x
+        h.allreduce(0, M, count, symar.F32, symar.TWOSHOT)      # bench.py's call, default launch shape
+        torch.cuda.synchronize()
+        assert h.status()[0] == symar.OK
+        assert h.last_kernel()[1] > 0                            # the bulk-copy kernel ran
+        want_bits = want.view(np.uint32)
+        for r in range(P):
+            got = h.read_rank(r, M, count, np.float32).view(np.uint32)
+            bad = np.flatnonzero(got != want_bits)
+            assert bad.size == 0, f"rank {r}: {bad.size} mismatches, first at {bad[0]}"
+    finally:
+        h.destroy()
+
+
+@pytest.mark.parametrize("P", [8, 4])
+def test_c5_decode_trace_160_calls_in_one_graph(P):
+    w = synth.WORKLOADS["c5"]
+    calls, count = w["calls"], w["count"]
+    nb = count * 2
+    xs = [synth.make_inputs(w["dist"], "bf16", P, count, w["seed"], call=k) for k in range(calls)]
+    wants = [O.allreduce(x)[0] for x in xs]
+    h = symar.SymHeap.on_torch(P, 24 << 20)
+    try:
+        h.autotune(symar.BF16)                                   # as bench.py does before capturing
+        for k in range(calls):
+            for q in range(P):
+                h.write_rank(q, k * nb, xs[k][q])
+        out0 = 10 << 20
+        s = torch.cuda.Stream()
+        g = torch.cuda.CUDAGraph()
+        torch.cuda.synchronize()
+        with torch.cuda.graph(g, stream=s):
+            for k in range(calls):
+                h.allreduce(k * nb, out0 + k * nb, count, symar.BF16, symar.AUTO, s.cuda_stream)
+        for rep in range(3):
+            for q in range(P):
+                h.write_rank(q, out0, np.zeros(calls * nb, dtype=np.uint8))
+            g.replay()
+            torch.cuda.synchronize()
+            assert h.status()[0] == symar.OK
+            for q in range(P):
+                got = h.read_rank(q, out0, calls * count, np.uint16).reshape(calls, count)
+                for k in range(calls):
+                    assert np.array_equal(got[k], wants[k]), (rep, q, k)
+    finally:
+        torch.cuda.synchronize()
+        h.destroy()
