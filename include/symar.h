@@ -20,8 +20,8 @@
  * that gives up records SYMAR_ERR_TIMEOUT in the heap's status word (read it
  * with symheap_status) and the kernel returns normally.
  *
- * Environment (read when a heap is created): SYMAR_ALGO = oneshot | twoshot | ll
- * replaces SYMAR_AUTO's choice; SYMAR_SPIN_LIMIT_US bounds device-side waits;
+ * Environment (read when a heap is created): SYMAR_ALGO = oneshot | twoshot | ll |
+ * sentinel replaces SYMAR_AUTO's choice; SYMAR_SPIN_LIMIT_US bounds device-side waits;
  * SYMAR_PDL = 1 enables programmatic dependent launch.
  *
  * Threading: a heap may be used from one host thread and one stream at a time
@@ -47,7 +47,11 @@ typedef enum {
                             low-latency algorithm based on the collected empirical results") */
     SYMAR_ONESHOT = 1,   /* Sec. III-A.1, pull form: every rank reads all P inputs           */
     SYMAR_TWOSHOT = 2,   /* Sec. III-A.2: reduce-scatter, then all-gather with flag handoff  */
-    SYMAR_LL      = 3    /* Sec. IV "LL" + Sec. V example: one-shot push, data+flag stores   */
+    SYMAR_LL      = 3,   /* Sec. IV "LL" + Sec. V example: one-shot push, data+flag stores   */
+    SYMAR_SENTINEL = 4   /* Sec. IV "Sentinel": one-shot push of bare data into scratch that
+                            holds a sentinel word; the receiver polls until every word has
+                            changed and restores the sentinel.  Never chosen by SYMAR_AUTO
+                            unless the tuner measured it to be fastest.                      */
 } symar_algo_t;
 
 enum {
@@ -74,6 +78,7 @@ typedef struct {
     size_t   bytes_per_rank;      /* user region as requested                                   */
     size_t   user_bytes;          /* user region as laid out (rounded up to SYMAR_ALIGN)        */
     size_t   ll_scratch_bytes;    /* per rank: 2 parities x slots x P senders x vecs x 32 B     */
+    size_t   sentinel_scratch_bytes; /* per rank: 2 parities x slots x P senders x vecs x 16 B   */
     size_t   flag_bytes;          /* per rank: ready + done flag arrays + epoch counters        */
     size_t   stride;              /* bytes from one rank segment to the next                    */
     size_t   total_bytes;         /* control block + P segments                                 */

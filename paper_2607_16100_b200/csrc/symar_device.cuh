@@ -73,6 +73,23 @@ __device__ __forceinline__ U64x2 ld_relaxed_v2u64(const void *p)
     return v;
 }
 
+// 16-byte strong accesses of four 32-bit elements (each element a single access)
+__device__ __forceinline__ void st_relaxed_v4(void *p, const uint4 &v)
+{
+    asm volatile("st.relaxed." SYMAR_SCOPE ".global.v4.u32 [%0], {%1, %2, %3, %4};" ::"l"(p), "r"(v.x), "r"(v.y),
+                 "r"(v.z), "r"(v.w)
+                 : "memory");
+}
+__device__ __forceinline__ uint4 ld_relaxed_v4(const void *p)
+{
+    uint4 v;
+    asm volatile("ld.relaxed." SYMAR_SCOPE ".global.v4.u32 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "l"(p)
+                 : "memory");
+    return v;
+}
+
 // A rank's OWN input is written before its kernel starts and never during it:
 // read-only path, no L1 allocation.
 __device__ __forceinline__ uint4 ld_own(const void *p)

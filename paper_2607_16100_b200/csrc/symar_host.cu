@@ -24,7 +24,7 @@ struct LaunchCfg {
 };
 
 constexpr int kBuckets = 40;   // bucket b holds messages of (2^(b-1), 2^b] bytes per rank
-constexpr int kAlgos   = 4;    // indexed by symar_algo_t
+constexpr int kAlgos   = 5;    // indexed by symar_algo_t
 
 struct Tuned {
     bool      valid = false;
@@ -69,8 +69,8 @@ struct symheap {
     unsigned  dbg_seed     = 0;
     unsigned  dbg_delay_ns = 0;
     LaunchCfg forced[kAlgos];
-    unsigned  variant[kAlgos] = {0, 0, 0, 0};
-    bool      variant_forced[kAlgos] = {false, false, false, false};
+    unsigned  variant[kAlgos] = {};
+    bool      variant_forced[kAlgos] = {};
     Tuned     tuned[2];
     int       last_algo = 0, last_ctas = 0, last_threads = 0;
     unsigned  last_variant = 0;
@@ -149,7 +149,8 @@ static LaunchCfg default_cfg(const symheap *h, int algo, uint64_t nvec)
     }
     c.threads = units >= 2048 ? 128 : round_threads(std::max<uint64_t>(units / 16, 32));
     uint64_t ctas = (units + c.threads - 1) / c.threads;
-    const uint64_t cap = algo == SYMAR_LL ? (uint64_t)kLLSlots : (uint64_t)std::max(1, 2 * h->num_sms / h->P);
+    const uint64_t cap = (algo == SYMAR_LL || algo == SYMAR_SENTINEL) ? (uint64_t)kLLSlots
+                                                                       : (uint64_t)std::max(1, 2 * h->num_sms / h->P);
     c.ctas = (int)std::max<uint64_t>(1, std::min(ctas, cap));
     return c;
 }
@@ -210,7 +211,7 @@ static int make_plan(symheap *h, size_t in_off, size_t out_off, size_t count, in
         p->smem     = bulk_smem_bytes(h->P, a.tile_vecs, a.stages);
     }
     if (!fn) return SYMAR_ERR_INVAL;
-    const int cap_slots = algo == SYMAR_LL ? kLLSlots : kMaxCtas;
+    const int cap_slots = (algo == SYMAR_LL || algo == SYMAR_SENTINEL) ? kLLSlots : kMaxCtas;
     const int cap_res   = std::max(1, max_resident(h, fn, cfg.threads, p->smem) / h->P);
     cfg.ctas = std::max(1, std::min({cfg.ctas, cap_slots, cap_res}));
 
@@ -221,6 +222,7 @@ static int make_plan(symheap *h, size_t in_off, size_t out_off, size_t count, in
     a.count      = count;
     a.nvec       = nvec;
     a.ll_off     = h->L.ll_off;
+    a.sn_off     = h->L.sn_off;
     a.ready_off  = h->L.ready_off;
     a.done_off   = h->L.done_off;
     a.epoch_off  = h->L.epoch_off;
@@ -237,7 +239,7 @@ static int make_plan(symheap *h, size_t in_off, size_t out_off, size_t count, in
         a.blk_log2 = cyclic ? kCyclicLog2 : kOneChunk;
         a.wide     = cyclic && ((in_off | out_off) % 32 == 0) && !(var & 2u);
     }
-    if (algo == SYMAR_LL) {
+    if (algo == SYMAR_LL || algo == SYMAR_SENTINEL) {
         // every CTA takes `cv` vectors per iteration; iterations alternate sub-buffers
         const uint64_t per_cta = (nvec + cfg.ctas - 1) / cfg.ctas;
         a.cv    = (uint32_t)std::max<uint64_t>(1, std::min<uint64_t>(per_cta, kLLSlotVecs));
@@ -273,7 +275,7 @@ static int run(symheap *h, const void *in, void *out, size_t count, int dtype, i
     size_t io = 0, oo = 0;
     int rc = check_buffers(h, in, out, count, dtype, &io, &oo);
     if (rc != SYMAR_OK) return rc;
-    if (algo < SYMAR_AUTO || algo > SYMAR_LL) return SYMAR_ERR_INVAL;
+    if (algo < SYMAR_AUTO || algo > SYMAR_SENTINEL) return SYMAR_ERR_INVAL;
     if (count == 0) return SYMAR_OK;
     Plan p;
     rc = make_plan(h, io, oo, count, dtype, algo, &p);
@@ -370,10 +372,10 @@ static int autotune(symheap *h, int dtype)
         const int reps = 7;
         double best_us = 1e30;
         tn.best_algo[b] = SYMAR_ONESHOT;
-        for (int algo = SYMAR_ONESHOT; algo <= SYMAR_LL && rc == SYMAR_OK; ++algo) {
+        for (int algo = SYMAR_ONESHOT; algo <= SYMAR_SENTINEL && rc == SYMAR_OK; ++algo) {
             tn.us[algo][b]  = 1e30;
             tn.cfg[algo][b] = LaunchCfg{};
-            if (algo == SYMAR_LL && bytes > (4u << 20)) continue;      // 2 P M scratch traffic: hopeless there
+            if ((algo == SYMAR_LL || algo == SYMAR_SENTINEL) && bytes > (4u << 20)) continue;   // P M scratch traffic per rank: hopeless there
             if (algo == SYMAR_ONESHOT && bytes > (32u << 20)) continue;
             const uint64_t work = algo == SYMAR_TWOSHOT ? (nvec + h->P - 1) / h->P : nvec;
             // kernel variants worth timing: the default; for two-shot in the bandwidth
@@ -459,11 +461,13 @@ static int create_common(symheap_t **heap, int P, size_t bytes_per_rank, void *m
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&h->num_sms, cudaDevAttrMultiProcessorCount, h->device);
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&h->max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, h->device);
     if (e == cudaSuccess) e = cudaMemset(h->mem, 0, kCtlBytes);
-    for (int q = 0; q < P && e == cudaSuccess; ++q)
+    for (int q = 0; q < P && e == cudaSuccess; ++q) {
         e = cudaMemset(h->seg0 + (size_t)q * L.stride + L.ll_off, 0, L.seg_bytes - L.ll_off);
+        if (e == cudaSuccess) e = cudaMemset(h->seg0 + (size_t)q * L.stride + L.sn_off, 0xff, L.sn_bytes);
+    }
     // Load every kernel this heap can launch now, so that a first call made
     // during stream capture does not trigger lazy module loading there.
-    for (int algo = SYMAR_ONESHOT; algo <= SYMAR_LL && e == cudaSuccess; ++algo)
+    for (int algo = SYMAR_ONESHOT; algo <= SYMAR_SENTINEL && e == cudaSuccess; ++algo)
         for (int dt = SYMAR_F32; dt <= SYMAR_BF16 && e == cudaSuccess; ++dt) {
             cudaFuncAttributes attr;
             e = cudaFuncGetAttributes(&attr, kernel_for(algo, dt, P, false));
@@ -489,7 +493,7 @@ static int create_common(symheap_t **heap, int P, size_t bytes_per_rank, void *m
     }
     if (const char *v = std::getenv("SYMAR_ALGO")) {
         const std::string a(v);
-        h->env_algo = a == "oneshot" ? SYMAR_ONESHOT : a == "twoshot" ? SYMAR_TWOSHOT : a == "ll" ? SYMAR_LL : 0;
+        h->env_algo = a == "oneshot" ? SYMAR_ONESHOT : a == "twoshot" ? SYMAR_TWOSHOT : a == "ll" ? SYMAR_LL : a == "sentinel" ? SYMAR_SENTINEL : 0;
     }
     if (const char *v = std::getenv("SYMAR_PDL")) h->pdl = std::atoi(v) != 0;
     *heap = h;
@@ -549,6 +553,7 @@ int symheap_info(const symheap_t *heap, symheap_info_t *info)
     info->bytes_per_rank   = heap->bytes_per_rank;
     info->user_bytes       = heap->L.user_bytes;
     info->ll_scratch_bytes = heap->L.ll_bytes;
+    info->sentinel_scratch_bytes = heap->L.sn_bytes;
     info->flag_bytes       = heap->L.seg_bytes - heap->L.ready_off;
     info->stride           = heap->L.stride;
     info->total_bytes      = heap->L.total;
@@ -567,9 +572,11 @@ int symheap_reset(symheap_t *heap, void *cuda_stream)
     if (!heap) return SYMAR_ERR_INVAL;
     cudaStream_t s = (cudaStream_t)cuda_stream;
     CU(cudaMemsetAsync(heap->mem, 0, kCtlBytes, s));
-    for (int q = 0; q < heap->P; ++q)
+    for (int q = 0; q < heap->P; ++q) {
         CU(cudaMemsetAsync(heap->seg0 + (size_t)q * heap->L.stride + heap->L.ll_off, 0,
                            heap->L.seg_bytes - heap->L.ll_off, s));
+        CU(cudaMemsetAsync(heap->seg0 + (size_t)q * heap->L.stride + heap->L.sn_off, 0xff, heap->L.sn_bytes, s));
+    }
     return SYMAR_OK;
 }
 
@@ -654,7 +661,7 @@ int symar_tuned_entry(const symheap_t *heap, symar_dtype_t dtype, int log2_bytes
     if (!heap || (dtype != SYMAR_F32 && dtype != SYMAR_BF16)) return SYMAR_ERR_INVAL;
     const Tuned &tn = heap->tuned[(int)dtype];
     if (!tn.valid || log2_bytes < tn.lo_bucket || log2_bytes > tn.hi_bucket) return SYMAR_ERR_INVAL;
-    if (algo < SYMAR_ONESHOT || algo > SYMAR_LL) return SYMAR_ERR_INVAL;
+    if (algo < SYMAR_ONESHOT || algo > SYMAR_SENTINEL) return SYMAR_ERR_INVAL;
     if (ctas_per_rank) *ctas_per_rank = tn.cfg[algo][log2_bytes].ctas;
     if (threads) *threads = tn.cfg[algo][log2_bytes].threads;
     if (host_us) *host_us = tn.us[algo][log2_bytes];
@@ -663,7 +670,7 @@ int symar_tuned_entry(const symheap_t *heap, symar_dtype_t dtype, int log2_bytes
 
 int symar_set_launch(symheap_t *heap, symar_algo_t algo, int ctas_per_rank, int threads)
 {
-    if (!heap || algo < SYMAR_ONESHOT || algo > SYMAR_LL) return SYMAR_ERR_INVAL;
+    if (!heap || algo < SYMAR_ONESHOT || algo > SYMAR_SENTINEL) return SYMAR_ERR_INVAL;
     if (ctas_per_rank < 0 || threads < 0 || threads > (int)kMaxThreads) return SYMAR_ERR_INVAL;
     heap->forced[algo] = LaunchCfg{ctas_per_rank, threads};
     return SYMAR_OK;
@@ -671,7 +678,7 @@ int symar_set_launch(symheap_t *heap, symar_algo_t algo, int ctas_per_rank, int 
 
 int symar_set_variant(symheap_t *heap, symar_algo_t algo, unsigned int variant)
 {
-    if (!heap || algo < SYMAR_ONESHOT || algo > SYMAR_LL) return SYMAR_ERR_INVAL;
+    if (!heap || algo < SYMAR_ONESHOT || algo > SYMAR_SENTINEL) return SYMAR_ERR_INVAL;
     heap->variant[algo]        = variant & 0x7fffffffu;
     heap->variant_forced[algo] = variant != 0;       // bit 31 alone forces the plain variant 0
     return SYMAR_OK;

@@ -334,6 +334,98 @@ __global__ void __launch_bounds__(kMaxThreads) ll_kernel(const KArgs a)
     if (t == 0) *ep = n0 + a.iters;
 }
 
+// One-shot push with sentinel synchronisation (Sec. IV "Sentinel"; Sec. V send / recv with
+// Reset / reset).  The receiving scratch holds the sentinel word everywhere; a sender
+// stores bare payload vectors (full payload bandwidth, half of LL's scratch); the
+// receiver polls a slot until none of its four words is the sentinel, takes the data
+// and stores the sentinel back.  A payload word that happens to equal the sentinel
+// (a NaN with all bits set) is sent with its lowest bit cleared: still a NaN, and
+// a sum with a NaN is a NaN either way, so no input value is forbidden.
+// Double buffering by iteration parity as in the LL kernel; with more than one
+// iteration per call a fence per iteration makes the restored sentinels visible
+// before a peer can target the same sub-buffer again (between calls the kernel
+// boundary does that).
+template <typename E, int P, bool DBG>
+__global__ void __launch_bounds__(kMaxThreads) sentinel_kernel(const KArgs a)
+{
+    const int c = blockIdx.x, r = blockIdx.y, C = gridDim.x;
+    const uint32_t t = threadIdx.x, T = blockDim.x;
+    char *seg_r  = a.seg0 + (size_t)r * a.stride;
+    uint64_t *ep = reinterpret_cast<uint64_t *>(seg_r + a.epoch_off) + c;
+    if (a.pdl) {
+        pdl_wait();
+        pdl_launch_dependents();
+    }
+    const uint64_t n0 = ld_relaxed_u64(ep);
+    if (DBG) debug_delay(a, r, c);
+    if (DBG && a.dbg_mute == r) return;       // test hook: this rank never joins
+
+    const char *in = seg_r + a.in_off;
+    char *out      = seg_r + a.out_off;
+    bool failed    = false;
+    uint4 kept     = make_uint4(0u, 0u, 0u, 0u);
+    const uint4 sentinel = make_uint4(kSentinelWord, kSentinelWord, kSentinelWord, kSentinelWord);
+    auto clean = [](uint32_t w) { return w == kSentinelWord ? (kSentinelWord & ~1u) : w; };
+
+    for (uint32_t it = 0; it < a.iters && !failed; ++it) {
+        const uint64_t n   = n0 + 1 + it;
+        const uint64_t v0  = ((uint64_t)it * C + c) * a.cv;
+        const uint32_t cnt = v0 < a.nvec ? (uint32_t)(a.nvec - v0 < a.cv ? a.nvec - v0 : a.cv) : 0u;
+        const uint64_t region = a.sn_off + ((uint64_t)(n & 1) * kLLSlots + c) * P * kSnSenderBytes;
+
+        for (uint32_t k = t; k < cnt; k += T) {          // bcast
+            uint4 x = ld_own(in + (v0 + k) * 16);
+            x = make_uint4(clean(x.x), clean(x.y), clean(x.z), clean(x.w));
+            if (k == t) kept = x;
+            char *dst = a.seg0 + region + (size_t)r * kSnSenderBytes + (size_t)k * 16;
+#pragma unroll
+            for (int q = 0; q < P; ++q) {
+                if (q != r) st_relaxed_v4(dst, x);
+                dst += a.stride;
+            }
+        }
+        for (uint32_t k = t; k < cnt && !failed; k += T) {   // recvReduce with reset
+            char *src = seg_r + region + (size_t)k * 16;
+            uint4 x[P];
+            unsigned need = ((1u << P) - 1u) & ~(1u << r);
+            Spin spin;
+            while (need != 0) {
+                uint4 d[P];
+#pragma unroll
+                for (int q = 0; q < P; ++q)
+                    if (need >> q & 1u) d[q] = ld_relaxed_v4(src + (size_t)q * kSnSenderBytes);
+#pragma unroll
+                for (int q = 0; q < P; ++q) {
+                    if ((need >> q & 1u) && d[q].x != kSentinelWord && d[q].y != kSentinelWord &&
+                        d[q].z != kSentinelWord && d[q].w != kSentinelWord) {
+                        x[q] = d[q];
+                        st_relaxed_v4(src + (size_t)q * kSnSenderBytes, sentinel);      // reset for reuse
+                        need &= ~(1u << q);
+                    }
+                }
+                if (need != 0 && spin.due() && spin.expired(a.spin_ns)) {
+                    report_timeout(a.ctl, r, __ffs(need) - 1, c);
+                    failed = true;
+                    break;
+                }
+            }
+            if (failed) break;
+            uint4 own = kept;
+            if (k != t) {
+                own = ld_own(in + (v0 + k) * 16);
+                own = make_uint4(clean(own.x), clean(own.y), clean(own.z), clean(own.w));
+            }
+#pragma unroll
+            for (int q = 0; q < P; ++q)
+                if (q == r) x[q] = own;
+            store_result(out, v0 + k, reduce_in_rank_order<E, P>(x), a.nvec, a.tail_bytes);
+        }
+        if (a.iters > 1) fence_acq_rel();
+    }
+    __syncthreads();
+    if (t == 0) *ep = n0 + a.iters;
+}
+
 // ---- dispatch ---------------------------------------------------------------------
 
 template <typename E, int P, bool DBG>
@@ -343,6 +435,7 @@ static KernelFn pick_algo(int algo)
         case SYMAR_ONESHOT: return oneshot_kernel<E, P, DBG>;
         case SYMAR_TWOSHOT: return twoshot_kernel<E, P, DBG>;
         case SYMAR_LL:      return ll_kernel<E, P, DBG>;
+        case SYMAR_SENTINEL: return sentinel_kernel<E, P, DBG>;
     }
     return nullptr;
 }

@@ -2,7 +2,7 @@
 // of libsymar (never by the CPU oracle).
 //
 // heap memory:  [ control block | segment 0 | segment 1 | ... | segment P-1 ]
-// segment q  :  [ user region | LL scratch | ready flags | done flags | epochs | pad ]
+// segment q  :  [ user region | LL scratch | sentinel scratch | ready flags | done flags | counters | pad ]
 //
 // Every rank segment has the same layout (symmetric objects: same offset + rank
 // id addresses a peer's copy), every region starts on a 4 KiB boundary.
@@ -65,6 +65,8 @@ struct Layout {
     size_t   user_bytes;     // rounded up
     size_t   ll_off;         // segment offset of the LL scratch
     size_t   ll_bytes;
+    size_t   sn_off;         // sentinel scratch: [parity][slot][sender][vector] x 16 B, pre-filled with 0xFF
+    size_t   sn_bytes;
     size_t   ready_off;      // kMaxCtas groups of kFlagGroup bytes
     size_t   done_off;
     size_t   epoch_off;      // kMaxCtas x u64 LL iteration counters, then kMaxCtas x u32
@@ -77,6 +79,10 @@ struct Layout {
 // bytes one sender occupies in one (parity, slot) region: vecs x 2 halves x 16 B
 constexpr size_t kLLSenderBytes = (size_t)kLLSlotVecs * 32;
 
+// sentinel mode: bare 16-byte vectors, no flag words
+constexpr size_t   kSnSenderBytes = (size_t)kLLSlotVecs * 16;
+constexpr uint32_t kSentinelWord  = 0xffffffffu;      // a negative NaN in fp32, two of them in bf16
+
 inline Layout make_layout(int P, size_t bytes_per_rank)
 {
     Layout L{};
@@ -84,7 +90,9 @@ inline Layout make_layout(int P, size_t bytes_per_rank)
     L.user_bytes = round_up(bytes_per_rank ? bytes_per_rank : 1, kAlign);
     L.ll_off     = L.user_bytes;
     L.ll_bytes   = (size_t)2 * kLLSlots * P * kLLSenderBytes;
-    L.ready_off  = L.ll_off + L.ll_bytes;
+    L.sn_off     = L.ll_off + L.ll_bytes;
+    L.sn_bytes   = (size_t)2 * kLLSlots * P * kSnSenderBytes;
+    L.ready_off  = L.sn_off + L.sn_bytes;
     L.done_off   = L.ready_off + (size_t)kMaxCtas * kFlagGroup;
     L.epoch_off  = L.done_off + (size_t)kMaxCtas * kFlagGroup;
     L.seg_bytes  = round_up(L.epoch_off + (size_t)kMaxCtas * (sizeof(uint64_t) + 2 * sizeof(uint32_t)), kAlign);
@@ -104,6 +112,7 @@ struct KArgs {
     uint64_t  count;         // elements per rank
     uint64_t  nvec;          // 16-byte vectors per rank, ceil(count * elem / 16)
     uint64_t  ll_off;
+    uint64_t  sn_off;
     uint64_t  ready_off;
     uint64_t  done_off;
     uint64_t  epoch_off;

@@ -49,6 +49,7 @@ def test_binding_constants_match_header():
         m = re.search(rf"{name}\s*=\s*(\d+)", HEADER)
         assert m and int(m.group(1)) == val
     for name, val in (("SYMAR_AUTO", 0), ("SYMAR_ONESHOT", 1), ("SYMAR_TWOSHOT", 2), ("SYMAR_LL", 3),
+                      ("SYMAR_SENTINEL", 4),
                       ("SYMAR_ERR_TIMEOUT", -4)):
         m = re.search(rf"{name}\s*=\s*(-?\d+)", HEADER)
         assert m and int(m.group(1)) == val
@@ -64,9 +65,11 @@ def test_required_bytes_layout(lib, P):
     # for double buffering.
     D = symar.LL_SLOTS * symar.LL_SLOT_VECS * 16
     ll = 2 * (2 * P * D)
+    # Table I, one-shot sentinel: N D per iteration (bare payload), again two parities
+    sentinel = 2 * (P * D)
     flags = 2 * symar.MAX_CTAS * 32 + symar.MAX_CTAS * 8
-    assert total >= P * (user + ll + flags)
-    assert total <= P * (user + ll + flags + 16 * symar.ALIGN) + 4096
+    assert total >= P * (user + ll + sentinel + flags)
+    assert total <= P * (user + ll + sentinel + flags + 16 * symar.ALIGN) + 4096
     assert total % symar.ALIGN == 0
     # monotone in the user size, and rounding never loses bytes
     assert symar.required_bytes(P, user + 1) >= total

@@ -9,7 +9,7 @@ from paper_2607_16100_b200 import symar, synth
 
 pytestmark = pytest.mark.gpu
 
-ALGOS = [symar.ONESHOT, symar.TWOSHOT, symar.LL]
+ALGOS = [symar.ONESHOT, symar.TWOSHOT, symar.LL, symar.SENTINEL]
 NP_DT = {symar.F32: np.float32, symar.BF16: np.uint16}
 DT = {"f32": symar.F32, "bf16": symar.BF16}
 USER = 8 << 20          # user region per rank of the shared test heaps
@@ -134,16 +134,45 @@ def test_forced_launch_shapes(heaps, algo, ctas, threads):
     assert_bits(got, O.allreduce(x))
 
 
-def test_ll_many_iterations_alternate_subbuffers(heaps):
+@pytest.mark.parametrize("algo", [symar.LL, symar.SENTINEL])
+def test_push_many_iterations_alternate_subbuffers(heaps, algo):
     # one CTA per rank, 1024 vectors per iteration: 300000 fp32 -> 75000 vectors -> 74 iterations
     h = heaps[4]
     x = synth.make_inputs("uniform", "f32", 4, 300000, seed=5)
-    h.set_launch(symar.LL, 1, 256)
+    h.set_launch(algo, 1, 256)
     try:
-        got = run(h, x, symar.F32, symar.LL)
+        got = run(h, x, symar.F32, algo)
+        got2 = run(h, x[::-1].copy(), symar.F32, algo)      # straight again on the same scratch
     finally:
-        h.set_launch(symar.LL, 0, 0)
+        h.set_launch(algo, 0, 0)
     assert_bits(got, O.allreduce(x))
+    assert_bits(got2, O.allreduce(x[::-1].copy()))
+
+
+def test_sentinel_mode_accepts_payload_equal_to_the_sentinel(heaps):
+    # words of all ones (a negative NaN; in bf16 two of them) are the scratch's
+    # sentinel; such payload is sent with one bit changed -- still NaN -- so the
+    # receiver is never left waiting and NaN-ness of the result is kept
+    h = heaps[8]
+    rng = np.random.default_rng(8)
+    x = synth.make_inputs("uniform", "f32", 8, 4096, seed=3)
+    xw = x.view(np.uint32)
+    xw[rng.integers(0, 8, 300), rng.integers(0, 4096, 300)] = 0xFFFFFFFF
+    want = O.allreduce(x)
+    got = run(h, x, symar.F32, symar.SENTINEL)
+    assert np.array_equal(np.isnan(got), np.isnan(want)) and np.isnan(want).sum() >= 250
+    keep = ~np.isnan(want)
+    assert_bits(np.where(keep, got, np.float32(0)), np.where(keep, want, np.float32(0)))
+    xb = synth.make_inputs("normal", "bf16", 8, 4096, seed=4)
+    xb.view(np.uint32)[rng.integers(0, 8, 200), rng.integers(0, 2048, 200)] = 0xFFFFFFFF
+    wantb = O.allreduce(xb)
+    gotb = run(h, xb, symar.BF16, symar.SENTINEL)
+    is_nan = lambda v: ((v & 0x7F80) == 0x7F80) & ((v & 0x007F) != 0)
+    assert np.array_equal(is_nan(gotb), is_nan(wantb))
+    assert_bits(np.where(is_nan(wantb), 0, gotb), np.where(is_nan(wantb), 0, wantb))
+    # and the scratch is whole again afterwards
+    y = synth.make_inputs("normal", "bf16", 8, 4096, seed=5)
+    assert_bits(run(h, y, symar.BF16, symar.SENTINEL), O.allreduce(y))
 
 
 FORCE_PLAIN = 1 << 31
@@ -153,7 +182,8 @@ FORCE_PLAIN = 1 << 31
 @pytest.mark.parametrize("P,dtype,dist", [(8, "bf16", "normal"), (4, "f32", "uniform"), (2, "bf16", "normal"),
                                           (1, "f32", "uniform")])
 @pytest.mark.parametrize("algo,variant", [(symar.ONESHOT, FORCE_PLAIN), (symar.ONESHOT, 0x100),
-                                          (symar.ONESHOT, 0x200), (symar.LL, FORCE_PLAIN), (symar.LL, 0x100)])
+                                          (symar.ONESHOT, 0x200), (symar.LL, FORCE_PLAIN), (symar.LL, 0x100),
+                                          (symar.SENTINEL, FORCE_PLAIN)])
 def test_unit_width_variants(heaps, algo, variant, P, dtype, dist, count):
     # 16, 8 or 4 bytes per thread: same bits, whatever the ragged tail
     h = heaps[P]
@@ -277,7 +307,7 @@ def test_mixed_algorithms_and_shapes_share_flags_safely(heaps):
     h = heaps[8]
     rng = np.random.default_rng(12)
     for i in range(60):
-        algo = ALGOS[int(rng.integers(0, 3))]
+        algo = ALGOS[int(rng.integers(0, len(ALGOS)))]
         count = int(rng.integers(1, 30000))
         dtype = ("f32", "bf16")[int(rng.integers(0, 2))]
         h.set_launch(algo, int(rng.integers(1, 40)), int(rng.choice([32, 64, 128, 256, 512])))
@@ -306,7 +336,7 @@ def test_graph_capture_replays(heaps):
     torch.cuda.synchronize()
     with torch.cuda.graph(g, stream=s):
         for k in range(calls):
-            algo = ALGOS[k % 3]
+            algo = ALGOS[k % len(ALGOS)]
             h.allreduce(k * nbytes, out0 + k * nbytes, count, symar.BF16, algo, s.cuda_stream)
     for rep in range(4):
         for q in range(8):
@@ -333,7 +363,7 @@ def test_programmatic_dependent_launch_keeps_results_and_order(heaps):
     h.set_pdl(True)
     try:
         s = torch.cuda.Stream()
-        chain = [ALGOS[k % 3] for k in range(9)]
+        chain = [ALGOS[k % len(ALGOS)] for k in range(9)]
         g = torch.cuda.CUDAGraph()
         with torch.cuda.graph(g, stream=s):
             for k, algo in enumerate(chain):
