@@ -160,6 +160,61 @@ int oracle_allreduce_bf16_mt(const uint16_t *in, uint16_t *out, int P, size_t co
     return 0;
 }
 
+/*
+ * Sibling collectives built from the same primitives (paper Sec. V, "NCCL Collective
+ * Integration": low-latency Broadcast, Reduce, ReduceScatter and AllGather; Sec. III:
+ * AllReduce decomposes into ReduceScatter + AllGather or Reduce + Broadcast).
+ * es = element size in bytes (4: fp32, 2: bf16).  Reductions use the same
+ * rank-ordered binary32 sum and single narrowing as the AllReduce above.
+ *
+ * reduce_scatter: in[P][P*n] -> out[P][n],   out[r][i] = sum_q in[q][r*n + i]
+ * all_gather    : in[P][n]   -> out[P][P*n], out[r][q*n + i] = in[q][i]
+ * broadcast     : in[P][n]   -> out[P][n],   out[r][i] = in[root][i]
+ * reduce        : in[P][n]   -> out[n] (the root's result), sum over ranks
+ */
+int oracle_reduce_scatter(const void *in, void *out, int P, size_t n, int es)
+{
+    if (!in || !out || P < 1 || (es != 4 && es != 2)) return -1;
+    const size_t row = (size_t)P * n;
+    for (int r = 0; r < P; ++r)
+        for (size_t i = 0; i < n; ++i) {
+            if (es == 4)
+                ((float *)out)[(size_t)r * n + i] = reduce_f32((const float *)in, P, row, (size_t)r * n + i);
+            else
+                ((uint16_t *)out)[(size_t)r * n + i] = reduce_bf16((const uint16_t *)in, P, row, (size_t)r * n + i);
+        }
+    return 0;
+}
+
+int oracle_all_gather(const void *in, void *out, int P, size_t n, int es)
+{
+    if (!in || !out || P < 1 || (es != 4 && es != 2)) return -1;
+    const unsigned char *src = (const unsigned char *)in;
+    unsigned char *dst = (unsigned char *)out;
+    for (int r = 0; r < P; ++r)
+        for (int q = 0; q < P; ++q)
+            memcpy(dst + ((size_t)r * P + q) * n * es, src + (size_t)q * n * es, n * es);
+    return 0;
+}
+
+int oracle_broadcast(const void *in, void *out, int P, size_t n, int es, int root)
+{
+    if (!in || !out || P < 1 || root < 0 || root >= P || (es != 4 && es != 2)) return -1;
+    for (int r = 0; r < P; ++r)
+        memcpy((unsigned char *)out + (size_t)r * n * es, (const unsigned char *)in + (size_t)root * n * es, n * es);
+    return 0;
+}
+
+int oracle_reduce(const void *in, void *out, int P, size_t n, int es)
+{
+    if (!in || !out || P < 1 || (es != 4 && es != 2)) return -1;
+    for (size_t i = 0; i < n; ++i) {
+        if (es == 4) ((float *)out)[i] = reduce_f32((const float *)in, P, n, i);
+        else ((uint16_t *)out)[i] = reduce_bf16((const uint16_t *)in, P, n, i);
+    }
+    return 0;
+}
+
 /* Team size of the *_mt entry points (0 or less: leave the runtime's default). */
 void oracle_set_threads(int n)
 {

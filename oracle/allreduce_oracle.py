@@ -60,6 +60,12 @@ def _load():
             fn = getattr(lib, name)
             fn.argtypes = [vp, vp, ci, sz, ctypes.POINTER(ci)]
             fn.restype = ci
+        for name in ("oracle_reduce_scatter", "oracle_all_gather", "oracle_reduce"):
+            fn = getattr(lib, name)
+            fn.argtypes = [vp, vp, ci, sz, ci]
+            fn.restype = ci
+        lib.oracle_broadcast.argtypes = [vp, vp, ci, sz, ci, ci]
+        lib.oracle_broadcast.restype = ci
         lib.oracle_set_threads.argtypes = [ci]
         lib.oracle_set_threads.restype = None
         lib.oracle_narrow_bf16.argtypes = [ctypes.c_float]
@@ -110,6 +116,57 @@ def allreduce_timed_team(x: np.ndarray, threads: int = 1):
     if rc != 0:
         raise RuntimeError(f"oracle returned {rc}")
     return out, team
+
+
+# ---------------------------------------------------------------------------
+# sibling collectives (Sec. V: Broadcast, Reduce, ReduceScatter, AllGather)
+# ---------------------------------------------------------------------------
+
+def reduce_scatter(x: np.ndarray) -> np.ndarray:
+    """x[P, P*n] -> out[P, n]; out[r] = rank-ordered sum over q of x[q, r*n:(r+1)*n]."""
+    _check(x)
+    x = np.ascontiguousarray(x)
+    P, total = x.shape
+    if total % P:
+        raise ValueError("row length must be a multiple of P")
+    n = total // P
+    out = np.empty((P, n), dtype=x.dtype)
+    if _load().oracle_reduce_scatter(x.ctypes.data, out.ctypes.data, P, n, x.dtype.itemsize) != 0:
+        raise RuntimeError("oracle_reduce_scatter failed")
+    return out
+
+
+def all_gather(x: np.ndarray) -> np.ndarray:
+    """x[P, n] -> out[P, P*n]; every rank holds the concatenation of all inputs."""
+    _check(x)
+    x = np.ascontiguousarray(x)
+    P, n = x.shape
+    out = np.empty((P, P * n), dtype=x.dtype)
+    if _load().oracle_all_gather(x.ctypes.data, out.ctypes.data, P, n, x.dtype.itemsize) != 0:
+        raise RuntimeError("oracle_all_gather failed")
+    return out
+
+
+def broadcast(x: np.ndarray, root: int) -> np.ndarray:
+    """x[P, n] -> out[P, n]; every rank holds the root's input."""
+    _check(x)
+    x = np.ascontiguousarray(x)
+    P, n = x.shape
+    out = np.empty_like(x)
+    if _load().oracle_broadcast(x.ctypes.data, out.ctypes.data, P, n, x.dtype.itemsize, root) != 0:
+        raise RuntimeError("oracle_broadcast failed")
+    return out
+
+
+def reduce(x: np.ndarray) -> np.ndarray:
+    """x[P, n] -> out[n]: the rank-ordered sum (what the root receives)."""
+    _check(x)
+    x = np.ascontiguousarray(x)
+    P, n = x.shape
+    out = np.empty(n, dtype=x.dtype)
+    if _load().oracle_reduce(x.ctypes.data, out.ctypes.data, P, n, x.dtype.itemsize) != 0:
+        raise RuntimeError("oracle_reduce failed")
+    return out
 
 
 def _set_omp_threads(n: int) -> None:

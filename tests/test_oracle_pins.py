@@ -248,3 +248,45 @@ def test_brute_force_small_grid_f32():
             for q in range(1, P):
                 acc = Fraction(float(_rn_f32(acc + Fraction(float(x[q, i])))))
             assert float(out[0, i]) == float(acc), (P, i)
+
+
+# ---- sibling collectives: pinned to the AllReduce oracle and to plain indexing ---------
+
+@pytest.mark.parametrize("dtype,dist", [("f32", "uniform"), ("bf16", "normal")])
+@pytest.mark.parametrize("P", [1, 2, 4, 8])
+def test_allreduce_is_reduce_scatter_then_all_gather(dtype, dist, P):
+    # Sec. III: AllReduce decomposes into ReduceScatter and AllGather
+    x = synth.make_inputs(dist, dtype, P, P * 37, seed=17)
+    assert bits_eq(O.all_gather(O.reduce_scatter(x)), O.allreduce(x))
+
+
+@pytest.mark.parametrize("dtype,dist", [("f32", "uniform"), ("bf16", "normal")])
+@pytest.mark.parametrize("P", [1, 2, 4, 8])
+def test_allreduce_is_reduce_then_broadcast(dtype, dist, P):
+    x = synth.make_inputs(dist, dtype, P, 101, seed=18)
+    red = O.reduce(x)
+    assert bits_eq(red, O.allreduce(x)[0])
+    for root in range(P):
+        y = x.copy()
+        y[root] = red
+        assert bits_eq(O.broadcast(y, root), O.allreduce(x))
+
+
+def test_data_movement_collectives_against_numpy_indexing():
+    x = synth.make_inputs("normal", "bf16", 4, 50, seed=19)
+    ag = O.all_gather(x)
+    assert ag.shape == (4, 200)
+    for r in range(4):
+        assert np.array_equal(ag[r], np.concatenate([x[q] for q in range(4)]))
+    for root in range(4):
+        assert np.array_equal(O.broadcast(x, root), np.tile(x[root], (4, 1)))
+
+
+def test_reduce_scatter_hand_case():
+    # P = 2, two elements per rank: rank 0 owns columns 0-1, rank 1 columns 2-3
+    x = np.array([[1.0, 2.0, 3.0, 4.0], [10.0, 20.0, 30.0, 40.0]], dtype=np.float32)
+    out = O.reduce_scatter(x)
+    assert np.array_equal(out, np.array([[11.0, 22.0], [33.0, 44.0]], dtype=np.float32))
+    # the order pin carries over: chunk sums are rank-ordered binary32 sums
+    y = np.array([[1.0] * 4, [1e8] * 4, [-1e8] * 4, [0.0] * 4], dtype=np.float32)
+    assert np.all(O.reduce_scatter(y) == 0.0) and np.all(O.reduce(y) == 0.0)
