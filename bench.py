@@ -314,6 +314,33 @@ def latency_suite(torch, symar, synth, hbm_gbs, quick=False, autotune=True):
             out["latency_16KB"]["cold_l2_single_call_us_p50"] = float(np.percentile(
                 [a_.elapsed_time(b_) * 1000.0 for a_, b_ in cold], 50))
             del scrub
+        # the sibling collectives at the decode-step message (16 KiB per rank of input or output)
+        if P == 8:
+            x = synth.make_inputs("normal", "bf16", P, 8192, synth.seed_for_config(2))
+            for q in range(P):
+                h.write_rank(q, 0, x[q])
+            sib = {}
+            ops = {
+                "reduce_scatter": (lambda s: h.reduce_scatter(0, out_off, 8192 // P, symar.BF16, s),
+                                   lambda: O.reduce_scatter(x), 8192 // P),
+                "all_gather": (lambda s: h.all_gather(0, out_off, 8192 // P, symar.BF16, s),
+                               lambda: O.all_gather(np.ascontiguousarray(x[:, :8192 // P])), 8192),
+                "broadcast": (lambda s: h.broadcast(0, out_off, 8192, symar.BF16, 3, s),
+                              lambda: O.broadcast(x, 3), 8192),
+                "reduce": (lambda s: h.reduce(0, out_off, 8192, symar.BF16, 3, s), lambda: O.reduce(x), 8192),
+            }
+            for name, (call, ref, n_out) in ops.items():
+                assert call(stream.cuda_stream) == 0
+                stream.synchronize()
+                if name == "reduce":
+                    exact = bool(np.array_equal(h.read_rank(3, out_off, n_out, np.uint16), ref()))
+                else:
+                    got = np.stack([h.read_rank(q, out_off, n_out, np.uint16) for q in range(P)])
+                    exact = bool(np.array_equal(got, ref()))
+                g = graph_of(torch, stream, lambda k, s, call=call: call(s), K)
+                r = time_graph(torch, g, stream, K, reps)
+                sib[name] = {"p50_us": r["p50"], "bit_exact": exact and h.status()[0] == 0}
+            out["sibling_collectives_16KB"] = sib
         # C3: sweep
         if P == 8:
             sweep = []

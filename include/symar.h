@@ -156,6 +156,30 @@ int allreduce_host(symheap_t *heap, const void *host_in, void *host_out,
                    const void *in, void *out, size_t count,
                    symar_dtype_t dtype, symar_algo_t algo, void *cuda_stream);
 
+/* ---- sibling collectives (Sec. V "NCCL Collective Integration": Broadcast, Reduce,
+ *      ReduceScatter and AllGather from the same primitives; Sec. III: AllReduce =
+ *      ReduceScatter + AllGather = Reduce + Broadcast) ----------------------------
+ *
+ * Same conventions as allreduce(): symmetric addresses, 16-byte aligned, out-of-place,
+ * one kernel per call on `cuda_stream`, one signal exchange, bounded waits.  Sums are
+ * the rank-ordered binary32 sum with one narrowing.  Every rank writes only its own
+ * output.
+ *   symar_reduce_scatter  in: P * recv_count elements per rank; rank r's out (recv_count
+ *                         elements) = sum over q of in[q][r * recv_count ...]
+ *   symar_all_gather      in: send_count elements per rank; every rank's out holds the
+ *                         P inputs back to back (P * send_count elements)
+ *   symar_broadcast       every rank's out = rank `root`'s in (count elements)
+ *   symar_reduce          rank `root`'s out = the sum of all ranks' in; other ranks' out
+ *                         is left untouched                                              */
+int symar_reduce_scatter(symheap_t *heap, const void *in, void *out, size_t recv_count,
+                         symar_dtype_t dtype, void *cuda_stream);
+int symar_all_gather(symheap_t *heap, const void *in, void *out, size_t send_count,
+                     symar_dtype_t dtype, void *cuda_stream);
+int symar_broadcast(symheap_t *heap, const void *in, void *out, size_t count,
+                    symar_dtype_t dtype, int root, void *cuda_stream);
+int symar_reduce(symheap_t *heap, const void *in, void *out, size_t count,
+                 symar_dtype_t dtype, int root, void *cuda_stream);
+
 /* ---- selector (Sec. VIII kernel selection; Sec. IX: selection is empirical) --
  *
  * Times every algorithm and launch shape over a power-of-two grid of message

@@ -290,6 +290,63 @@ static int run(symheap *h, const void *in, void *out, size_t count, int dtype, i
     return SYMAR_OK;
 }
 
+// ---- sibling collectives --------------------------------------------------------------
+// op: 0 ReduceScatter (in: P*n per rank, out: n), 1 AllGather (in: n, out: P*n),
+//     2 Broadcast, 3 Reduce (in: n, out: n).  n = `count` elements.
+static int run_collective(symheap *h, int op, const void *in, void *out, size_t count, int dtype, int root,
+                          cudaStream_t s)
+{
+    if (!h || !in || !out) return SYMAR_ERR_INVAL;
+    if (dtype != SYMAR_F32 && dtype != SYMAR_BF16) return SYMAR_ERR_INVAL;
+    if ((op == 2 || op == 3) && (root < 0 || root >= h->P)) return SYMAR_ERR_INVAL;
+    const size_t es = elem_size(dtype);
+    if (count != 0 && (count * es) / count != es) return SYMAR_ERR_INVAL;
+    const size_t bytes = count * es;
+    if (bytes > h->bytes_per_rank) return SYMAR_ERR_INVAL;
+    const size_t in_total  = op == 0 ? bytes * h->P : bytes;
+    const size_t out_total = op == 1 ? bytes * h->P : bytes;
+    const char *pi = (const char *)in, *po = (const char *)out;
+    if (pi < h->seg0 || po < h->seg0) return SYMAR_ERR_INVAL;
+    const size_t io = pi - h->seg0, oo = po - h->seg0;
+    if ((io | oo) & 15) return SYMAR_ERR_INVAL;
+    if (io > h->bytes_per_rank || in_total > h->bytes_per_rank - io) return SYMAR_ERR_INVAL;
+    if (oo > h->bytes_per_rank || out_total > h->bytes_per_rank - oo) return SYMAR_ERR_INVAL;
+    if (bytes != 0 && io < oo + out_total && oo < io + in_total) return SYMAR_ERR_INVAL;     // out-of-place only
+    if (count == 0) return SYMAR_OK;
+
+    // widest unit that every per-rank offset is aligned to
+    const bool strided = op == 0 || op == 1;              // chunk q starts at q * bytes
+    const int unit = (!strided || bytes % 16 == 0) ? 16 : (bytes % 4 == 0 ? 4 : 2);
+    const uint64_t units = (bytes + unit - 1) / unit;
+    int threads = units >= 2048 ? 128 : round_threads(std::max<uint64_t>(units / 16, 32));
+    const int cap = std::max(1, std::min({(int)kMaxCtas, collective_resident(op, dtype, h->P, threads, h->num_sms) / h->P,
+                                          std::max(1, 2 * h->num_sms / h->P)}));
+    const int ctas = (int)std::max<uint64_t>(1, std::min<uint64_t>((units + threads - 1) / threads, (uint64_t)cap));
+
+    KArgs a;
+    std::memset(&a, 0, sizeof a);
+    a.seg0      = h->seg0;
+    a.stride    = h->L.stride;
+    a.in_off    = io;
+    a.out_off   = oo;
+    a.count     = count;
+    a.ready_off = h->L.ready_off;
+    a.done_off  = h->L.done_off;
+    a.epoch_off = h->L.epoch_off;
+    a.ctl       = h->ctl;
+    a.spin_ns   = h->spin_ns;
+    a.pdl       = h->pdl ? 1u : 0u;
+    a.dbg_mute  = -1;
+    cudaError_t e = launch_collective(op, dtype, h->P, ctas, threads, a, bytes, root, unit, s);
+    if (e != cudaSuccess) return cuda_fail(e, "collective launch");
+    h->last_algo    = SYMAR_ONESHOT;
+    h->last_ctas    = ctas;
+    h->last_threads = threads;
+    h->last_variant = (unsigned)unit;
+    h->last_smem    = 0;
+    return SYMAR_OK;
+}
+
 // ---- autotuner ---------------------------------------------------------------------
 
 // Median per-call time (us) of K back-to-back calls captured in one graph.
@@ -617,6 +674,30 @@ int allreduce_host(symheap_t *heap, const void *host_in, void *host_out, const v
         CU(cudaMemcpyAsync((char *)host_out + (size_t)r * bytes, heap->seg0 + (size_t)r * heap->L.stride + oo,
                            bytes, cudaMemcpyDeviceToHost, s));
     return SYMAR_OK;
+}
+
+int symar_reduce_scatter(symheap_t *heap, const void *in, void *out, size_t recv_count, symar_dtype_t dtype,
+                         void *cuda_stream)
+{
+    return run_collective(heap, 0, in, out, recv_count, (int)dtype, 0, (cudaStream_t)cuda_stream);
+}
+
+int symar_all_gather(symheap_t *heap, const void *in, void *out, size_t send_count, symar_dtype_t dtype,
+                     void *cuda_stream)
+{
+    return run_collective(heap, 1, in, out, send_count, (int)dtype, 0, (cudaStream_t)cuda_stream);
+}
+
+int symar_broadcast(symheap_t *heap, const void *in, void *out, size_t count, symar_dtype_t dtype, int root,
+                    void *cuda_stream)
+{
+    return run_collective(heap, 2, in, out, count, (int)dtype, root, (cudaStream_t)cuda_stream);
+}
+
+int symar_reduce(symheap_t *heap, const void *in, void *out, size_t count, symar_dtype_t dtype, int root,
+                 void *cuda_stream)
+{
+    return run_collective(heap, 3, in, out, count, (int)dtype, root, (cudaStream_t)cuda_stream);
 }
 
 int allreduce_autotune(symheap_t *heap, symar_dtype_t dtype)

@@ -40,6 +40,10 @@ SIGNATURES = [
     ("allreduce", c_int, [c_void_p, c_void_p, c_void_p, c_size_t, c_int, c_int, c_void_p]),
     ("allreduce_host", c_int, [c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, c_int, c_int,
                                c_void_p]),
+    ("symar_reduce_scatter", c_int, [c_void_p, c_void_p, c_void_p, c_size_t, c_int, c_void_p]),
+    ("symar_all_gather", c_int, [c_void_p, c_void_p, c_void_p, c_size_t, c_int, c_void_p]),
+    ("symar_broadcast", c_int, [c_void_p, c_void_p, c_void_p, c_size_t, c_int, c_int, c_void_p]),
+    ("symar_reduce", c_int, [c_void_p, c_void_p, c_void_p, c_size_t, c_int, c_int, c_void_p]),
     ("allreduce_autotune", c_int, [c_void_p, c_int]),
     ("symar_last_choice", c_int, [c_void_p, POINTER(c_int), POINTER(c_int), POINTER(c_int)]),
     ("symar_last_kernel", c_int, [c_void_p, POINTER(c_uint), POINTER(c_size_t)]),
@@ -193,6 +197,23 @@ class SymHeap:
         base = self.base
         _ck(self._lib.allreduce_host(self._h, host_in, host_out, base + in_off, base + out_off, count,
                                      dtype, algo, stream), "allreduce_host")
+
+    # -- sibling collectives (raw status codes; offsets become rank-0 symmetric addresses) --
+    def reduce_scatter(self, in_off, out_off, recv_count, dtype, stream=0) -> int:
+        return int(self._lib.symar_reduce_scatter(self._h, self.base + in_off, self.base + out_off, recv_count,
+                                                  dtype, stream))
+
+    def all_gather(self, in_off, out_off, send_count, dtype, stream=0) -> int:
+        return int(self._lib.symar_all_gather(self._h, self.base + in_off, self.base + out_off, send_count,
+                                              dtype, stream))
+
+    def broadcast(self, in_off, out_off, count, dtype, root, stream=0) -> int:
+        return int(self._lib.symar_broadcast(self._h, self.base + in_off, self.base + out_off, count, dtype,
+                                             root, stream))
+
+    def reduce(self, in_off, out_off, count, dtype, root, stream=0) -> int:
+        return int(self._lib.symar_reduce(self._h, self.base + in_off, self.base + out_off, count, dtype, root,
+                                          stream))
 
     # -- data movement helpers for heaps that live in a torch tensor --
     def _bytes_view(self, rank: int, offset: int, nbytes: int):
