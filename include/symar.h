@@ -207,6 +207,13 @@ int symar_query_choice(symheap_t *heap, size_t count, symar_dtype_t dtype,
 int symar_tuned_entry(const symheap_t *heap, symar_dtype_t dtype, int log2_bytes,
                       symar_algo_t algo, int *ctas_per_rank, int *threads, double *host_us);
 
+/* Write / read the tuned table as a small text file (host path), so that a
+ * deployment tunes once per machine.  Loading rejects a file written for another
+ * rank count or with out-of-range entries (SYMAR_ERR_INVAL); launch shapes are
+ * re-clamped to what is co-resident at call time in any case.                   */
+int symar_table_save(const symheap_t *heap, const char *host_path);
+int symar_table_load(symheap_t *heap, const char *host_path);
+
 /* Force the launch shape of one algorithm (0 = back to table/default).  The
  * library still clamps P * ctas_per_rank to what is co-resident on the device:
  * CTAs of different ranks wait for one another, so all must be resident.       */

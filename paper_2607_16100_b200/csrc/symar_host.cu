@@ -749,6 +749,84 @@ int symar_tuned_entry(const symheap_t *heap, symar_dtype_t dtype, int log2_bytes
     return SYMAR_OK;
 }
 
+// The tuned table as text: one header line, then per dtype and size bucket one "best"
+// line and one line per algorithm.  Lets a deployment tune once per machine.
+int symar_table_save(const symheap_t *heap, const char *host_path)
+{
+    if (!heap || !host_path) return SYMAR_ERR_INVAL;
+    FILE *f = std::fopen(host_path, "w");
+    if (!f) return SYMAR_ERR_INVAL;
+    std::fprintf(f, "symar-table 1 P %d\n", heap->P);
+    for (int dt = 0; dt < 2; ++dt) {
+        const Tuned &tn = heap->tuned[dt];
+        if (!tn.valid) continue;
+        std::fprintf(f, "dtype %d buckets %d %d\n", dt, tn.lo_bucket, tn.hi_bucket);
+        for (int b = tn.lo_bucket; b <= tn.hi_bucket; ++b) {
+            std::fprintf(f, "best %d %d\n", b, tn.best_algo[b]);
+            for (int a = SYMAR_ONESHOT; a < kAlgos; ++a)
+                std::fprintf(f, "cfg %d %d %d %d %d %.6g\n", b, a, tn.cfg[a][b].ctas, tn.cfg[a][b].threads,
+                             tn.cfg[a][b].variant, tn.us[a][b]);
+        }
+    }
+    return std::fclose(f) == 0 ? SYMAR_OK : SYMAR_ERR_INVAL;
+}
+
+int symar_table_load(symheap_t *heap, const char *host_path)
+{
+    if (!heap || !host_path) return SYMAR_ERR_INVAL;
+    FILE *f = std::fopen(host_path, "r");
+    if (!f) return SYMAR_ERR_INVAL;
+    int version = 0, P = 0;
+    if (std::fscanf(f, "symar-table %d P %d", &version, &P) != 2 || version != 1 || P != heap->P) {
+        std::fclose(f);
+        return SYMAR_ERR_INVAL;          // written for another rank count or format
+    }
+    Tuned loaded[2];
+    int dt = -1;
+    char word[16];
+    bool ok = true;
+    while (ok && std::fscanf(f, "%15s", word) == 1) {
+        const std::string w(word);
+        if (w == "dtype") {
+            int lo, hi;
+            ok = std::fscanf(f, "%d buckets %d %d", &dt, &lo, &hi) == 3 && dt >= 0 && dt < 2 && lo >= 0 &&
+                 hi < kBuckets && lo <= hi;
+            if (ok) {
+                loaded[dt]           = Tuned{};
+                loaded[dt].lo_bucket = lo;
+                loaded[dt].hi_bucket = hi;
+                loaded[dt].valid     = true;
+                for (int b = 0; b < kBuckets; ++b) {
+                    loaded[dt].best_algo[b] = SYMAR_ONESHOT;
+                    for (int a = 0; a < kAlgos; ++a) loaded[dt].us[a][b] = 1e30;
+                }
+            }
+        } else if (w == "best") {
+            int b, a;
+            ok = dt >= 0 && std::fscanf(f, "%d %d", &b, &a) == 2 && b >= 0 && b < kBuckets && a >= SYMAR_ONESHOT &&
+                 a < kAlgos;
+            if (ok) loaded[dt].best_algo[b] = a;
+        } else if (w == "cfg") {
+            int b, a, c, t, v;
+            double us;
+            ok = dt >= 0 && std::fscanf(f, "%d %d %d %d %d %lf", &b, &a, &c, &t, &v, &us) == 6 && b >= 0 &&
+                 b < kBuckets && a >= SYMAR_ONESHOT && a < kAlgos && c >= 0 && c <= kMaxCtas && t >= 0 &&
+                 t <= (int)kMaxThreads;
+            if (ok) {
+                loaded[dt].cfg[a][b] = LaunchCfg{c, t, v};
+                loaded[dt].us[a][b]  = us;
+            }
+        } else {
+            ok = false;
+        }
+    }
+    std::fclose(f);
+    if (!ok) return SYMAR_ERR_INVAL;
+    for (int d = 0; d < 2; ++d)
+        if (loaded[d].valid) heap->tuned[d] = loaded[d];
+    return SYMAR_OK;
+}
+
 int symar_set_launch(symheap_t *heap, symar_algo_t algo, int ctas_per_rank, int threads)
 {
     if (!heap || algo < SYMAR_ONESHOT || algo > SYMAR_SENTINEL) return SYMAR_ERR_INVAL;

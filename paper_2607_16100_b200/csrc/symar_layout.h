@@ -36,11 +36,13 @@ constexpr size_t   kMaxThreads  = 512;
 __host__ __device__ constexpr size_t ready_count_off(int c) { return (size_t)kMaxCtas * 8 + (size_t)c * 4; }
 __host__ __device__ constexpr size_t done_count_off(int c) { return (size_t)kMaxCtas * 12 + (size_t)c * 4; }
 
-// variant bits (performance experiments; same results)
-enum : uint32_t {
-    kVarLateCount = 1u,    // one-shot: publish the exchange count at kernel exit instead of
-                           // right after the exchange
-};
+// Variant bits carried in KArgs::variant (every variant computes the same bits):
+//   one-shot : bits 8-9 = bytes per thread (0: 16, 1: 8, 2: 4)
+//   LL       : bit 8    = 8 instead of 16 payload bytes per thread
+//   two-shot : bit 0 = contiguous chunks for large messages, bit 1 = 16-byte accesses,
+//              bit 2 = never the bulk-copy kernel, bits 8-10 = bulk pipeline depth,
+//              bits 12-13 = log2(bulk tile size / 4 KiB)
+//   sibling collectives: the unit size in bytes (16, 4 or 2)
 
 constexpr uint32_t kOneChunk     = 0xffu;   // KArgs::blk_log2: rank r owns one contiguous chunk
 constexpr uint32_t kCyclicLog2   = 9;       // block-cyclic block: 512 vectors = 8 KiB

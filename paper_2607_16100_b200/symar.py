@@ -50,6 +50,8 @@ SIGNATURES = [
     ("symar_query_choice", c_int, [c_void_p, c_size_t, c_int, POINTER(c_int), POINTER(c_int), POINTER(c_int)]),
     ("symar_tuned_entry", c_int, [c_void_p, c_int, c_int, c_int, POINTER(c_int), POINTER(c_int),
                                   POINTER(c_double)]),
+    ("symar_table_save", c_int, [c_void_p, c_char_p]),
+    ("symar_table_load", c_int, [c_void_p, c_char_p]),
     ("symar_set_launch", c_int, [c_void_p, c_int, c_int, c_int]),
     ("symar_set_variant", c_int, [c_void_p, c_int, c_uint]),
     ("symar_set_pdl", c_int, [c_void_p, c_int]),
@@ -269,6 +271,12 @@ class SymHeap:
         if rc != OK:
             return None
         return c.value, t.value, us.value
+
+    def table_save(self, path: str) -> None:
+        _ck(self._lib.symar_table_save(self._h, str(path).encode()), "symar_table_save")
+
+    def table_load(self, path: str) -> None:
+        _ck(self._lib.symar_table_load(self._h, str(path).encode()), "symar_table_load")
 
     def set_launch(self, algo: int, ctas_per_rank: int, threads: int) -> None:
         _ck(self._lib.symar_set_launch(self._h, algo, ctas_per_rank, threads), "symar_set_launch")

@@ -408,6 +408,34 @@ def test_auto_default_and_after_autotune():
         h.destroy()
 
 
+def test_tuned_table_round_trips_through_a_file(tmp_path):
+    a = symar.SymHeap.on_torch(4, 1 << 18)
+    b = symar.SymHeap.on_torch(4, 1 << 18)
+    c = symar.SymHeap.on_torch(2, 1 << 18)
+    try:
+        a.autotune(symar.BF16)
+        path = tmp_path / "table.txt"
+        a.table_save(path)
+        b.table_load(path)
+        for count in (8, 512, 8192, 50000):
+            assert a.query_choice(count, symar.BF16) == b.query_choice(count, symar.BF16)
+        for log2 in range(4, 17):
+            for algo in ALGOS:
+                assert a.tuned_entry(symar.BF16, log2, algo)[:2] == b.tuned_entry(symar.BF16, log2, algo)[:2]
+        with pytest.raises(symar.SymarError):
+            c.table_load(path)                       # written for another rank count
+        bad = tmp_path / "bad.txt"
+        bad.write_text("symar-table 1 P 4\ndtype 1 buckets 4 6\ncfg 5 2 9999 64 0 1.0\n")
+        with pytest.raises(symar.SymarError):
+            b.table_load(bad)
+        x = synth.make_inputs("normal", "bf16", 4, 8192, seed=1)
+        assert_bits(run(b, x, symar.BF16, symar.AUTO, in_off=0, out_off=1 << 17), O.allreduce(x))
+    finally:
+        torch.cuda.synchronize()
+        for h in (a, b, c):
+            h.destroy()
+
+
 # ---- errors --------------------------------------------------------------------------------
 
 def test_argument_errors(heaps):
