@@ -201,8 +201,9 @@ def latency_suite(torch, symar, synth, hbm_gbs, quick=False, autotune=True):
     out = {}
     stream = torch.cuda.Stream()
     K, reps = 64, (60 if quick else 300)
-    names = {symar.ONESHOT: "oneshot", symar.TWOSHOT: "twoshot", symar.LL: "ll", symar.SENTINEL: "sentinel",
-             symar.AUTO: "auto"}
+    names = dict(symar.ALGO_NAMES)
+    ALL = (symar.ONESHOT, symar.TWOSHOT, symar.LL, symar.SENTINEL, symar.TWOSHOT_LL, symar.TWOSHOT_SENTINEL,
+           symar.AUTO)
 
     # speed-of-light parts (paper Sec. VI), measured here
     fence_ns = symar.probe_fence(20000)
@@ -258,8 +259,7 @@ def latency_suite(torch, symar, synth, hbm_gbs, quick=False, autotune=True):
 
         # C2: 16 KiB per rank
         if P == 8:
-            row = bench_size(8192, (symar.ONESHOT, symar.TWOSHOT, symar.LL, symar.SENTINEL, symar.AUTO),
-                             stream_too=True)
+            row = bench_size(8192, ALL, stream_too=True)
             best = min(row.values(), key=lambda r: r["p50"])
             floor = empty_floor(best["ctas_per_rank"], P, best["threads"])
             floor11 = empty_floor(1, 1, 1)
@@ -291,7 +291,7 @@ def latency_suite(torch, symar, synth, hbm_gbs, quick=False, autotune=True):
         if P == 8:
             small = []
             for nbytes in (128, 1024, 4096):
-                row = bench_size(nbytes // 2, (symar.ONESHOT, symar.TWOSHOT, symar.LL, symar.SENTINEL, symar.AUTO))
+                row = bench_size(nbytes // 2, ALL)
                 fl = empty_floor(row["auto"]["ctas_per_rank"], P, row["auto"]["threads"])
                 s_ol = fl["p50"] + rt_ns / 1000.0 + 2 * P * nbytes / (hbm_gbs * 1e9) * 1e6
                 small.append({"bytes_per_rank": nbytes, "p50_us": {k: v["p50"] for k, v in row.items()},
@@ -345,7 +345,7 @@ def latency_suite(torch, symar, synth, hbm_gbs, quick=False, autotune=True):
         if P == 8:
             sweep = []
             for B in synth.WORKLOADS["c3"]["batch"]:
-                row = bench_size(8192 * B, (symar.ONESHOT, symar.TWOSHOT, symar.LL, symar.SENTINEL, symar.AUTO))
+                row = bench_size(8192 * B, ALL)
                 named = {k: v["p50"] for k, v in row.items() if k != "auto"}
                 best_name = min(named, key=named.get)
                 sweep.append({"bytes_per_rank": 16384 * B, "p50_us": {k: v["p50"] for k, v in row.items()},

@@ -48,10 +48,14 @@ typedef enum {
     SYMAR_ONESHOT = 1,   /* Sec. III-A.1, pull form: every rank reads all P inputs           */
     SYMAR_TWOSHOT = 2,   /* Sec. III-A.2: reduce-scatter, then all-gather with flag handoff  */
     SYMAR_LL      = 3,   /* Sec. IV "LL" + Sec. V example: one-shot push, data+flag stores   */
-    SYMAR_SENTINEL = 4   /* Sec. IV "Sentinel": one-shot push of bare data into scratch that
+    SYMAR_SENTINEL = 4,  /* Sec. IV "Sentinel": one-shot push of bare data into scratch that
                             holds a sentinel word; the receiver polls until every word has
-                            changed and restores the sentinel.  Never chosen by SYMAR_AUTO
-                            unless the tuner measured it to be fastest.                      */
+                            changed and restores the sentinel.                               */
+    SYMAR_TWOSHOT_LL = 5,       /* Table I "Two-shot (LL)": reduce-scatter and all-gather both
+                                   pushed through the LL scratch, synchronised by the data    */
+    SYMAR_TWOSHOT_SENTINEL = 6  /* Table I "Two-shot (Sentinel)": the same through the sentinel
+                                   scratch.  (SYMAR_AUTO picks algorithms 3..6 only where the
+                                   tuner measured them to be fastest.)                        */
 } symar_algo_t;
 
 enum {

@@ -24,7 +24,10 @@ struct LaunchCfg {
 };
 
 constexpr int kBuckets = 40;   // bucket b holds messages of (2^(b-1), 2^b] bytes per rank
-constexpr int kAlgos   = 5;    // indexed by symar_algo_t
+constexpr int kAlgos   = 7;    // indexed by symar_algo_t
+constexpr int kLastAlgo = SYMAR_TWOSHOT_SENTINEL;
+static bool is_push(int algo) { return algo >= SYMAR_LL; }            // uses per-slot scratch and epochs
+static bool is_twoshot_push(int algo) { return algo == SYMAR_TWOSHOT_LL || algo == SYMAR_TWOSHOT_SENTINEL; }
 
 struct Tuned {
     bool      valid = false;
@@ -121,7 +124,8 @@ static LaunchCfg default_cfg(const symheap *h, int algo, uint64_t nvec)
 {
     LaunchCfg c;
     c.variant = 0;
-    const uint64_t work = algo == SYMAR_TWOSHOT ? (nvec + h->P - 1) / h->P : nvec;   // vectors per rank partition
+    const uint64_t work = (algo == SYMAR_TWOSHOT || is_twoshot_push(algo)) ? (nvec + h->P - 1) / h->P
+                                                                            : nvec;   // vectors per rank partition
     if (algo == SYMAR_TWOSHOT && nvec >= kBulkMinVec) {
         // Bandwidth regime.  HBM3e delivers most when few, long streams are in
         // flight: about 100 CTAs in total, each with one 64 KiB stage (P tiles)
@@ -149,8 +153,7 @@ static LaunchCfg default_cfg(const symheap *h, int algo, uint64_t nvec)
     }
     c.threads = units >= 2048 ? 128 : round_threads(std::max<uint64_t>(units / 16, 32));
     uint64_t ctas = (units + c.threads - 1) / c.threads;
-    const uint64_t cap = (algo == SYMAR_LL || algo == SYMAR_SENTINEL) ? (uint64_t)kLLSlots
-                                                                       : (uint64_t)std::max(1, 2 * h->num_sms / h->P);
+    const uint64_t cap = is_push(algo) ? (uint64_t)kLLSlots : (uint64_t)std::max(1, 2 * h->num_sms / h->P);
     c.ctas = (int)std::max<uint64_t>(1, std::min(ctas, cap));
     return c;
 }
@@ -211,7 +214,7 @@ static int make_plan(symheap *h, size_t in_off, size_t out_off, size_t count, in
         p->smem     = bulk_smem_bytes(h->P, a.tile_vecs, a.stages);
     }
     if (!fn) return SYMAR_ERR_INVAL;
-    const int cap_slots = (algo == SYMAR_LL || algo == SYMAR_SENTINEL) ? kLLSlots : kMaxCtas;
+    const int cap_slots = is_push(algo) ? kLLSlots : kMaxCtas;
     const int cap_res   = std::max(1, max_resident(h, fn, cfg.threads, p->smem) / h->P);
     cfg.ctas = std::max(1, std::min({cfg.ctas, cap_slots, cap_res}));
 
@@ -239,11 +242,14 @@ static int make_plan(symheap *h, size_t in_off, size_t out_off, size_t count, in
         a.blk_log2 = cyclic ? kCyclicLog2 : kOneChunk;
         a.wide     = cyclic && ((in_off | out_off) % 32 == 0) && !(var & 2u);
     }
-    if (algo == SYMAR_LL || algo == SYMAR_SENTINEL) {
-        // every CTA takes `cv` vectors per iteration; iterations alternate sub-buffers
-        const uint64_t per_cta = (nvec + cfg.ctas - 1) / cfg.ctas;
-        a.cv    = (uint32_t)std::max<uint64_t>(1, std::min<uint64_t>(per_cta, kLLSlotVecs));
-        a.iters = (uint32_t)((nvec + (uint64_t)a.cv * cfg.ctas - 1) / ((uint64_t)a.cv * cfg.ctas));
+    if (is_push(algo)) {
+        // every CTA takes `cv` positions per iteration; iterations alternate sub-buffers.  The
+        // two-shot forms walk chunk positions and keep half of a scratch row for each phase.
+        const uint64_t span    = is_twoshot_push(algo) ? (nvec + h->P - 1) / h->P : nvec;
+        const uint64_t max_cv  = is_twoshot_push(algo) ? kLLSlotVecs / 2 : kLLSlotVecs;
+        const uint64_t per_cta = (span + cfg.ctas - 1) / cfg.ctas;
+        a.cv    = (uint32_t)std::max<uint64_t>(1, std::min<uint64_t>(per_cta, max_cv));
+        a.iters = (uint32_t)((span + (uint64_t)a.cv * cfg.ctas - 1) / ((uint64_t)a.cv * cfg.ctas));
     }
     p->algo = algo;
     p->cfg  = cfg;
@@ -275,7 +281,7 @@ static int run(symheap *h, const void *in, void *out, size_t count, int dtype, i
     size_t io = 0, oo = 0;
     int rc = check_buffers(h, in, out, count, dtype, &io, &oo);
     if (rc != SYMAR_OK) return rc;
-    if (algo < SYMAR_AUTO || algo > SYMAR_SENTINEL) return SYMAR_ERR_INVAL;
+    if (algo < SYMAR_AUTO || algo > kLastAlgo) return SYMAR_ERR_INVAL;
     if (count == 0) return SYMAR_OK;
     Plan p;
     rc = make_plan(h, io, oo, count, dtype, algo, &p);
@@ -429,12 +435,12 @@ static int autotune(symheap *h, int dtype)
         const int reps = 7;
         double best_us = 1e30;
         tn.best_algo[b] = SYMAR_ONESHOT;
-        for (int algo = SYMAR_ONESHOT; algo <= SYMAR_SENTINEL && rc == SYMAR_OK; ++algo) {
+        for (int algo = SYMAR_ONESHOT; algo <= kLastAlgo && rc == SYMAR_OK; ++algo) {
             tn.us[algo][b]  = 1e30;
             tn.cfg[algo][b] = LaunchCfg{};
-            if ((algo == SYMAR_LL || algo == SYMAR_SENTINEL) && bytes > (4u << 20)) continue;   // P M scratch traffic per rank: hopeless there
+            if (is_push(algo) && bytes > (4u << 20)) continue;   // scratch traffic through L2: hopeless there
             if (algo == SYMAR_ONESHOT && bytes > (32u << 20)) continue;
-            const uint64_t work = algo == SYMAR_TWOSHOT ? (nvec + h->P - 1) / h->P : nvec;
+            const uint64_t work = (algo == SYMAR_TWOSHOT || is_twoshot_push(algo)) ? (nvec + h->P - 1) / h->P : nvec;
             // kernel variants worth timing: the default; for two-shot in the bandwidth
             // regime the bulk kernel's tile sizes and depths, and the register kernel
             std::vector<int> variants = {0};
@@ -524,7 +530,7 @@ static int create_common(symheap_t **heap, int P, size_t bytes_per_rank, void *m
     }
     // Load every kernel this heap can launch now, so that a first call made
     // during stream capture does not trigger lazy module loading there.
-    for (int algo = SYMAR_ONESHOT; algo <= SYMAR_SENTINEL && e == cudaSuccess; ++algo)
+    for (int algo = SYMAR_ONESHOT; algo <= kLastAlgo && e == cudaSuccess; ++algo)
         for (int dt = SYMAR_F32; dt <= SYMAR_BF16 && e == cudaSuccess; ++dt) {
             cudaFuncAttributes attr;
             e = cudaFuncGetAttributes(&attr, kernel_for(algo, dt, P, false));
@@ -550,7 +556,8 @@ static int create_common(symheap_t **heap, int P, size_t bytes_per_rank, void *m
     }
     if (const char *v = std::getenv("SYMAR_ALGO")) {
         const std::string a(v);
-        h->env_algo = a == "oneshot" ? SYMAR_ONESHOT : a == "twoshot" ? SYMAR_TWOSHOT : a == "ll" ? SYMAR_LL : a == "sentinel" ? SYMAR_SENTINEL : 0;
+        h->env_algo = a == "oneshot" ? SYMAR_ONESHOT : a == "twoshot" ? SYMAR_TWOSHOT : a == "ll" ? SYMAR_LL : a == "sentinel" ? SYMAR_SENTINEL
+                      : a == "twoshot_ll" ? SYMAR_TWOSHOT_LL : a == "twoshot_sentinel" ? SYMAR_TWOSHOT_SENTINEL : 0;
     }
     if (const char *v = std::getenv("SYMAR_PDL")) h->pdl = std::atoi(v) != 0;
     *heap = h;
@@ -742,7 +749,7 @@ int symar_tuned_entry(const symheap_t *heap, symar_dtype_t dtype, int log2_bytes
     if (!heap || (dtype != SYMAR_F32 && dtype != SYMAR_BF16)) return SYMAR_ERR_INVAL;
     const Tuned &tn = heap->tuned[(int)dtype];
     if (!tn.valid || log2_bytes < tn.lo_bucket || log2_bytes > tn.hi_bucket) return SYMAR_ERR_INVAL;
-    if (algo < SYMAR_ONESHOT || algo > SYMAR_SENTINEL) return SYMAR_ERR_INVAL;
+    if (algo < SYMAR_ONESHOT || algo > kLastAlgo) return SYMAR_ERR_INVAL;
     if (ctas_per_rank) *ctas_per_rank = tn.cfg[algo][log2_bytes].ctas;
     if (threads) *threads = tn.cfg[algo][log2_bytes].threads;
     if (host_us) *host_us = tn.us[algo][log2_bytes];
@@ -829,7 +836,7 @@ int symar_table_load(symheap_t *heap, const char *host_path)
 
 int symar_set_launch(symheap_t *heap, symar_algo_t algo, int ctas_per_rank, int threads)
 {
-    if (!heap || algo < SYMAR_ONESHOT || algo > SYMAR_SENTINEL) return SYMAR_ERR_INVAL;
+    if (!heap || algo < SYMAR_ONESHOT || algo > kLastAlgo) return SYMAR_ERR_INVAL;
     if (ctas_per_rank < 0 || threads < 0 || threads > (int)kMaxThreads) return SYMAR_ERR_INVAL;
     heap->forced[algo] = LaunchCfg{ctas_per_rank, threads};
     return SYMAR_OK;
@@ -837,7 +844,7 @@ int symar_set_launch(symheap_t *heap, symar_algo_t algo, int ctas_per_rank, int 
 
 int symar_set_variant(symheap_t *heap, symar_algo_t algo, unsigned int variant)
 {
-    if (!heap || algo < SYMAR_ONESHOT || algo > SYMAR_SENTINEL) return SYMAR_ERR_INVAL;
+    if (!heap || algo < SYMAR_ONESHOT || algo > kLastAlgo) return SYMAR_ERR_INVAL;
     heap->variant[algo]        = variant & 0x7fffffffu;
     heap->variant_forced[algo] = variant != 0;       // bit 31 alone forces the plain variant 0
     return SYMAR_OK;

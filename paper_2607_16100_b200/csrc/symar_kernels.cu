@@ -426,6 +426,150 @@ __global__ void __launch_bounds__(kMaxThreads) sentinel_kernel(const KArgs a)
     if (t == 0) *ep = n0 + a.iters;
 }
 
+// ---- two-shot over the push buffers (the paper's AllReduce_LLBuffer_Twoshot; Table I rows
+//      "Two-shot (LL)" and "Two-shot (Sentinel)") ------------------------------------------
+// Rank r pushes vector p of chunk q of its input into rank q's scratch, every rank
+// reduces the chunk it owns, pushes the reduced vector into every peer's scratch and
+// collects the other chunks from its own scratch.  Two synchronisations, both carried
+// by the data (LL flag words or the sentinel), none by a barrier; per-rank volume
+// 2 (P-1) M / P payload bytes (twice that with LL flags).  The first half of a scratch
+// row takes the reduce-scatter traffic, the second half the all-gather traffic.
+template <bool SENT>
+struct PushRow {
+    static constexpr size_t kRowBytes = SENT ? kSnSenderBytes : kLLSenderBytes;
+    __device__ static __forceinline__ void send(char *row, uint32_t j, const uint4 &x, uint32_t e)
+    {
+        if (SENT) {
+            st_relaxed_v4(row + (size_t)j * 16, x);
+        } else {
+            const uint64_t hi_e = (uint64_t)e << 32;
+            st_relaxed_v2u64(row + (size_t)j * 16, hi_e | x.x, hi_e | x.y);
+            st_relaxed_v2u64(row + (size_t)kLLSlotVecs * 16 + (size_t)j * 16, hi_e | x.z, hi_e | x.w);
+        }
+    }
+    // true when the vector has arrived (sentinel mode then restores the sentinel)
+    __device__ static __forceinline__ bool try_recv(char *row, uint32_t j, uint32_t e, uint4 &x)
+    {
+        if (SENT) {
+            const uint4 d = ld_relaxed_v4(row + (size_t)j * 16);
+            if (d.x == kSentinelWord || d.y == kSentinelWord || d.z == kSentinelWord || d.w == kSentinelWord)
+                return false;
+            x = d;
+            st_relaxed_v4(row + (size_t)j * 16,
+                          make_uint4(kSentinelWord, kSentinelWord, kSentinelWord, kSentinelWord));
+            return true;
+        } else {
+            const U64x2 lo = ld_relaxed_v2u64(row + (size_t)j * 16);
+            const U64x2 hi = ld_relaxed_v2u64(row + (size_t)kLLSlotVecs * 16 + (size_t)j * 16);
+            if ((uint32_t)(lo.a >> 32) != e || (uint32_t)(lo.b >> 32) != e || (uint32_t)(hi.a >> 32) != e ||
+                (uint32_t)(hi.b >> 32) != e)
+                return false;
+            x = make_uint4((uint32_t)lo.a, (uint32_t)lo.b, (uint32_t)hi.a, (uint32_t)hi.b);
+            return true;
+        }
+    }
+    // sentinel mode cannot carry a word equal to the sentinel: clear its lowest bit (still a NaN)
+    __device__ static __forceinline__ uint4 clean(const uint4 &x)
+    {
+        if (!SENT) return x;
+        auto c = [](uint32_t w) { return w == kSentinelWord ? (kSentinelWord & ~1u) : w; };
+        return make_uint4(c(x.x), c(x.y), c(x.z), c(x.w));
+    }
+};
+
+template <typename E, int P, bool SENT, bool DBG>
+__global__ void __launch_bounds__(kMaxThreads) twoshot_push_kernel(const KArgs a)
+{
+    using Row = PushRow<SENT>;
+    const int c = blockIdx.x, r = blockIdx.y, C = gridDim.x;
+    const uint32_t t = threadIdx.x, T = blockDim.x;
+    char *seg_r  = a.seg0 + (size_t)r * a.stride;
+    uint64_t *ep = reinterpret_cast<uint64_t *>(seg_r + a.epoch_off) + c;
+    if (a.pdl) {
+        pdl_wait();
+        pdl_launch_dependents();
+    }
+    const uint64_t n0 = ld_relaxed_u64(ep);
+    if (DBG) debug_delay(a, r, c);
+    if (DBG && a.dbg_mute == r) return;       // test hook: this rank never joins
+
+    const char *in = seg_r + a.in_off;
+    char *out      = seg_r + a.out_off;
+    const uint64_t chv  = (a.nvec + P - 1) / P;            // vectors per chunk; chunk q = [q chv, (q+1) chv)
+    const uint32_t half = kLLSlotVecs / 2;                 // all-gather positions start here
+    bool failed = false;
+
+    for (uint32_t it = 0; it < a.iters && !failed; ++it) {
+        const uint64_t n  = n0 + 1 + it;
+        const uint32_t e  = flag_of(n);
+        const uint64_t p0 = ((uint64_t)it * C + c) * a.cv;             // first chunk position of this CTA
+        const uint32_t cnt = p0 < chv ? (uint32_t)(chv - p0 < a.cv ? chv - p0 : a.cv) : 0u;
+        const uint64_t region = (SENT ? a.sn_off : a.ll_off) + ((uint64_t)(n & 1) * kLLSlots + c) * P * Row::kRowBytes;
+        auto valid = [&](int q, uint64_t p) { return (uint64_t)q * chv + p < a.nvec; };
+        // my row r in rank q's region / rank q's row in my region
+        auto peer_row = [&](int q) { return a.seg0 + (size_t)q * a.stride + region + (size_t)r * Row::kRowBytes; };
+        auto my_row   = [&](int q) { return seg_r + region + (size_t)q * Row::kRowBytes; };
+
+        for (uint32_t k = t; k < cnt; k += T) {                        // reduce-scatter: push
+#pragma unroll
+            for (int q = 0; q < P; ++q)
+                if (q != r && valid(q, p0 + k))
+                    Row::send(peer_row(q), k, Row::clean(ld_own(in + ((uint64_t)q * chv + p0 + k) * 16)), e);
+        }
+        for (uint32_t k = t; k < cnt && !failed; k += T) {
+            const uint64_t p = p0 + k;
+            if (valid(r, p)) {                                          // reduce the owned vector
+                uint4 x[P];
+                unsigned need = ((1u << P) - 1u) & ~(1u << r);
+                Spin spin;
+                while (need != 0) {
+#pragma unroll
+                    for (int q = 0; q < P; ++q)
+                        if ((need >> q & 1u) && Row::try_recv(my_row(q), k, e, x[q])) need &= ~(1u << q);
+                    if (need != 0 && spin.due() && spin.expired(a.spin_ns)) {
+                        report_timeout(a.ctl, r, __ffs(need) - 1, c);
+                        failed = true;
+                        break;
+                    }
+                }
+                if (failed) break;
+                const uint4 own = Row::clean(ld_own(in + ((uint64_t)r * chv + p) * 16));
+#pragma unroll
+                for (int q = 0; q < P; ++q)
+                    if (q == r) x[q] = own;
+                const uint4 res = Row::clean(reduce_in_rank_order<E, P>(x));
+#pragma unroll
+                for (int q = 0; q < P; ++q)                             // all-gather: push
+                    if (q != r) Row::send(peer_row(q), half + k, res, e);
+                store_result(out, (uint64_t)r * chv + p, res, a.nvec, a.tail_bytes);
+            }
+            unsigned need = 0;                                          // all-gather: collect
+#pragma unroll
+            for (int q = 0; q < P; ++q)
+                if (q != r && valid(q, p)) need |= 1u << q;
+            Spin spin;
+            while (need != 0) {
+#pragma unroll
+                for (int q = 0; q < P; ++q) {
+                    uint4 d;
+                    if ((need >> q & 1u) && Row::try_recv(my_row(q), half + k, e, d)) {
+                        store_result(out, (uint64_t)q * chv + p, d, a.nvec, a.tail_bytes);
+                        need &= ~(1u << q);
+                    }
+                }
+                if (need != 0 && spin.due() && spin.expired(a.spin_ns)) {
+                    report_timeout(a.ctl, r, __ffs(need) - 1, c);
+                    failed = true;
+                    break;
+                }
+            }
+        }
+        if (SENT && a.iters > 1) fence_acq_rel();      // restored sentinels before the sub-buffer's next use
+    }
+    __syncthreads();
+    if (t == 0) *ep = n0 + a.iters;
+}
+
 // ---- dispatch ---------------------------------------------------------------------
 
 template <typename E, int P, bool DBG>
@@ -436,6 +580,8 @@ static KernelFn pick_algo(int algo)
         case SYMAR_TWOSHOT: return twoshot_kernel<E, P, DBG>;
         case SYMAR_LL:      return ll_kernel<E, P, DBG>;
         case SYMAR_SENTINEL: return sentinel_kernel<E, P, DBG>;
+        case SYMAR_TWOSHOT_LL: return twoshot_push_kernel<E, P, false, DBG>;
+        case SYMAR_TWOSHOT_SENTINEL: return twoshot_push_kernel<E, P, true, DBG>;
     }
     return nullptr;
 }

@@ -14,8 +14,9 @@ _PKG = Path(__file__).resolve().parent
 LIB_PATH = _PKG / "libsymar.so"
 
 F32, BF16 = 0, 1
-AUTO, ONESHOT, TWOSHOT, LL, SENTINEL = 0, 1, 2, 3, 4
-ALGO_NAMES = {AUTO: "auto", ONESHOT: "oneshot", TWOSHOT: "twoshot", LL: "ll", SENTINEL: "sentinel"}
+AUTO, ONESHOT, TWOSHOT, LL, SENTINEL, TWOSHOT_LL, TWOSHOT_SENTINEL = 0, 1, 2, 3, 4, 5, 6
+ALGO_NAMES = {AUTO: "auto", ONESHOT: "oneshot", TWOSHOT: "twoshot", LL: "ll", SENTINEL: "sentinel",
+              TWOSHOT_LL: "twoshot_ll", TWOSHOT_SENTINEL: "twoshot_sentinel"}
 DTYPE_NAMES = {F32: "f32", BF16: "bf16"}
 DTYPE_SIZE = {F32: 4, BF16: 2}
 

@@ -9,7 +9,8 @@ from paper_2607_16100_b200 import symar, synth
 
 pytestmark = pytest.mark.gpu
 
-ALGOS = [symar.ONESHOT, symar.TWOSHOT, symar.LL, symar.SENTINEL, symar.AUTO]
+ALGOS = [symar.ONESHOT, symar.TWOSHOT, symar.LL, symar.SENTINEL, symar.TWOSHOT_LL, symar.TWOSHOT_SENTINEL,
+         symar.AUTO]
 DT = {"f32": symar.F32, "bf16": symar.BF16}
 NP = {"f32": np.float32, "bf16": np.uint16}
 

@@ -9,7 +9,7 @@ from paper_2607_16100_b200 import symar, synth
 
 pytestmark = pytest.mark.gpu
 
-ALGOS = [symar.ONESHOT, symar.TWOSHOT, symar.LL, symar.SENTINEL]
+ALGOS = [symar.ONESHOT, symar.TWOSHOT, symar.LL, symar.SENTINEL, symar.TWOSHOT_LL, symar.TWOSHOT_SENTINEL]
 NP_DT = {symar.F32: np.float32, symar.BF16: np.uint16}
 DT = {"f32": symar.F32, "bf16": symar.BF16}
 USER = 8 << 20          # user region per rank of the shared test heaps
@@ -134,7 +134,7 @@ def test_forced_launch_shapes(heaps, algo, ctas, threads):
     assert_bits(got, O.allreduce(x))
 
 
-@pytest.mark.parametrize("algo", [symar.LL, symar.SENTINEL])
+@pytest.mark.parametrize("algo", [symar.LL, symar.SENTINEL, symar.TWOSHOT_LL, symar.TWOSHOT_SENTINEL])
 def test_push_many_iterations_alternate_subbuffers(heaps, algo):
     # one CTA per rank, 1024 vectors per iteration: 300000 fp32 -> 75000 vectors -> 74 iterations
     h = heaps[4]
@@ -159,10 +159,13 @@ def test_sentinel_mode_accepts_payload_equal_to_the_sentinel(heaps):
     xw = x.view(np.uint32)
     xw[rng.integers(0, 8, 300), rng.integers(0, 4096, 300)] = 0xFFFFFFFF
     want = O.allreduce(x)
-    got = run(h, x, symar.F32, symar.SENTINEL)
-    assert np.array_equal(np.isnan(got), np.isnan(want)) and np.isnan(want).sum() >= 250
-    keep = ~np.isnan(want)
-    assert_bits(np.where(keep, got, np.float32(0)), np.where(keep, want, np.float32(0)))
+    for algo in (symar.SENTINEL, symar.TWOSHOT_SENTINEL):
+        got = run(h, x, symar.F32, algo)
+        assert np.array_equal(np.isnan(got), np.isnan(want)) and np.isnan(want).sum() >= 250
+        keep = ~np.isnan(want)
+        assert_bits(np.where(keep, got, np.float32(0)), np.where(keep, want, np.float32(0)))
+        for q in range(1, 8):                 # every rank holds the same bits, NaN payloads included
+            assert np.array_equal(got[q].view(np.uint32), got[0].view(np.uint32))
     xb = synth.make_inputs("normal", "bf16", 8, 4096, seed=4)
     xb.view(np.uint32)[rng.integers(0, 8, 200), rng.integers(0, 2048, 200)] = 0xFFFFFFFF
     wantb = O.allreduce(xb)
@@ -183,7 +186,8 @@ FORCE_PLAIN = 1 << 31
                                           (1, "f32", "uniform")])
 @pytest.mark.parametrize("algo,variant", [(symar.ONESHOT, FORCE_PLAIN), (symar.ONESHOT, 0x100),
                                           (symar.ONESHOT, 0x200), (symar.LL, FORCE_PLAIN), (symar.LL, 0x100),
-                                          (symar.SENTINEL, FORCE_PLAIN)])
+                                          (symar.SENTINEL, FORCE_PLAIN), (symar.TWOSHOT_LL, FORCE_PLAIN),
+                                          (symar.TWOSHOT_SENTINEL, FORCE_PLAIN)])
 def test_unit_width_variants(heaps, algo, variant, P, dtype, dist, count):
     # 16, 8 or 4 bytes per thread: same bits, whatever the ragged tail
     h = heaps[P]
