@@ -341,6 +341,44 @@ def latency_suite(torch, symar, synth, hbm_gbs, quick=False, autotune=True):
                 r = time_graph(torch, g, stream, K, reps)
                 sib[name] = {"p50_us": r["p50"], "bit_exact": exact and h.status()[0] == 0}
             out["sibling_collectives_16KB"] = sib
+        # Sec. VII "Impact of Scratch Buffer": a 32 MiB message through the push algorithms with
+        # ever smaller scratch, i.e. more iterations, each with its own synchronisation
+        if P == 8 and not quick:
+            hs = symar.SymHeap.on_torch(P, 64 << 20)
+            cnt32 = (32 << 20) // 2
+            xs32 = synth.make_inputs("normal", "bf16", P, cnt32, 77)
+            for q in range(P):
+                hs.write_rank(q, 0, xs32[q])
+            want32 = O.allreduce_timed_team(xs32, threads=0)[0][0]
+            sweep32 = []
+            for limit in (16 << 10, 64 << 10, 256 << 10, 1 << 20):
+                hs.set_scratch_limit(limit)
+                row = {"scratch_payload_bytes_per_iteration": limit, "ms": {}, "bit_exact": True}
+                for algo in (symar.LL, symar.SENTINEL, symar.TWOSHOT_LL, symar.TWOSHOT_SENTINEL):
+                    with torch.cuda.stream(stream):
+                        hs.allreduce(0, 32 << 20, cnt32, symar.BF16, algo, stream.cuda_stream)
+                        a_, b_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                        a_.record(stream)
+                        for _ in range(3):
+                            hs.allreduce(0, 32 << 20, cnt32, symar.BF16, algo, stream.cuda_stream)
+                        b_.record(stream)
+                    stream.synchronize()
+                    row["ms"][names[algo]] = a_.elapsed_time(b_) / 3
+                    got = hs.read_rank(P - 1, 32 << 20, cnt32, np.uint16)
+                    row["bit_exact"] = row["bit_exact"] and bool(np.array_equal(got, want32)) and hs.status()[0] == 0
+                sweep32.append(row)
+            hs.set_scratch_limit(0)
+            with torch.cuda.stream(stream):
+                a_, b_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                hs.allreduce(0, 32 << 20, cnt32, symar.BF16, symar.TWOSHOT, stream.cuda_stream)
+                a_.record(stream)
+                for _ in range(3):
+                    hs.allreduce(0, 32 << 20, cnt32, symar.BF16, symar.TWOSHOT, stream.cuda_stream)
+                b_.record(stream)
+            stream.synchronize()
+            out["scratch_sweep_32MiB"] = {"rows": sweep32, "flag_twoshot_ms_for_reference": a_.elapsed_time(b_) / 3}
+            hs.destroy()
+            del xs32
         # C3: sweep
         if P == 8:
             sweep = []

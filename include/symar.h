@@ -240,6 +240,13 @@ int symar_set_variant(symheap_t *heap, symar_algo_t algo, unsigned int variant);
  * unchanged -- only launch latency of back-to-back calls is hidden.            */
 int symar_set_pdl(symheap_t *heap, int enabled);
 
+/* Pretend the push algorithms (LL, sentinel, and their two-shot forms) had a smaller
+ * scratch buffer: at most `payload_bytes_per_iteration` bytes of each rank's message are
+ * reduced per iteration (Table I's D), so larger messages take more iterations, each
+ * with its own synchronisation (Sec. VII "Impact of Scratch Buffer").  0 = use all of
+ * the scratch (1 MiB of payload per rank and iteration for the one-shot forms).       */
+int symar_set_scratch_limit(symheap_t *heap, size_t payload_bytes_per_iteration);
+
 /* Upper bound of any device-side wait, in microseconds (default 2 000 000). */
 int symar_set_spin_limit_us(symheap_t *heap, unsigned int microseconds);
 

@@ -68,6 +68,7 @@ struct symheap {
     uint64_t  spin_ns = 2000000000ull;
     bool      pdl          = false;
     int       env_algo     = 0;       // SYMAR_ALGO override of SYMAR_AUTO, 0 = none
+    size_t    scratch_limit = 0;      // push algorithms: payload bytes per rank and iteration, 0 = all there is
     int       dbg_mute     = -1;
     unsigned  dbg_seed     = 0;
     unsigned  dbg_delay_ns = 0;
@@ -196,7 +197,8 @@ static int make_plan(symheap *h, size_t in_off, size_t out_off, size_t count, in
     if (cfg.variant < 0) cfg.variant = 0;
     const unsigned var = (unsigned)cfg.variant;
 
-    cfg.threads = std::min<int>(std::max(32, (cfg.threads + 31) / 32 * 32), (int)kMaxThreads);
+    cfg.threads = std::min<int>(std::max(32, (cfg.threads + 31) / 32 * 32),
+                                is_twoshot_push(algo) ? (int)kPushTwoshotMaxThreads : (int)kMaxThreads);
     KArgs &a = p->args;
     std::memset(&a, 0, sizeof a);
     KernelFn fn = kernel_for(algo, dtype, h->P, dbg_on(h));
@@ -249,6 +251,10 @@ static int make_plan(symheap *h, size_t in_off, size_t out_off, size_t count, in
         const uint64_t max_cv  = is_twoshot_push(algo) ? kLLSlotVecs / 2 : kLLSlotVecs;
         const uint64_t per_cta = (span + cfg.ctas - 1) / cfg.ctas;
         a.cv    = (uint32_t)std::max<uint64_t>(1, std::min<uint64_t>(per_cta, max_cv));
+        if (h->scratch_limit) {      // a smaller scratch buffer: fewer positions per iteration, more iterations
+            const uint64_t per_iter = std::max<uint64_t>(1, h->scratch_limit / 16 / (is_twoshot_push(algo) ? h->P : 1));
+            a.cv = (uint32_t)std::max<uint64_t>(1, std::min<uint64_t>(a.cv, per_iter / cfg.ctas));
+        }
         a.iters = (uint32_t)((span + (uint64_t)a.cv * cfg.ctas - 1) / ((uint64_t)a.cv * cfg.ctas));
     }
     p->algo = algo;
@@ -854,6 +860,13 @@ int symar_set_pdl(symheap_t *heap, int enabled)
 {
     if (!heap) return SYMAR_ERR_INVAL;
     heap->pdl = enabled != 0;
+    return SYMAR_OK;
+}
+
+int symar_set_scratch_limit(symheap_t *heap, size_t payload_bytes_per_iteration)
+{
+    if (!heap) return SYMAR_ERR_INVAL;
+    heap->scratch_limit = payload_bytes_per_iteration;
     return SYMAR_OK;
 }
 

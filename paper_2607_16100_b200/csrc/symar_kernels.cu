@@ -447,24 +447,40 @@ struct PushRow {
             st_relaxed_v2u64(row + (size_t)kLLSlotVecs * 16 + (size_t)j * 16, hi_e | x.z, hi_e | x.w);
         }
     }
+    // Receiving is split into load / check so that a caller can put the loads of all
+    // peers in flight before it looks at any of them.
+    struct Raw { U64x2 lo, hi; };        // sentinel mode uses `lo` only (one 16-byte vector)
+    __device__ static __forceinline__ Raw load(const char *row, uint32_t j)
+    {
+        Raw d;
+        if (SENT) {
+            const uint4 v = ld_relaxed_v4(row + (size_t)j * 16);
+            d.lo.a = (uint64_t)v.y << 32 | v.x;
+            d.lo.b = (uint64_t)v.w << 32 | v.z;
+            d.hi   = d.lo;
+        } else {
+            d.lo = ld_relaxed_v2u64(row + (size_t)j * 16);
+            d.hi = ld_relaxed_v2u64(row + (size_t)kLLSlotVecs * 16 + (size_t)j * 16);
+        }
+        return d;
+    }
     // true when the vector has arrived (sentinel mode then restores the sentinel)
-    __device__ static __forceinline__ bool try_recv(char *row, uint32_t j, uint32_t e, uint4 &x)
+    __device__ static __forceinline__ bool check(char *row, uint32_t j, const Raw &d, uint32_t e, uint4 &x)
     {
         if (SENT) {
-            const uint4 d = ld_relaxed_v4(row + (size_t)j * 16);
-            if (d.x == kSentinelWord || d.y == kSentinelWord || d.z == kSentinelWord || d.w == kSentinelWord)
+            const uint4 v = make_uint4((uint32_t)d.lo.a, (uint32_t)(d.lo.a >> 32), (uint32_t)d.lo.b,
+                                       (uint32_t)(d.lo.b >> 32));
+            if (v.x == kSentinelWord || v.y == kSentinelWord || v.z == kSentinelWord || v.w == kSentinelWord)
                 return false;
-            x = d;
+            x = v;
             st_relaxed_v4(row + (size_t)j * 16,
                           make_uint4(kSentinelWord, kSentinelWord, kSentinelWord, kSentinelWord));
             return true;
         } else {
-            const U64x2 lo = ld_relaxed_v2u64(row + (size_t)j * 16);
-            const U64x2 hi = ld_relaxed_v2u64(row + (size_t)kLLSlotVecs * 16 + (size_t)j * 16);
-            if ((uint32_t)(lo.a >> 32) != e || (uint32_t)(lo.b >> 32) != e || (uint32_t)(hi.a >> 32) != e ||
-                (uint32_t)(hi.b >> 32) != e)
+            if ((uint32_t)(d.lo.a >> 32) != e || (uint32_t)(d.lo.b >> 32) != e || (uint32_t)(d.hi.a >> 32) != e ||
+                (uint32_t)(d.hi.b >> 32) != e)
                 return false;
-            x = make_uint4((uint32_t)lo.a, (uint32_t)lo.b, (uint32_t)hi.a, (uint32_t)hi.b);
+            x = make_uint4((uint32_t)d.lo.a, (uint32_t)d.lo.b, (uint32_t)d.hi.a, (uint32_t)d.hi.b);
             return true;
         }
     }
@@ -478,7 +494,7 @@ struct PushRow {
 };
 
 template <typename E, int P, bool SENT, bool DBG>
-__global__ void __launch_bounds__(kMaxThreads) twoshot_push_kernel(const KArgs a)
+__global__ void __launch_bounds__(kPushTwoshotMaxThreads) twoshot_push_kernel(const KArgs a)
 {
     using Row = PushRow<SENT>;
     const int c = blockIdx.x, r = blockIdx.y, C = gridDim.x;
@@ -511,10 +527,13 @@ __global__ void __launch_bounds__(kMaxThreads) twoshot_push_kernel(const KArgs a
         auto my_row   = [&](int q) { return seg_r + region + (size_t)q * Row::kRowBytes; };
 
         for (uint32_t k = t; k < cnt; k += T) {                        // reduce-scatter: push
+            uint4 mine[P];
 #pragma unroll
             for (int q = 0; q < P; ++q)
-                if (q != r && valid(q, p0 + k))
-                    Row::send(peer_row(q), k, Row::clean(ld_own(in + ((uint64_t)q * chv + p0 + k) * 16)), e);
+                if (q != r && valid(q, p0 + k)) mine[q] = ld_own(in + ((uint64_t)q * chv + p0 + k) * 16);
+#pragma unroll
+            for (int q = 0; q < P; ++q)
+                if (q != r && valid(q, p0 + k)) Row::send(peer_row(q), k, Row::clean(mine[q]), e);
         }
         for (uint32_t k = t; k < cnt && !failed; k += T) {
             const uint64_t p = p0 + k;
@@ -523,9 +542,13 @@ __global__ void __launch_bounds__(kMaxThreads) twoshot_push_kernel(const KArgs a
                 unsigned need = ((1u << P) - 1u) & ~(1u << r);
                 Spin spin;
                 while (need != 0) {
+                    typename Row::Raw d[P];
 #pragma unroll
                     for (int q = 0; q < P; ++q)
-                        if ((need >> q & 1u) && Row::try_recv(my_row(q), k, e, x[q])) need &= ~(1u << q);
+                        if (need >> q & 1u) d[q] = Row::load(my_row(q), k);
+#pragma unroll
+                    for (int q = 0; q < P; ++q)
+                        if ((need >> q & 1u) && Row::check(my_row(q), k, d[q], e, x[q])) need &= ~(1u << q);
                     if (need != 0 && spin.due() && spin.expired(a.spin_ns)) {
                         report_timeout(a.ctl, r, __ffs(need) - 1, c);
                         failed = true;
@@ -549,11 +572,15 @@ __global__ void __launch_bounds__(kMaxThreads) twoshot_push_kernel(const KArgs a
                 if (q != r && valid(q, p)) need |= 1u << q;
             Spin spin;
             while (need != 0) {
+                typename Row::Raw d[P];
+#pragma unroll
+                for (int q = 0; q < P; ++q)
+                    if (need >> q & 1u) d[q] = Row::load(my_row(q), half + k);
 #pragma unroll
                 for (int q = 0; q < P; ++q) {
-                    uint4 d;
-                    if ((need >> q & 1u) && Row::try_recv(my_row(q), half + k, e, d)) {
-                        store_result(out, (uint64_t)q * chv + p, d, a.nvec, a.tail_bytes);
+                    uint4 v;
+                    if ((need >> q & 1u) && Row::check(my_row(q), half + k, d[q], e, v)) {
+                        store_result(out, (uint64_t)q * chv + p, v, a.nvec, a.tail_bytes);
                         need &= ~(1u << q);
                     }
                 }

@@ -56,6 +56,7 @@ SIGNATURES = [
     ("symar_set_launch", c_int, [c_void_p, c_int, c_int, c_int]),
     ("symar_set_variant", c_int, [c_void_p, c_int, c_uint]),
     ("symar_set_pdl", c_int, [c_void_p, c_int]),
+    ("symar_set_scratch_limit", c_int, [c_void_p, c_size_t]),
     ("symar_set_spin_limit_us", c_int, [c_void_p, c_uint]),
     ("symar_debug_inject", c_int, [c_void_p, c_int, c_uint, c_uint]),
     ("allreduce_static", c_int, [c_void_p, c_void_p, c_size_t, c_int, c_size_t, c_int, c_void_p, c_void_p]),
@@ -287,6 +288,9 @@ class SymHeap:
 
     def set_pdl(self, enabled: bool) -> None:
         _ck(self._lib.symar_set_pdl(self._h, 1 if enabled else 0), "symar_set_pdl")
+
+    def set_scratch_limit(self, payload_bytes_per_iteration: int) -> None:
+        _ck(self._lib.symar_set_scratch_limit(self._h, payload_bytes_per_iteration), "symar_set_scratch_limit")
 
     def set_spin_limit_us(self, us: int) -> None:
         _ck(self._lib.symar_set_spin_limit_us(self._h, us), "symar_set_spin_limit_us")

@@ -128,7 +128,8 @@ def test_forced_launch_shapes(heaps, algo, ctas, threads):
     try:
         got = run(h, x, symar.BF16, algo)
         a, c, t = h.last_choice()
-        assert (a, c, t) == (algo, ctas, threads)
+        cap = 256 if algo in (symar.TWOSHOT_LL, symar.TWOSHOT_SENTINEL) else 512    # register-heavy kernel
+        assert (a, c, t) == (algo, ctas, min(threads, cap))
     finally:
         h.set_launch(algo, 0, 0)
     assert_bits(got, O.allreduce(x))
@@ -147,6 +148,19 @@ def test_push_many_iterations_alternate_subbuffers(heaps, algo):
         h.set_launch(algo, 0, 0)
     assert_bits(got, O.allreduce(x))
     assert_bits(got2, O.allreduce(x[::-1].copy()))
+
+
+@pytest.mark.parametrize("algo", [symar.LL, symar.SENTINEL, symar.TWOSHOT_LL, symar.TWOSHOT_SENTINEL])
+@pytest.mark.parametrize("limit", [16, 4096, 100000])
+def test_small_scratch_buffers_take_more_iterations(heaps, algo, limit):
+    h = heaps[8]
+    x = synth.make_inputs("normal", "bf16", 8, 90001, seed=limit)
+    h.set_scratch_limit(limit)
+    try:
+        got = run(h, x, symar.BF16, algo)
+    finally:
+        h.set_scratch_limit(0)
+    assert_bits(got, O.allreduce(x), f"algo {algo} scratch {limit}")
 
 
 def test_sentinel_mode_accepts_payload_equal_to_the_sentinel(heaps):
