@@ -450,7 +450,7 @@ def main():
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--quick", action="store_true", help="fewer latency samples")
     ap.add_argument("--latency-only", action="store_true", help="skip the bandwidth workload (no `value`)")
-    ap.add_argument("--no-autotune", action="store_true", help="latency section with the built-in launch shapes")
+    ap.add_argument("--no-autotune", action="store_true", help="built-in launch shapes: no tuning of the bandwidth workload's size nor of the latency section")
     ap.add_argument("--ctas", type=int, default=0)
     ap.add_argument("--threads", type=int, default=0)
     ap.add_argument("--variant", type=lambda v: int(v, 0), default=0, help="two-shot kernel variant bits")
@@ -501,12 +501,21 @@ def main():
     x = synth.make_inputs(w["dist"], w["dtype"], P, count, w["seed"] + rank)
     in_off, out_off = 0, (M + 4095) // 4096 * 4096
     heap = symar.SymHeap.on_torch(P, out_off + M, device=f"cuda:{local}")
+    tune_s = None
+    if args.ctas or args.threads or args.variant:
+        if args.ctas or args.threads:
+            heap.set_launch(symar.TWOSHOT, args.ctas, args.threads)
+        if args.variant:
+            heap.set_variant(symar.TWOSHOT, args.variant)
+    elif not args.no_autotune:
+        # the launch shape for exactly this message size, measured on this GPU (untimed set-up,
+        # as a deployment would do once); overwrites the user region, so inputs go in after it
+        t0 = time.time()
+        heap.autotune_size(symar.F32, count)
+        torch.cuda.synchronize()
+        tune_s = time.time() - t0
     for q in range(P):
         heap.write_rank(q, in_off, x[q])
-    if args.ctas or args.threads:
-        heap.set_launch(symar.TWOSHOT, args.ctas, args.threads)
-    if args.variant:
-        heap.set_variant(symar.TWOSHOT, args.variant)
     stream = torch.cuda.Stream()
     sh = stream.cuda_stream
     step = lambda: heap.allreduce(in_off, out_off, count, symar.F32, symar.TWOSHOT, sh)
@@ -569,7 +578,7 @@ def main():
                         "two-shot reduce-scatter + all-gather; value = 2*P*M bytes / time",
             "P": P, "elements_per_rank": count, "algo": "twoshot", "ctas_per_rank": ctas, "threads": threads,
             "kernel": kernel, "bulk_tile_KiB": tile_kib, "bulk_stages": ((variant >> 8) & 7) or None,
-            "dynamic_smem_bytes": smem,
+            "dynamic_smem_bytes": smem, "shape_tuned_for_this_size_seconds": tune_s,
             "l2": f"inputs {P * M >> 20} MiB + outputs {P * M >> 20} MiB per step, far larger than the 126 MB L2; "
                   "no flush needed",
             "multi_gpu": "replicas only (independent heaps, no exchange between GPUs)",
@@ -588,8 +597,8 @@ def main():
             "traffic": None,
         },
     }
-    traffic_note = ROOT / "profiles" / "twoshot_bulk_f32_p8_traffic.txt"
-    if traffic_note.exists() and smem and count == synth.WORKLOADS["c4"]["count"]:
+    traffic_note = ROOT / "profiles" / ("twoshot_bulk_f32_p8_traffic.txt" if smem else "twoshot_f32_p8_traffic.txt")
+    if traffic_note.exists() and count == synth.WORKLOADS["c4"]["count"]:
         kv = dict(l.split("=", 1) for l in traffic_note.read_text().splitlines() if "=" in l and not l.startswith("#"))
         line["roofline"]["traffic"] = int(kv["dram_bytes_per_launch_at_full_size "].strip())
         line["roofline"]["traffic_source"] = kv["source "].strip()

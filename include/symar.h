@@ -193,6 +193,13 @@ int symar_reduce(symheap_t *heap, const void *in, void *out, size_t count,
  * every rank.  Before it is called, built-in default thresholds apply.         */
 int allreduce_autotune(symheap_t *heap, symar_dtype_t dtype);
 
+/* The same for ONE message size: times every algorithm, shape and variant on messages
+ * of exactly `count` elements per rank (2 * count elements must fit in the user region)
+ * and records the winners for that size's bucket only, next to whatever the table
+ * already holds.  A second or two even for hundreds of MiB; for deployments that know
+ * their message sizes, and for sizes beyond the 64 MiB grid.  OVERWRITES the user region. */
+int allreduce_autotune_size(symheap_t *heap, symar_dtype_t dtype, size_t count);
+
 /* What the last allreduce() on this heap launched (for reporting). */
 int symar_last_choice(const symheap_t *heap, symar_algo_t *algo,
                       int *ctas_per_rank, int *threads);

@@ -35,6 +35,7 @@ struct Tuned {
     LaunchCfg cfg[kAlgos][kBuckets];
     double    us[kAlgos][kBuckets];
     int       lo_bucket = 0, hi_bucket = -1;
+    bool      have[kBuckets] = {};     // buckets tuned one at a time (allreduce_autotune_size)
 };
 
 static thread_local std::string g_last_cuda_error;
@@ -185,12 +186,18 @@ static int make_plan(symheap *h, size_t in_off, size_t out_off, size_t count, in
     const size_t bytes = count * es;
     const uint64_t nvec = (bytes + 15) / 16;
     const Tuned &tn    = h->tuned[dtype];
-    const int b        = tn.valid ? std::min(std::max(bucket_of(bytes), tn.lo_bucket), tn.hi_bucket) : 0;
+    // the size's own bucket if it was tuned, else the nearest bucket of a full table
+    int b = bucket_of(bytes);
+    bool tuned = tn.have[b];
+    if (!tuned && tn.valid) {
+        b     = std::min(std::max(b, tn.lo_bucket), tn.hi_bucket);
+        tuned = true;
+    }
 
-    if (algo == SYMAR_AUTO) algo = h->env_algo ? h->env_algo : (tn.valid ? tn.best_algo[b] : default_algo(bytes));
+    if (algo == SYMAR_AUTO) algo = h->env_algo ? h->env_algo : (tuned ? tn.best_algo[b] : default_algo(bytes));
 
     LaunchCfg cfg = default_cfg(h, algo, nvec);
-    if (tn.valid && tn.cfg[algo][b].ctas > 0) cfg = tn.cfg[algo][b];
+    if (tuned && tn.cfg[algo][b].ctas > 0) cfg = tn.cfg[algo][b];
     if (h->forced[algo].ctas > 0) cfg.ctas = h->forced[algo].ctas;
     if (h->forced[algo].threads > 0) cfg.threads = h->forced[algo].threads;
     if (h->variant_forced[algo]) cfg.variant = (int)h->variant[algo];
@@ -407,20 +414,17 @@ static int time_calls(symheap *h, cudaStream_t s, size_t count, int dtype, int a
     return SYMAR_OK;
 }
 
-static int autotune(symheap *h, int dtype)
+// Times every algorithm, launch shape and kernel variant on messages of `bytes` per rank
+// and records the winners in bucket b of `tn`.
+static int tune_bucket(symheap *h, int dtype, int b, size_t bytes, cudaStream_t s, Tuned &tn)
 {
     static const int kThreads[] = {64, 128, 256, 512};
     static const int kCtas[]    = {1, 2, 4, 8, 10, 12, 15, 16, 18, 24, 32, 37, 48, 64, 74};
-    const size_t es = elem_size(dtype);
-    Tuned tn;
-    size_t max_bytes = std::min<size_t>(h->bytes_per_rank / 2 / kAlign * kAlign, (size_t)64 << 20);
-    if (max_bytes < 16) return SYMAR_ERR_INVAL;
-    tn.lo_bucket = 4;
-    tn.hi_bucket = 4;
-    while (tn.hi_bucket + 1 < kBuckets && ((size_t)1 << (tn.hi_bucket + 1)) <= max_bytes) ++tn.hi_bucket;
-
-    cudaStream_t s;
-    CU(cudaStreamCreateWithFlags(&s, cudaStreamNonBlocking));
+    const size_t es     = elem_size(dtype);
+    const size_t count  = bytes / es;
+    const uint64_t nvec = (bytes + 15) / 16;
+    const int K    = bytes <= (1u << 20) ? 24 : (bytes <= (16u << 20) ? 6 : 2);
+    const int reps = 7;
     LaunchCfg saved[kAlgos];
     unsigned saved_variant[kAlgos];
     bool saved_forced[kAlgos];
@@ -429,71 +433,61 @@ static int autotune(symheap *h, int dtype)
         saved_variant[a] = h->variant[a];
         saved_forced[a]  = h->variant_forced[a];
     }
-    const Tuned saved_tuned = h->tuned[dtype];
-    h->tuned[dtype].valid = false;
-
     int rc = SYMAR_OK;
-    for (int b = tn.lo_bucket; b <= tn.hi_bucket && rc == SYMAR_OK; ++b) {
-        const size_t bytes  = (size_t)1 << b;
-        const size_t count  = bytes / es;
-        const uint64_t nvec = bytes / 16;
-        const int K    = bytes <= (1u << 20) ? 24 : (bytes <= (16u << 20) ? 6 : 2);
-        const int reps = 7;
-        double best_us = 1e30;
-        tn.best_algo[b] = SYMAR_ONESHOT;
-        for (int algo = SYMAR_ONESHOT; algo <= kLastAlgo && rc == SYMAR_OK; ++algo) {
-            tn.us[algo][b]  = 1e30;
-            tn.cfg[algo][b] = LaunchCfg{};
-            if (is_push(algo) && bytes > (4u << 20)) continue;   // scratch traffic through L2: hopeless there
-            if (algo == SYMAR_ONESHOT && bytes > (32u << 20)) continue;
-            const uint64_t work = (algo == SYMAR_TWOSHOT || is_twoshot_push(algo)) ? (nvec + h->P - 1) / h->P : nvec;
-            // kernel variants worth timing: the default; for two-shot in the bandwidth
-            // regime the bulk kernel's tile sizes and depths, and the register kernel
-            std::vector<int> variants = {0};
-            const bool bulk = algo == SYMAR_TWOSHOT && nvec >= kBulkMinVec;
-            if (bulk)
-                variants = {bulk_variant(2, 1), bulk_variant(3, 1), bulk_variant(2, 2), bulk_variant(3, 0),
-                            bulk_variant(4, 0), 4};
-            else if (algo == SYMAR_ONESHOT && bytes <= (1u << 20))
-                variants = {0, 0x100, 0x200};            // 16, 8 or 4 bytes per thread
-            else if (algo == SYMAR_LL && bytes <= (256u << 10))
-                variants = {0, 0x100};                   // 16 or 8 bytes of payload per thread
-            for (int var : variants) {
-                // threads a shape needs: one per unit of this variant
-                const uint64_t units = bulk ? work : work << ((var >> 8) & 3);
-                for (int T : kThreads) {
-                    if (bulk && var != 4 && T != 128 && T != 256) continue;
-                    for (int C : kCtas) {
-                        // skip shapes with far more threads than vectors, except the smallest
-                        if ((uint64_t)C * T > 2 * units && !(C == 1 && T == 64)) continue;
-                        // and shapes that would leave each thread hundreds of units
-                        if (!bulk && units / ((uint64_t)C * T) > 4096) continue;
-                        if (bulk && (C * h->P < 48)) continue;
-                        h->forced[algo]         = LaunchCfg{C, T, var};
-                        h->variant[algo]        = (unsigned)var;
-                        h->variant_forced[algo] = true;
-                        Plan p;
-                        if (make_plan(h, 0, round_up(bytes, kAlign), count, dtype, algo, &p) != SYMAR_OK) continue;
-                        if (p.cfg.ctas != C || p.cfg.threads != T) continue;   // clamped: a duplicate of another shape
-                        double us = 0;
-                        rc = time_calls(h, s, count, dtype, algo, K, reps, &us);
-                        if (rc != SYMAR_OK) break;
-                        if (us < tn.us[algo][b]) {
-                            tn.us[algo][b]  = us;
-                            tn.cfg[algo][b] = LaunchCfg{C, T, var};
-                        }
-                    }
+    double best_us = 1e30;
+    tn.best_algo[b] = SYMAR_ONESHOT;
+    for (int algo = SYMAR_ONESHOT; algo <= kLastAlgo && rc == SYMAR_OK; ++algo) {
+        tn.us[algo][b]  = 1e30;
+        tn.cfg[algo][b] = LaunchCfg{};
+        if (is_push(algo) && bytes > (4u << 20)) continue;   // scratch traffic through L2: hopeless there
+        if (algo != SYMAR_TWOSHOT && bytes > (32u << 20)) continue;   // only two-shot moves the minimum of bytes
+        const uint64_t work = (algo == SYMAR_TWOSHOT || is_twoshot_push(algo)) ? (nvec + h->P - 1) / h->P : nvec;
+        // kernel variants worth timing: the default; for two-shot in the bandwidth
+        // regime the bulk kernel's tile sizes and depths, and the register kernel
+        std::vector<int> variants = {0};
+        const bool bulk = algo == SYMAR_TWOSHOT && nvec >= kBulkMinVec;
+        if (bulk)
+            variants = {bulk_variant(2, 1), bulk_variant(3, 1), bulk_variant(2, 2), bulk_variant(3, 0),
+                        bulk_variant(4, 0), 4};
+        else if (algo == SYMAR_ONESHOT && bytes <= (1u << 20))
+            variants = {0, 0x100, 0x200};            // 16, 8 or 4 bytes per thread
+        else if (algo == SYMAR_LL && bytes <= (256u << 10))
+            variants = {0, 0x100};                   // 16 or 8 bytes of payload per thread
+        for (int var : variants) {
+            // threads a shape needs: one per unit of this variant
+            const uint64_t units = bulk ? work : work << ((var >> 8) & 3);
+            for (int T : kThreads) {
+                if (bulk && var != 4 && T != 128 && T != 256) continue;
+                for (int C : kCtas) {
+                    // skip shapes with far more threads than vectors, except the smallest
+                    if ((uint64_t)C * T > 2 * units && !(C == 1 && T == 64)) continue;
+                    // and shapes that would leave each thread hundreds of units
+                    if (!bulk && units / ((uint64_t)C * T) > 4096) continue;
+                    if (bulk && (C * h->P < 48)) continue;
+                    h->forced[algo]         = LaunchCfg{C, T, var};
+                    h->variant[algo]        = (unsigned)var;
+                    h->variant_forced[algo] = true;
+                    Plan p;
+                    if (make_plan(h, 0, round_up(bytes, kAlign), count, dtype, algo, &p) != SYMAR_OK) continue;
+                    if (p.cfg.ctas != C || p.cfg.threads != T) continue;   // clamped: a duplicate of another shape
+                    double us = 0;
+                    rc = time_calls(h, s, count, dtype, algo, K, reps, &us);
                     if (rc != SYMAR_OK) break;
+                    if (us < tn.us[algo][b]) {
+                        tn.us[algo][b]  = us;
+                        tn.cfg[algo][b] = LaunchCfg{C, T, var};
+                    }
                 }
                 if (rc != SYMAR_OK) break;
             }
-            h->forced[algo]         = saved[algo];
-            h->variant[algo]        = saved_variant[algo];
-            h->variant_forced[algo] = saved_forced[algo];
-            if (tn.us[algo][b] < best_us) {
-                best_us         = tn.us[algo][b];
-                tn.best_algo[b] = algo;
-            }
+            if (rc != SYMAR_OK) break;
+        }
+        h->forced[algo]         = saved[algo];
+        h->variant[algo]        = saved_variant[algo];
+        h->variant_forced[algo] = saved_forced[algo];
+        if (tn.us[algo][b] < best_us) {
+            best_us         = tn.us[algo][b];
+            tn.best_algo[b] = algo;
         }
     }
     for (int a = 0; a < kAlgos; ++a) {
@@ -501,13 +495,63 @@ static int autotune(symheap *h, int dtype)
         h->variant[a]        = saved_variant[a];
         h->variant_forced[a] = saved_forced[a];
     }
+    return rc;
+}
+
+// only_bytes == 0: the whole power-of-two grid; else just the bucket of that size, at that size
+static int autotune(symheap *h, int dtype, size_t only_bytes)
+{
+    const size_t es = elem_size(dtype);
+    const size_t fit = h->bytes_per_rank / 2 / kAlign * kAlign;      // input and output side by side
+    if (fit < 16) return SYMAR_ERR_INVAL;
+    cudaStream_t s;
+    CU(cudaStreamCreateWithFlags(&s, cudaStreamNonBlocking));
+    const Tuned saved_tuned = h->tuned[dtype];
+    int rc = SYMAR_OK;
+    if (only_bytes) {
+        const size_t bytes = only_bytes / es * es;
+        if (bytes < es || bytes > fit) {
+            cudaStreamDestroy(s);
+            return SYMAR_ERR_INVAL;
+        }
+        Tuned tn      = saved_tuned;
+        const int b   = bucket_of(bytes);
+        tn.have[b]    = false;
+        h->tuned[dtype].valid = false;                 // time with defaults, not with a stale table
+        std::memset(h->tuned[dtype].have, 0, sizeof h->tuned[dtype].have);
+        rc = tune_bucket(h, dtype, b, bytes, s, tn);
+        tn.have[b] = rc == SYMAR_OK;
+        cudaStreamSynchronize(s);
+        cudaStreamDestroy(s);
+        h->tuned[dtype] = rc == SYMAR_OK ? tn : saved_tuned;
+        return rc;
+    }
+    Tuned tn;
+    const size_t max_bytes = std::min<size_t>(fit, (size_t)64 << 20);
+    tn.lo_bucket = 4;
+    tn.hi_bucket = 4;
+    while (tn.hi_bucket + 1 < kBuckets && ((size_t)1 << (tn.hi_bucket + 1)) <= max_bytes) ++tn.hi_bucket;
+    h->tuned[dtype].valid = false;
+    std::memset(h->tuned[dtype].have, 0, sizeof h->tuned[dtype].have);
+    for (int b = tn.lo_bucket; b <= tn.hi_bucket && rc == SYMAR_OK; ++b)
+        rc = tune_bucket(h, dtype, b, (size_t)1 << b, s, tn);
     cudaStreamSynchronize(s);
     cudaStreamDestroy(s);
     if (rc != SYMAR_OK) {
         h->tuned[dtype] = saved_tuned;
         return rc;
     }
-    tn.valid        = true;
+    tn.valid = true;
+    for (int b = 0; b < kBuckets; ++b) tn.have[b] = saved_tuned.have[b] && (b < tn.lo_bucket || b > tn.hi_bucket);
+    // keep individually tuned buckets outside the grid
+    for (int b = 0; b < kBuckets; ++b)
+        if (tn.have[b]) {
+            tn.best_algo[b] = saved_tuned.best_algo[b];
+            for (int a = 0; a < kAlgos; ++a) {
+                tn.cfg[a][b] = saved_tuned.cfg[a][b];
+                tn.us[a][b]  = saved_tuned.us[a][b];
+            }
+        }
     h->tuned[dtype] = tn;
     return SYMAR_OK;
 }
@@ -716,7 +760,14 @@ int symar_reduce(symheap_t *heap, const void *in, void *out, size_t count, symar
 int allreduce_autotune(symheap_t *heap, symar_dtype_t dtype)
 {
     if (!heap || (dtype != SYMAR_F32 && dtype != SYMAR_BF16)) return SYMAR_ERR_INVAL;
-    return autotune(heap, (int)dtype);
+    return autotune(heap, (int)dtype, 0);
+}
+
+int allreduce_autotune_size(symheap_t *heap, symar_dtype_t dtype, size_t count)
+{
+    if (!heap || (dtype != SYMAR_F32 && dtype != SYMAR_BF16) || count == 0) return SYMAR_ERR_INVAL;
+    if (count > heap->bytes_per_rank / elem_size((int)dtype)) return SYMAR_ERR_INVAL;
+    return autotune(heap, (int)dtype, count * elem_size((int)dtype));
 }
 
 int symar_last_choice(const symheap_t *heap, symar_algo_t *algo, int *ctas_per_rank, int *threads)
@@ -754,7 +805,9 @@ int symar_tuned_entry(const symheap_t *heap, symar_dtype_t dtype, int log2_bytes
 {
     if (!heap || (dtype != SYMAR_F32 && dtype != SYMAR_BF16)) return SYMAR_ERR_INVAL;
     const Tuned &tn = heap->tuned[(int)dtype];
-    if (!tn.valid || log2_bytes < tn.lo_bucket || log2_bytes > tn.hi_bucket) return SYMAR_ERR_INVAL;
+    if (log2_bytes < 0 || log2_bytes >= kBuckets) return SYMAR_ERR_INVAL;
+    if (!tn.have[log2_bytes] && (!tn.valid || log2_bytes < tn.lo_bucket || log2_bytes > tn.hi_bucket))
+        return SYMAR_ERR_INVAL;
     if (algo < SYMAR_ONESHOT || algo > kLastAlgo) return SYMAR_ERR_INVAL;
     if (ctas_per_rank) *ctas_per_rank = tn.cfg[algo][log2_bytes].ctas;
     if (threads) *threads = tn.cfg[algo][log2_bytes].threads;
@@ -772,9 +825,15 @@ int symar_table_save(const symheap_t *heap, const char *host_path)
     std::fprintf(f, "symar-table 1 P %d\n", heap->P);
     for (int dt = 0; dt < 2; ++dt) {
         const Tuned &tn = heap->tuned[dt];
-        if (!tn.valid) continue;
-        std::fprintf(f, "dtype %d buckets %d %d\n", dt, tn.lo_bucket, tn.hi_bucket);
-        for (int b = tn.lo_bucket; b <= tn.hi_bucket; ++b) {
+        bool any = tn.valid;
+        for (int b = 0; b < kBuckets; ++b) any = any || tn.have[b];
+        if (!any) continue;
+        // "buckets 0 -1": no grid, only buckets tuned one at a time ("have" lines)
+        std::fprintf(f, "dtype %d buckets %d %d\n", dt, tn.valid ? tn.lo_bucket : 0, tn.valid ? tn.hi_bucket : -1);
+        for (int b = 0; b < kBuckets; ++b) {
+            const bool in_grid = tn.valid && b >= tn.lo_bucket && b <= tn.hi_bucket;
+            if (!in_grid && !tn.have[b]) continue;
+            if (tn.have[b]) std::fprintf(f, "have %d\n", b);
             std::fprintf(f, "best %d %d\n", b, tn.best_algo[b]);
             for (int a = SYMAR_ONESHOT; a < kAlgos; ++a)
                 std::fprintf(f, "cfg %d %d %d %d %d %.6g\n", b, a, tn.cfg[a][b].ctas, tn.cfg[a][b].threads,
@@ -795,6 +854,7 @@ int symar_table_load(symheap_t *heap, const char *host_path)
         return SYMAR_ERR_INVAL;          // written for another rank count or format
     }
     Tuned loaded[2];
+    bool seen[2] = {false, false};
     int dt = -1;
     char word[16];
     bool ok = true;
@@ -803,17 +863,22 @@ int symar_table_load(symheap_t *heap, const char *host_path)
         if (w == "dtype") {
             int lo, hi;
             ok = std::fscanf(f, "%d buckets %d %d", &dt, &lo, &hi) == 3 && dt >= 0 && dt < 2 && lo >= 0 &&
-                 hi < kBuckets && lo <= hi;
+                 hi < kBuckets && (lo <= hi || (lo == 0 && hi == -1));
             if (ok) {
                 loaded[dt]           = Tuned{};
                 loaded[dt].lo_bucket = lo;
                 loaded[dt].hi_bucket = hi;
-                loaded[dt].valid     = true;
+                loaded[dt].valid     = lo <= hi;
+                seen[dt]             = true;
                 for (int b = 0; b < kBuckets; ++b) {
                     loaded[dt].best_algo[b] = SYMAR_ONESHOT;
                     for (int a = 0; a < kAlgos; ++a) loaded[dt].us[a][b] = 1e30;
                 }
             }
+        } else if (w == "have") {
+            int b;
+            ok = dt >= 0 && std::fscanf(f, "%d", &b) == 1 && b >= 0 && b < kBuckets;
+            if (ok) loaded[dt].have[b] = true;
         } else if (w == "best") {
             int b, a;
             ok = dt >= 0 && std::fscanf(f, "%d %d", &b, &a) == 2 && b >= 0 && b < kBuckets && a >= SYMAR_ONESHOT &&
@@ -836,7 +901,7 @@ int symar_table_load(symheap_t *heap, const char *host_path)
     std::fclose(f);
     if (!ok) return SYMAR_ERR_INVAL;
     for (int d = 0; d < 2; ++d)
-        if (loaded[d].valid) heap->tuned[d] = loaded[d];
+        if (seen[d]) heap->tuned[d] = loaded[d];
     return SYMAR_OK;
 }
 

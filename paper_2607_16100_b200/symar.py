@@ -46,6 +46,7 @@ SIGNATURES = [
     ("symar_broadcast", c_int, [c_void_p, c_void_p, c_void_p, c_size_t, c_int, c_int, c_void_p]),
     ("symar_reduce", c_int, [c_void_p, c_void_p, c_void_p, c_size_t, c_int, c_int, c_void_p]),
     ("allreduce_autotune", c_int, [c_void_p, c_int]),
+    ("allreduce_autotune_size", c_int, [c_void_p, c_int, c_size_t]),
     ("symar_last_choice", c_int, [c_void_p, POINTER(c_int), POINTER(c_int), POINTER(c_int)]),
     ("symar_last_kernel", c_int, [c_void_p, POINTER(c_uint), POINTER(c_size_t)]),
     ("symar_query_choice", c_int, [c_void_p, c_size_t, c_int, POINTER(c_int), POINTER(c_int), POINTER(c_int)]),
@@ -250,6 +251,9 @@ class SymHeap:
     # -- selector --
     def autotune(self, dtype: int) -> None:
         _ck(self._lib.allreduce_autotune(self._h, dtype), "allreduce_autotune")
+
+    def autotune_size(self, dtype: int, count: int) -> None:
+        _ck(self._lib.allreduce_autotune_size(self._h, dtype, count), "allreduce_autotune_size")
 
     def last_choice(self):
         a, c, t = c_int(), c_int(), c_int()

@@ -430,6 +430,42 @@ def test_auto_default_and_after_autotune():
         h.destroy()
 
 
+def test_autotune_of_one_size_fills_only_its_bucket(tmp_path):
+    h = symar.SymHeap.on_torch(4, 1 << 20)
+    g = symar.SymHeap.on_torch(4, 1 << 20)
+    try:
+        count = 3 * 4096 + 5                                     # 49172 B of f32: bucket 16 (the next power of two)
+        before = h.query_choice(1024, symar.F32)
+        h.autotune_size(symar.F32, count)
+        assert h.tuned_entry(symar.F32, 16, symar.ONESHOT) is not None
+        assert h.tuned_entry(symar.F32, 15, symar.ONESHOT) is None      # other buckets untouched
+        assert h.query_choice(1024, symar.F32) == before                # and still on the defaults
+        a, c, t = h.query_choice(count, symar.F32)
+        best = min(ALGOS, key=lambda algo: h.tuned_entry(symar.F32, 16, algo)[2])
+        assert a == best and (c, t) == h.tuned_entry(symar.F32, 16, a)[:2]
+        x = synth.make_inputs("normal", "f32", 4, count, seed=3)
+        assert_bits(run(h, x, symar.F32, symar.AUTO), O.allreduce(x))
+        assert h.last_choice() == (a, c, t)
+        # survives a file round trip without a grid table beside it
+        path = tmp_path / "one.txt"
+        h.table_save(path)
+        g.table_load(path)
+        assert g.query_choice(count, symar.F32) == (a, c, t)
+        assert g.tuned_entry(symar.F32, 15, symar.ONESHOT) is None
+        # a later full tuning keeps nothing stale inside its grid and stays bit-exact
+        h.autotune(symar.F32)
+        assert h.tuned_entry(symar.F32, 15, symar.ONESHOT) is not None
+        assert_bits(run(h, x, symar.F32, symar.AUTO, poison=False), O.allreduce(x))
+        with pytest.raises(symar.SymarError):
+            h.autotune_size(symar.F32, (1 << 20) // 4)          # input and output would not fit
+        with pytest.raises(symar.SymarError):
+            h.autotune_size(symar.F32, 0)
+    finally:
+        torch.cuda.synchronize()
+        h.destroy()
+        g.destroy()
+
+
 def test_tuned_table_round_trips_through_a_file(tmp_path):
     a = symar.SymHeap.on_torch(4, 1 << 18)
     b = symar.SymHeap.on_torch(4, 1 << 18)
