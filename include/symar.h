@@ -329,6 +329,12 @@ int symar_probe_pingpong(int iterations, double *host_ns_per_round_trip);
  * depends on where the two SMs and the flag's L2 slice sit on the chip.        */
 int symar_probe_pingpong_pair(int iterations, int partner_block, double *host_ns_per_round_trip,
                               int *host_smids);
+/* The general form: a launch of `grid_blocks` one-thread blocks (2..1024) in which only
+ * `first_block` (which sends first and takes the time) and `partner_block` play.  Measured
+ * on B200: the round trip differs by up to 2x with the SM the FIRST block lands on and
+ * hardly at all with the partner's, so a representative bound samples both.     */
+int symar_probe_pingpong_blocks(int iterations, int first_block, int partner_block, int grid_blocks,
+                                double *host_ns_per_round_trip, int *host_smids);
 
 #ifdef __cplusplus
 }

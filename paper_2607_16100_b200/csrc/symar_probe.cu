@@ -53,20 +53,21 @@ __global__ void fence_kernel(unsigned *scratch, int iters, unsigned long long *o
 
 constexpr unsigned kSpinLimit = 1u << 22;   // polls; far above any real round trip
 
-// flags[0] is written by block 0 and watched by block 1; flags[32] the reverse
+// flags[0] is written by the first block and watched by its partner; flags[32] the reverse
 // (separate 128-byte lines).  out[0] = ns, out[1] = 1 on timeout, out[2..3] = SM ids.
-__global__ void pingpong_kernel(unsigned *flags, int iters, unsigned long long *out, int partner)
+__global__ void pingpong_kernel(unsigned *flags, int iters, unsigned long long *out, int first, int partner)
 {
-    // blocks other than 0 and `partner` only fill the SMs in between
-    if (blockIdx.x != 0 && (int)blockIdx.x != partner) return;
+    // blocks other than `first` and `partner` only fill the SMs in between
+    if ((int)blockIdx.x != first && (int)blockIdx.x != partner) return;
+    const bool starts = (int)blockIdx.x == first;
     unsigned smid;
     asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
-    unsigned *mine   = flags + (blockIdx.x == 0 ? 0 : 32);
-    unsigned *theirs = flags + (blockIdx.x == 0 ? 32 : 0);
-    out[2 + (blockIdx.x == 0 ? 0 : 1)] = smid;
+    unsigned *mine   = flags + (starts ? 0 : 32);
+    unsigned *theirs = flags + (starts ? 32 : 0);
+    out[2 + (starts ? 0 : 1)] = smid;
     bool dead = false;
     unsigned long long t0 = 0;
-    if (blockIdx.x == 0) {
+    if (starts) {
         // one untimed exchange first, so that both blocks are known to be running
         for (int i = 1; i <= iters + 1 && !dead; ++i) {
             if (i == 2) t0 = timer_ns();
@@ -137,17 +138,19 @@ int symar_probe_fence(int iterations, double *host_ns_per_fence)
     return SYMAR_OK;
 }
 
-int symar_probe_pingpong_pair(int iterations, int partner_block, double *host_ns_per_round_trip,
-                              int *host_smids)
+int symar_probe_pingpong_blocks(int iterations, int first_block, int partner_block, int grid_blocks,
+                                double *host_ns_per_round_trip, int *host_smids)
 {
-    if (iterations < 1 || partner_block < 1 || partner_block > 1023 || !host_ns_per_round_trip)
+    if (iterations < 1 || grid_blocks < 2 || grid_blocks > 1024 || first_block < 0 || partner_block < 0 ||
+        first_block >= grid_blocks || partner_block >= grid_blocks || first_block == partner_block ||
+        !host_ns_per_round_trip)
         return SYMAR_ERR_INVAL;
     unsigned char *buf = nullptr;
     if (cudaMalloc(&buf, 1024) != cudaSuccess) return SYMAR_ERR_NOMEM;
     cudaMemset(buf, 0, 1024);
     unsigned long long h[4] = {0, 0, 0, 0};
-    pingpong_kernel<<<partner_block + 1, 1>>>((unsigned *)buf, iterations, (unsigned long long *)(buf + 512),
-                                              partner_block);
+    pingpong_kernel<<<grid_blocks, 1>>>((unsigned *)buf, iterations, (unsigned long long *)(buf + 512), first_block,
+                                        partner_block);
     int rc = sync_and_fetch((unsigned long long *)(buf + 512), h, 4);
     cudaFree(buf);
     if (rc != SYMAR_OK) return rc;
@@ -159,6 +162,14 @@ int symar_probe_pingpong_pair(int iterations, int partner_block, double *host_ns
     if (h[2] == h[3]) return SYMAR_ERR_UNSUPPORTED;   // both blocks landed on one SM: not an L2 round trip
     *host_ns_per_round_trip = (double)h[0] / iterations;
     return SYMAR_OK;
+}
+
+int symar_probe_pingpong_pair(int iterations, int partner_block, double *host_ns_per_round_trip,
+                              int *host_smids)
+{
+    if (partner_block < 1 || partner_block > 1023) return SYMAR_ERR_INVAL;
+    return symar_probe_pingpong_blocks(iterations, 0, partner_block, partner_block + 1, host_ns_per_round_trip,
+                                       host_smids);
 }
 
 int symar_probe_pingpong(int iterations, double *host_ns_per_round_trip)

@@ -67,6 +67,7 @@ SIGNATURES = [
     ("symar_probe_fence", c_int, [c_int, POINTER(c_double)]),
     ("symar_probe_pingpong", c_int, [c_int, POINTER(c_double)]),
     ("symar_probe_pingpong_pair", c_int, [c_int, c_int, POINTER(c_double), POINTER(c_int)]),
+    ("symar_probe_pingpong_blocks", c_int, [c_int, c_int, c_int, c_int, POINTER(c_double), POINTER(c_int)]),
 ]
 
 
@@ -334,6 +335,15 @@ def probe_pingpong(iterations: int = 20000) -> float:
     v = c_double()
     _ck(load().symar_probe_pingpong(iterations, byref(v)), "symar_probe_pingpong")
     return v.value
+
+
+def probe_pingpong_blocks(first_block: int, partner_block: int, grid_blocks: int, iterations: int = 20000):
+    """(ns per round trip, (smid_first, smid_partner)); only the two named blocks of the launch play."""
+    v = c_double()
+    sm = (c_int * 2)()
+    _ck(load().symar_probe_pingpong_blocks(iterations, first_block, partner_block, grid_blocks, byref(v), sm),
+        "symar_probe_pingpong_blocks")
+    return v.value, (sm[0], sm[1])
 
 
 def probe_pingpong_pair(partner_block: int, iterations: int = 20000):

@@ -119,3 +119,22 @@ def test_c5_decode_trace_160_calls_in_one_graph(P):
     finally:
         torch.cuda.synchronize()
         h.destroy()
+
+
+def test_speed_of_light_probes_return_plausible_values():
+    """The pieces of the latency bound (Sec. VI): every probe ends by itself and gives sub-10-us figures."""
+    fence = symar.probe_fence(2000)
+    assert 10.0 < fence < 10_000.0
+    rt, sm = symar.probe_pingpong_pair(1, 2000)
+    assert 50.0 < rt < 10_000.0 and sm[0] != sm[1]
+    nsm = torch.cuda.get_device_properties(0).multi_processor_count
+    rt2, sm2 = symar.probe_pingpong_blocks(nsm // 2, 3, nsm, 2000)
+    assert 50.0 < rt2 < 10_000.0 and sm2[0] != sm2[1]
+    with pytest.raises(symar.SymarError):
+        symar.probe_pingpong_blocks(5, 5, nsm, 100)              # a block cannot play against itself
+    with pytest.raises(symar.SymarError):
+        symar.probe_pingpong_blocks(0, nsm, nsm, 100)            # partner outside the launch
+    s = torch.cuda.Stream()
+    symar.probe_empty(4, 8, 128, s.cuda_stream)
+    symar.probe_empty_pdl(4, 8, 128, s.cuda_stream)
+    s.synchronize()
