@@ -53,9 +53,19 @@ typedef enum {
                             changed and restores the sentinel.                               */
     SYMAR_TWOSHOT_LL = 5,       /* Table I "Two-shot (LL)": reduce-scatter and all-gather both
                                    pushed through the LL scratch, synchronised by the data    */
-    SYMAR_TWOSHOT_SENTINEL = 6  /* Table I "Two-shot (Sentinel)": the same through the sentinel
+    SYMAR_TWOSHOT_SENTINEL = 6, /* Table I "Two-shot (Sentinel)": the same through the sentinel
                                    scratch.  (SYMAR_AUTO picks algorithms 3..6 only where the
                                    tuner measured them to be fastest.)                        */
+    SYMAR_TWOSHOT_ATOMIC = 7    /* Sec. IV "LL128 Atomic AllReduce" / Table I last row: every rank
+                                   ADDS its part of chunk t into rank t's scratch with 16-byte
+                                   vector atomics; a contribution counter rides in each 128-byte
+                                   line; the owner polls it, then stores the sums everywhere.
+                                   NOT bit-reproducible (the order of the binary32 atomic adds is
+                                   free): results stay within gamma_{P-1} * sum|x_q| of the exact
+                                   sum; subnormals are flushed by the atomics.  bf16 is
+                                   accumulated in binary32 and narrowed once.  One call reduces
+                                   at most 31 * 4096 * P * P elements (SYMAR_ERR_UNSUPPORTED
+                                   above).  Never chosen by SYMAR_AUTO or the tuner.           */
 } symar_algo_t;
 
 enum {
@@ -83,6 +93,7 @@ typedef struct {
     size_t   user_bytes;          /* user region as laid out (rounded up to SYMAR_ALIGN)        */
     size_t   ll_scratch_bytes;    /* per rank: 2 parities x slots x P senders x vecs x 32 B     */
     size_t   sentinel_scratch_bytes; /* per rank: 2 parities x slots x P senders x vecs x 16 B   */
+    size_t   atomic_scratch_bytes; /* per rank: 2 parities x 512 KiB x P of 128-byte lines     */
     size_t   flag_bytes;          /* per rank: ready + done flag arrays + epoch counters        */
     size_t   stride;              /* bytes from one rank segment to the next                    */
     size_t   total_bytes;         /* control block + P segments                                 */

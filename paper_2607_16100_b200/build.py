@@ -10,7 +10,8 @@ PKG = Path(__file__).resolve().parent
 ROOT = PKG.parent
 CSRC = PKG / "csrc"
 LIB = PKG / "libsymar.so"
-SOURCES = ["symar_kernels.cu", "symar_bulk.cu", "symar_host.cu", "symar_probe.cu", "symar_static.cu", "symar_coll.cu"]
+SOURCES = ["symar_kernels.cu", "symar_bulk.cu", "symar_host.cu", "symar_probe.cu", "symar_static.cu", "symar_coll.cu",
+           "symar_atomic.cu"]
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a",

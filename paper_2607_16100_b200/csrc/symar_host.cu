@@ -24,9 +24,14 @@ struct LaunchCfg {
 };
 
 constexpr int kBuckets = 40;   // bucket b holds messages of (2^(b-1), 2^b] bytes per rank
-constexpr int kAlgos   = 7;    // indexed by symar_algo_t
-constexpr int kLastAlgo = SYMAR_TWOSHOT_SENTINEL;
-static bool is_push(int algo) { return algo >= SYMAR_LL; }            // uses per-slot scratch and epochs
+constexpr int kAlgos   = 8;    // indexed by symar_algo_t
+constexpr int kLastAlgo = SYMAR_TWOSHOT_ATOMIC;
+constexpr int kLastTuned = SYMAR_TWOSHOT_SENTINEL;   // the tuner and AUTO stay with the bit-reproducible algorithms
+static bool is_push(int algo) { return algo >= SYMAR_LL && algo <= SYMAR_TWOSHOT_SENTINEL; }   // per-slot scratch and epochs
+static KernelFn any_kernel_for(int algo, int dtype, int P, bool dbg)
+{
+    return algo == SYMAR_TWOSHOT_ATOMIC ? atomic_kernel_for(dtype, P, dbg) : kernel_for(algo, dtype, P, dbg);
+}
 static bool is_twoshot_push(int algo) { return algo == SYMAR_TWOSHOT_LL || algo == SYMAR_TWOSHOT_SENTINEL; }
 
 struct Tuned {
@@ -208,8 +213,20 @@ static int make_plan(symheap *h, size_t in_off, size_t out_off, size_t count, in
                                 is_twoshot_push(algo) ? (int)kPushTwoshotMaxThreads : (int)kMaxThreads);
     KArgs &a = p->args;
     std::memset(&a, 0, sizeof a);
-    KernelFn fn = kernel_for(algo, dtype, h->P, dbg_on(h));
+    KernelFn fn = any_kernel_for(algo, dtype, h->P, dbg_on(h));
     p->smem     = 0;
+    if (algo == SYMAR_TWOSHOT_ATOMIC) {
+        // one 8-thread group per 128-byte line of 31 elements; a chunk must fit in one scratch half
+        const uint64_t ch = (count + h->P - 1) / h->P;
+        const uint64_t nl = (ch + kAtLinePayload - 1) / kAtLinePayload;
+        if (nl > at_lines_per_half(h->P)) return SYMAR_ERR_UNSUPPORTED;
+        if (h->forced[algo].threads <= 0 && !(tuned && tn.cfg[algo][b].ctas > 0))
+            cfg.threads = nl * 8 >= 256 ? 256 : round_threads(std::max<uint64_t>(nl * 8, 32));
+        cfg.threads = std::max(32, (cfg.threads + 31) / 32 * 32);
+        if (h->forced[algo].ctas <= 0 && !(tuned && tn.cfg[algo][b].ctas > 0))
+            cfg.ctas = (int)std::max<uint64_t>(
+                1, std::min<uint64_t>((nl * 8 + cfg.threads - 1) / cfg.threads, (uint64_t)std::max(1, h->num_sms / h->P)));
+    }
     // bandwidth regime of two-shot: the bulk-copy kernel (the test hooks live in
     // the register kernel only)
     if (algo == SYMAR_TWOSHOT && nvec >= kBulkMinVec && !dbg_on(h) && !(var & 4u)) {
@@ -223,7 +240,7 @@ static int make_plan(symheap *h, size_t in_off, size_t out_off, size_t count, in
         p->smem     = bulk_smem_bytes(h->P, a.tile_vecs, a.stages);
     }
     if (!fn) return SYMAR_ERR_INVAL;
-    const int cap_slots = is_push(algo) ? kLLSlots : kMaxCtas;
+    const int cap_slots = (is_push(algo) || algo == SYMAR_TWOSHOT_ATOMIC) ? kLLSlots : kMaxCtas;
     const int cap_res   = std::max(1, max_resident(h, fn, cfg.threads, p->smem) / h->P);
     cfg.ctas = std::max(1, std::min({cfg.ctas, cap_slots, cap_res}));
 
@@ -235,6 +252,7 @@ static int make_plan(symheap *h, size_t in_off, size_t out_off, size_t count, in
     a.nvec       = nvec;
     a.ll_off     = h->L.ll_off;
     a.sn_off     = h->L.sn_off;
+    a.at_off     = h->L.at_off;
     a.ready_off  = h->L.ready_off;
     a.done_off   = h->L.done_off;
     a.epoch_off  = h->L.epoch_off;
@@ -436,7 +454,7 @@ static int tune_bucket(symheap *h, int dtype, int b, size_t bytes, cudaStream_t 
     int rc = SYMAR_OK;
     double best_us = 1e30;
     tn.best_algo[b] = SYMAR_ONESHOT;
-    for (int algo = SYMAR_ONESHOT; algo <= kLastAlgo && rc == SYMAR_OK; ++algo) {
+    for (int algo = SYMAR_ONESHOT; algo <= kLastTuned && rc == SYMAR_OK; ++algo) {
         tn.us[algo][b]  = 1e30;
         tn.cfg[algo][b] = LaunchCfg{};
         if (is_push(algo) && bytes > (4u << 20)) continue;   // scratch traffic through L2: hopeless there
@@ -583,7 +601,7 @@ static int create_common(symheap_t **heap, int P, size_t bytes_per_rank, void *m
     for (int algo = SYMAR_ONESHOT; algo <= kLastAlgo && e == cudaSuccess; ++algo)
         for (int dt = SYMAR_F32; dt <= SYMAR_BF16 && e == cudaSuccess; ++dt) {
             cudaFuncAttributes attr;
-            e = cudaFuncGetAttributes(&attr, kernel_for(algo, dt, P, false));
+            e = cudaFuncGetAttributes(&attr, any_kernel_for(algo, dt, P, false));
             if (e == cudaSuccess && algo == SYMAR_TWOSHOT) {
                 KernelFn bk = bulk_kernel_for(dt, P);
                 e = cudaFuncGetAttributes(&attr, bk);
@@ -607,7 +625,8 @@ static int create_common(symheap_t **heap, int P, size_t bytes_per_rank, void *m
     if (const char *v = std::getenv("SYMAR_ALGO")) {
         const std::string a(v);
         h->env_algo = a == "oneshot" ? SYMAR_ONESHOT : a == "twoshot" ? SYMAR_TWOSHOT : a == "ll" ? SYMAR_LL : a == "sentinel" ? SYMAR_SENTINEL
-                      : a == "twoshot_ll" ? SYMAR_TWOSHOT_LL : a == "twoshot_sentinel" ? SYMAR_TWOSHOT_SENTINEL : 0;
+                      : a == "twoshot_ll" ? SYMAR_TWOSHOT_LL : a == "twoshot_sentinel" ? SYMAR_TWOSHOT_SENTINEL
+                      : a == "twoshot_atomic" ? SYMAR_TWOSHOT_ATOMIC : 0;
     }
     if (const char *v = std::getenv("SYMAR_PDL")) h->pdl = std::atoi(v) != 0;
     *heap = h;
@@ -668,6 +687,7 @@ int symheap_info(const symheap_t *heap, symheap_info_t *info)
     info->user_bytes       = heap->L.user_bytes;
     info->ll_scratch_bytes = heap->L.ll_bytes;
     info->sentinel_scratch_bytes = heap->L.sn_bytes;
+    info->atomic_scratch_bytes = heap->L.at_bytes;
     info->flag_bytes       = heap->L.seg_bytes - heap->L.ready_off;
     info->stride           = heap->L.stride;
     info->total_bytes      = heap->L.total;

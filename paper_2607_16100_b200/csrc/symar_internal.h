@@ -16,6 +16,9 @@ KernelFn kernel_for(int algo, int dtype, int P, bool dbg);
 // shared memory); needs bulk_smem_bytes() of dynamic shared memory.
 KernelFn bulk_kernel_for(int dtype, int P);
 
+// Two-shot with atomic accumulation in the owner's scratch (symar_atomic.cu).
+KernelFn atomic_kernel_for(int dtype, int P, bool dbg);
+
 // grid = (ctas_per_rank, P), block = threads; returns the launch status.
 cudaError_t launch_kernel(KernelFn fn, int P, int ctas_per_rank, int threads, size_t smem_bytes,
                           const KArgs &args, cudaStream_t stream);

@@ -2,7 +2,7 @@
 // of libsymar (never by the CPU oracle).
 //
 // heap memory:  [ control block | segment 0 | segment 1 | ... | segment P-1 ]
-// segment q  :  [ user region | LL scratch | sentinel scratch | ready flags | done flags | counters | pad ]
+// segment q  :  [ user region | LL scratch | sentinel scratch | atomic scratch | ready flags | done flags | counters | pad ]
 //
 // Every rank segment has the same layout (symmetric objects: same offset + rank
 // id addresses a peer's copy), every region starts on a 4 KiB boundary.
@@ -43,6 +43,7 @@ __host__ __device__ constexpr size_t done_count_off(int c) { return (size_t)kMax
 //   two-shot : bit 0 = contiguous chunks for large messages, bit 1 = 16-byte accesses,
 //              bit 2 = never the bulk-copy kernel, bits 8-10 = bulk pipeline depth,
 //              bits 12-13 = log2(bulk tile size / 4 KiB)
+//   atomic two-shot: bit 0 = skip the confirming re-read of a completed line
 //   sibling collectives: the unit size in bytes (16, 4 or 2)
 
 constexpr uint32_t kOneChunk     = 0xffu;   // KArgs::blk_log2: rank r owns one contiguous chunk
@@ -70,6 +71,8 @@ struct Layout {
     size_t   ll_bytes;
     size_t   sn_off;         // sentinel scratch: [parity][slot][sender][vector] x 16 B, pre-filled with 0xFF
     size_t   sn_bytes;
+    size_t   at_off;         // atomic two-shot: [parity][line] x 128 B of binary32 accumulators, zero when idle
+    size_t   at_bytes;
     size_t   ready_off;      // kMaxCtas groups of kFlagGroup bytes
     size_t   done_off;
     size_t   epoch_off;      // kMaxCtas x u64 LL iteration counters, then kMaxCtas x u32
@@ -86,6 +89,14 @@ constexpr size_t kLLSenderBytes = (size_t)kLLSlotVecs * 32;
 constexpr size_t   kSnSenderBytes = (size_t)kLLSlotVecs * 16;
 constexpr uint32_t kSentinelWord  = 0xffffffffu;      // a negative NaN in fp32, two of them in bf16
 
+// atomic two-shot (Sec. IV "LL128 Atomic AllReduce"): a 128-byte line holds one
+// contribution counter and 31 binary32 accumulators; a rank's chunk of one call
+// must fit in one parity half of its scratch
+constexpr size_t   kAtLineBytes        = 128;
+constexpr uint32_t kAtLinePayload      = 31;
+constexpr size_t   kAtHalfBytesPerRank = (size_t)512 << 10;     // x P ranks = one parity half
+__host__ __device__ constexpr uint64_t at_lines_per_half(int P) { return kAtHalfBytesPerRank * (uint64_t)P / kAtLineBytes; }
+
 inline Layout make_layout(int P, size_t bytes_per_rank)
 {
     Layout L{};
@@ -95,7 +106,9 @@ inline Layout make_layout(int P, size_t bytes_per_rank)
     L.ll_bytes   = (size_t)2 * kLLSlots * P * kLLSenderBytes;
     L.sn_off     = L.ll_off + L.ll_bytes;
     L.sn_bytes   = (size_t)2 * kLLSlots * P * kSnSenderBytes;
-    L.ready_off  = L.sn_off + L.sn_bytes;
+    L.at_off     = L.sn_off + L.sn_bytes;
+    L.at_bytes   = (size_t)2 * kAtHalfBytesPerRank * P;
+    L.ready_off  = L.at_off + L.at_bytes;
     L.done_off   = L.ready_off + (size_t)kMaxCtas * kFlagGroup;
     L.epoch_off  = L.done_off + (size_t)kMaxCtas * kFlagGroup;
     L.seg_bytes  = round_up(L.epoch_off + (size_t)kMaxCtas * (sizeof(uint64_t) + 2 * sizeof(uint32_t)), kAlign);
@@ -116,6 +129,7 @@ struct KArgs {
     uint64_t  nvec;          // 16-byte vectors per rank, ceil(count * elem / 16)
     uint64_t  ll_off;
     uint64_t  sn_off;
+    uint64_t  at_off;
     uint64_t  ready_off;
     uint64_t  done_off;
     uint64_t  epoch_off;

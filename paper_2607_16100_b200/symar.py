@@ -14,9 +14,9 @@ _PKG = Path(__file__).resolve().parent
 LIB_PATH = _PKG / "libsymar.so"
 
 F32, BF16 = 0, 1
-AUTO, ONESHOT, TWOSHOT, LL, SENTINEL, TWOSHOT_LL, TWOSHOT_SENTINEL = 0, 1, 2, 3, 4, 5, 6
+AUTO, ONESHOT, TWOSHOT, LL, SENTINEL, TWOSHOT_LL, TWOSHOT_SENTINEL, TWOSHOT_ATOMIC = 0, 1, 2, 3, 4, 5, 6, 7
 ALGO_NAMES = {AUTO: "auto", ONESHOT: "oneshot", TWOSHOT: "twoshot", LL: "ll", SENTINEL: "sentinel",
-              TWOSHOT_LL: "twoshot_ll", TWOSHOT_SENTINEL: "twoshot_sentinel"}
+              TWOSHOT_LL: "twoshot_ll", TWOSHOT_SENTINEL: "twoshot_sentinel", TWOSHOT_ATOMIC: "twoshot_atomic"}
 DTYPE_NAMES = {F32: "f32", BF16: "bf16"}
 DTYPE_SIZE = {F32: 4, BF16: 2}
 
@@ -83,7 +83,8 @@ class SymarError(RuntimeError):
 class HeapInfo(ctypes.Structure):
     _fields_ = [
         ("P", c_int), ("bytes_per_rank", c_size_t), ("user_bytes", c_size_t),
-        ("ll_scratch_bytes", c_size_t), ("sentinel_scratch_bytes", c_size_t), ("flag_bytes", c_size_t),
+        ("ll_scratch_bytes", c_size_t), ("sentinel_scratch_bytes", c_size_t), ("atomic_scratch_bytes", c_size_t),
+        ("flag_bytes", c_size_t),
         ("stride", c_size_t),
         ("total_bytes", c_size_t), ("base", c_void_p),
     ]

@@ -67,9 +67,12 @@ def test_required_bytes_layout(lib, P):
     ll = 2 * (2 * P * D)
     # Table I, one-shot sentinel: N D per iteration (bare payload), again two parities
     sentinel = 2 * (P * D)
+    # Table I, two-shot LL128 atomic: about D / N per iteration; this build gives every
+    # rank two parity halves of 512 KiB x P of 128-byte accumulator lines
+    atomic = 2 * (512 << 10) * P
     flags = 2 * symar.MAX_CTAS * 32 + symar.MAX_CTAS * 8
-    assert total >= P * (user + ll + sentinel + flags)
-    assert total <= P * (user + ll + sentinel + flags + 16 * symar.ALIGN) + 4096
+    assert total >= P * (user + ll + sentinel + atomic + flags)
+    assert total <= P * (user + ll + sentinel + atomic + flags + 16 * symar.ALIGN) + 4096
     assert total % symar.ALIGN == 0
     # monotone in the user size, and rounding never loses bytes
     assert symar.required_bytes(P, user + 1) >= total
