@@ -251,11 +251,12 @@ int symar_set_launch(symheap_t *heap, symar_algo_t algo, int ctas_per_rank, int 
  * default), bits 12-13 = log2 of its tile size over 4 KiB.                        */
 int symar_set_variant(symheap_t *heap, symar_algo_t algo, unsigned int variant);
 
-/* Programmatic dependent launch (off by default).  When on, every allreduce() is
- * launched so that the NEXT kernel of the stream may become resident while it
- * still runs; each AllReduce kernel first waits until the previous grid of the
- * stream has completed and its writes are visible, so results and ordering are
- * unchanged -- only launch latency of back-to-back calls is hidden.            */
+/* Programmatic dependent launch (ON by default; SYMAR_PDL=0 in the environment or
+ * enabled = 0 here turns it off).  When on, every kernel of the library is launched
+ * so that it may become resident while the previous kernel of the stream still runs;
+ * its first instruction waits until that grid has completed and its writes are
+ * visible, so results and ordering are unchanged -- only the launch latency of
+ * back-to-back calls is hidden (measured: -0.25 us of 1.95 us per 16 KiB call).  */
 int symar_set_pdl(symheap_t *heap, int enabled);
 
 /* Pretend the push algorithms (LL, sentinel, and their two-shot forms) had a smaller

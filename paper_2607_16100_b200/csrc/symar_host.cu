@@ -72,7 +72,7 @@ struct symheap {
     int       num_sms = 0;
     int       max_smem = 48 * 1024;   // opt-in dynamic shared memory per CTA
     uint64_t  spin_ns = 2000000000ull;
-    bool      pdl          = false;
+    bool      pdl          = true;    // programmatic dependent launch of every kernel
     int       env_algo     = 0;       // SYMAR_ALGO override of SYMAR_AUTO, 0 = none
     size_t    scratch_limit = 0;      // push algorithms: payload bytes per rank and iteration, 0 = all there is
     int       dbg_mute     = -1;
@@ -491,7 +491,10 @@ static int tune_bucket(symheap *h, int dtype, int b, size_t bytes, cudaStream_t 
                     double us = 0;
                     rc = time_calls(h, s, count, dtype, algo, K, reps, &us);
                     if (rc != SYMAR_OK) break;
-                    if (us < tn.us[algo][b]) {
+                    // a larger launch must win by more than the timing noise (1.5 %) to displace a smaller one
+                    const LaunchCfg &cur = tn.cfg[algo][b];
+                    const bool larger    = cur.ctas > 0 && (long)C * T > (long)cur.ctas * cur.threads;
+                    if (us < tn.us[algo][b] * (larger ? 0.985 : 1.0)) {
                         tn.us[algo][b]  = us;
                         tn.cfg[algo][b] = LaunchCfg{C, T, var};
                     }

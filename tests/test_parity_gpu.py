@@ -372,7 +372,8 @@ def test_graph_capture_replays(heaps):
             assert_bits(got, want, f"replay {rep} call {k}")
 
 
-def test_programmatic_dependent_launch_keeps_results_and_order(heaps):
+@pytest.mark.parametrize("pdl", [True, False])
+def test_programmatic_dependent_launch_keeps_results_and_order(heaps, pdl):
     # back-to-back calls whose input is the previous call's output: with the
     # launch attribute on, each kernel may become resident early but must not
     # touch the heap before its predecessor has finished
@@ -382,7 +383,7 @@ def test_programmatic_dependent_launch_keeps_results_and_order(heaps):
     x = synth.make_inputs("normal", "bf16", 8, count, seed=606)
     for q in range(8):
         h.write_rank(q, 0, x[q])
-    h.set_pdl(True)
+    h.set_pdl(pdl)                              # on is the default; off must give the same
     try:
         s = torch.cuda.Stream()
         chain = [ALGOS[k % len(ALGOS)] for k in range(9)]
@@ -404,7 +405,7 @@ def test_programmatic_dependent_launch_keeps_results_and_order(heaps):
             got = run(h, x, symar.BF16, algo, in_off=0, out_off=1 << 20, poison=False)
             assert_bits(got, O.allreduce(x))
     finally:
-        h.set_pdl(False)
+        h.set_pdl(True)
 
 
 # ---- AUTO, autotune -----------------------------------------------------------------------
