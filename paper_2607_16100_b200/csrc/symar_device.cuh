@@ -154,6 +154,12 @@ __device__ __forceinline__ uint64_t globaltimer_ns()
 // has completed and its writes are visible.  Without the attribute both calls
 // do nothing.
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+// The same, with addresses that are to be ready BEFORE the wait: a kernel made
+// resident early computes them while its predecessor still runs.
+__device__ __forceinline__ void pdl_wait_holding(const void *p0, const void *p1, const void *p2)
+{
+    asm volatile("griddepcontrol.wait;" ::"l"(p0), "l"(p1), "l"(p2) : "memory");
+}
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;"); }
 
 // ---- bounded waiting ------------------------------------------------------------
@@ -380,21 +386,34 @@ __device__ __forceinline__ void debug_delay(const KArgs &a, int rank, int cta)
 // kernel started, and a kernel boundary makes it visible to every later reader
 // -- so it is a relaxed increment and costs no fence on the critical path.
 // `want` receives the count to publish.  Returns false if the wait ran out.
+// The addresses one exchange touches, computable before the kernel may touch memory.
+struct ExchangePtrs {
+    uint32_t       *signal;   // thread t < P: this rank's word in peer t's flag group
+    const uint32_t *mine;     // lane q: peer q's word in this rank's flag group
+};
+template <int P>
+__device__ __forceinline__ ExchangePtrs exchange_ptrs(const KArgs &a, uint64_t flags_off, int r, int c)
+{
+    const uint32_t t    = threadIdx.x;
+    const uint32_t lane = t & 31u;
+    ExchangePtrs p;
+    p.signal = reinterpret_cast<uint32_t *>(a.seg0 + (size_t)(t < P ? t : 0) * a.stride + flags_off +
+                                            (size_t)c * kFlagGroup) + r;
+    p.mine   = reinterpret_cast<const uint32_t *>(a.seg0 + (size_t)r * a.stride + flags_off + (size_t)c * kFlagGroup) +
+             (lane < P ? lane : 0);
+    return p;
+}
+
 template <int P, bool RELEASE>
-__device__ __forceinline__ bool flag_exchange(const KArgs &a, uint64_t flags_off, const uint32_t *count,
-                                              int r, int c, bool silent, bool all_warps, uint32_t &want)
+__device__ __forceinline__ bool flag_exchange_at(const KArgs &a, const ExchangePtrs &p, const uint32_t *count, int r,
+                                                 int c, bool silent, bool all_warps, uint32_t &want)
 {
     const uint32_t t    = threadIdx.x;
     const uint32_t lane = t & 31u;
     if (t < P && !silent) {
-        uint32_t *dst =
-            reinterpret_cast<uint32_t *>(a.seg0 + t * a.stride + flags_off + (size_t)c * kFlagGroup) + r;
-        if (RELEASE) red_release_inc_u32(dst);
-        else red_relaxed_inc_u32(dst);
+        if (RELEASE) red_release_inc_u32(p.signal);
+        else red_relaxed_inc_u32(p.signal);
     }
-    const uint32_t *mine =
-        reinterpret_cast<const uint32_t *>(a.seg0 + (size_t)r * a.stride + flags_off + (size_t)c * kFlagGroup) +
-        (lane < P ? lane : 0);
     const uint32_t n = ld_relaxed_u32(count);
     if (!all_warps && t >= 32) {
         want = n + 1;
@@ -402,7 +421,7 @@ __device__ __forceinline__ bool flag_exchange(const KArgs &a, uint64_t flags_off
     }
     Spin spin;
     for (;;) {
-        const uint32_t f = ld_acquire_u32(mine);
+        const uint32_t f = ld_acquire_u32(p.mine);
         want = n + 1;
         // ">= want": a peer may already have signalled its next call
         const unsigned late = __ballot_sync(0xffffffffu, lane < P && (int32_t)(f - want) < 0);
@@ -412,6 +431,13 @@ __device__ __forceinline__ bool flag_exchange(const KArgs &a, uint64_t flags_off
             return false;
         }
     }
+}
+
+template <int P, bool RELEASE>
+__device__ __forceinline__ bool flag_exchange(const KArgs &a, uint64_t flags_off, const uint32_t *count,
+                                              int r, int c, bool silent, bool all_warps, uint32_t &want)
+{
+    return flag_exchange_at<P, RELEASE>(a, exchange_ptrs<P>(a, flags_off, r, c), count, r, c, silent, all_warps, want);
 }
 
 // Reduce-scatter + all-gather of one 16-byte vector: P loads, the rank-ordered

@@ -49,12 +49,13 @@ __global__ void __launch_bounds__(kMaxThreads) oneshot_kernel(const KArgs a)
     const uint32_t t = threadIdx.x, T = blockDim.x;
     char *seg_r = a.seg0 + (size_t)r * a.stride;
     uint32_t *count = reinterpret_cast<uint32_t *>(seg_r + a.epoch_off + ready_count_off(c));
-    if (a.pdl) pdl_wait();                    // the previous call has left the heap
+    const ExchangePtrs xp = exchange_ptrs<P>(a, a.ready_off, r, c);
+    if (a.pdl) pdl_wait_holding(xp.signal, xp.mine, count);   // the previous call has left the heap
     if (DBG) debug_delay(a, r, c);
     if (DBG && a.dbg_mute == r) return;       // test hook: this rank never joins
 
     uint32_t want;
-    const bool ok = flag_exchange<P, false>(a, a.ready_off, count, r, c, false, true, want);
+    const bool ok = flag_exchange_at<P, false>(a, xp, count, r, c, false, true, want);
     // Every warp has consumed the count; publish the next one now so that its
     // store drains while the data is in flight.
     __syncthreads();
