@@ -348,6 +348,18 @@ int symar_probe_pingpong_pair(int iterations, int partner_block, double *host_ns
 int symar_probe_pingpong_blocks(int iterations, int first_block, int partner_block, int grid_blocks,
                                 double *host_ns_per_round_trip, int *host_smids);
 
+/* ---- host side of the thread-level buffer primitives (symar_llbuffer.cuh; Sec. V
+ *      "Host-side Functions": a scratch-size helper and the sentinel initialiser) ---- */
+
+/* Bytes ONE rank's copy of an LLBuffer needs: sync_mode 0 = LL (every element occupies twice
+ * its size), 1 = sentinel; elem_bytes 4 or 8; slots_per_cta elements per CTA and epoch; ctas
+ * CTAs per rank; round_robin sub-buffers (0 counts as 1).  0 for bad arguments.              */
+size_t symar_llbuffer_bytes(int sync_mode, size_t elem_bytes, size_t slots_per_cta, int ctas, int round_robin);
+
+/* Fills `bytes` bytes of device memory with the sentinel (all ones) on the given stream:
+ * what sentinel mode expects before the first send.  (LL mode expects zeros: cudaMemset.)   */
+int symar_llbuffer_init_sentinel(void *device_ptr, size_t bytes, void *cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

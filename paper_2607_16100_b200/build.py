@@ -1,4 +1,5 @@
-"""Build libsymar.so (the C-ABI CUDA library) in-tree with nvcc for sm_100a."""
+"""Build libsymar.so (the C-ABI CUDA library) and the example kernel written on the public
+device header, in-tree with nvcc for sm_100a."""
 from __future__ import annotations
 
 import os
@@ -13,6 +14,9 @@ LIB = PKG / "libsymar.so"
 SOURCES = ["symar_kernels.cu", "symar_bulk.cu", "symar_host.cu", "symar_probe.cu", "symar_static.cu", "symar_coll.cu",
            "symar_atomic.cu"]
 
+EXAMPLE_SRC = PKG / "examples" / "llbuffer_oneshot.cu"
+EXAMPLE_LIB = PKG / "libsymar_example.so"
+
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a",
     "-O3", "-std=c++17", "-lineinfo",
@@ -26,7 +30,7 @@ def _stale() -> bool:
     if not LIB.exists():
         return True
     t = LIB.stat().st_mtime
-    deps = list(CSRC.iterdir()) + [ROOT / "include" / "symar.h", Path(__file__)]
+    deps = list(CSRC.iterdir()) + [ROOT / "include" / "symar.h", Path(__file__)]   # (the example has its own check)
     return any(d.stat().st_mtime > t for d in deps)
 
 
@@ -46,5 +50,19 @@ def build_lib(force: bool = False, verbose: bool = False) -> Path:
     return LIB
 
 
+def build_example(force: bool = False) -> Path:
+    """The one-shot AllReduce of examples/llbuffer_oneshot.cu: uses include/symar_llbuffer.cuh only."""
+    deps = [EXAMPLE_SRC, ROOT / "include" / "symar_llbuffer.cuh", Path(__file__)]
+    if not force and EXAMPLE_LIB.exists() and all(d.stat().st_mtime <= EXAMPLE_LIB.stat().st_mtime for d in deps):
+        return EXAMPLE_LIB
+    nvcc = os.environ.get("NVCC", "nvcc")
+    tmp = EXAMPLE_LIB.with_suffix(f".so.tmp{os.getpid()}")
+    cmd = [nvcc, *NVCC_FLAGS, "--extended-lambda", "-I", str(ROOT / "include"), "-o", str(tmp), str(EXAMPLE_SRC)]
+    subprocess.run(cmd, check=True)
+    os.replace(tmp, EXAMPLE_LIB)
+    return EXAMPLE_LIB
+
+
 if __name__ == "__main__":
     print(build_lib(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    print(build_example(force="--force" in sys.argv))

@@ -977,4 +977,18 @@ int symar_debug_inject(symheap_t *heap, int mute_rank, unsigned int delay_seed, 
 
 const char *symar_last_cuda_error(void) { return g_last_cuda_error.c_str(); }
 
+size_t symar_llbuffer_bytes(int sync_mode, size_t elem_bytes, size_t slots_per_cta, int ctas, int round_robin)
+{
+    if ((sync_mode != 0 && sync_mode != 1) || (elem_bytes != 4 && elem_bytes != 8) || ctas < 1 || round_robin < 0)
+        return 0;
+    return (sync_mode == 0 ? 2 : 1) * elem_bytes * slots_per_cta * (size_t)ctas * (size_t)(round_robin ? round_robin : 1);
+}
+
+int symar_llbuffer_init_sentinel(void *device_ptr, size_t bytes, void *cuda_stream)
+{
+    if (!device_ptr) return SYMAR_ERR_INVAL;
+    CU(cudaMemsetAsync(device_ptr, 0xff, bytes, (cudaStream_t)cuda_stream));
+    return SYMAR_OK;
+}
+
 }  // extern "C"

@@ -1,0 +1,123 @@
+// A one-shot AllReduce(sum) written ONLY with the public thread-level primitives of
+// symar_llbuffer.cuh, after the example of the paper's Sec. V ("Example One-shot
+// AllReduce"): wrap symmetric scratch memory in an LLBuffer with double buffering; every
+// thread loads a 32-bit word of its rank's input, broadcasts it into its row of every
+// peer's region, receives and reduces the P rows in rank order, stores the result, and
+// advances the epoch.  Works for any message size (several epochs per launch).
+//
+// The P ranks are the rows of the grid (blockIdx.y), as everywhere in this library; all
+// P * ctas CTAs wait for one another and must be co-resident, so keep the grid small.
+// Not a tuned kernel: it shows that a collective is a dozen lines on top of the primitives,
+// and it is the test vehicle of the header (tests/test_llbuffer_gpu.py).
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+
+#include "symar_llbuffer.cuh"
+
+using namespace symar;
+
+namespace {
+
+struct F32Acc {
+    float v;
+    __device__ static F32Acc widen(uint32_t w) { return {__uint_as_float(w)}; }
+    __device__ static F32Acc add(F32Acc a, F32Acc b) { return {__fadd_rn(a.v, b.v)}; }
+    __device__ uint32_t narrow() const { return __float_as_uint(v); }
+};
+struct BF16x2Acc {                      // one word = two bf16 elements, accumulated in binary32
+    float lo, hi;
+    __device__ static BF16x2Acc widen(uint32_t w) { return {__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u)}; }
+    __device__ static BF16x2Acc add(BF16x2Acc a, BF16x2Acc b) { return {__fadd_rn(a.lo, b.lo), __fadd_rn(a.hi, b.hi)}; }
+    __device__ uint32_t narrow() const
+    {
+        __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
+        return *reinterpret_cast<uint32_t *>(&h);
+    }
+};
+
+template <LLSync Mode, int P, typename Acc>
+__global__ void oneshot_llbuffer_kernel(const char *in0, char *out0, size_t io_stride, char *scratch0,
+                                        size_t scratch_stride, size_t nwords, uint64_t epoch, int slots_per_cta,
+                                        unsigned *fail)
+{
+    const int cta = blockIdx.x, ctas = gridDim.x, rank = blockIdx.y;
+    // region of a CTA and epoch: P rows (one per sender) of slots_per_cta slots
+    LLBuffer<Mode> buf(scratch0, scratch_stride, rank, P, cta, ctas,
+                       (size_t)P * slots_per_cta * LLBuffer<Mode>::template slotBytes<uint32_t>(), 2, epoch, 1u << 20);
+    const uint32_t *in = reinterpret_cast<const uint32_t *>(in0 + (size_t)rank * io_stride);
+    uint32_t *out      = reinterpret_cast<uint32_t *>(out0 + (size_t)rank * io_stride);
+    const size_t per_epoch = (size_t)ctas * slots_per_cta;
+    for (size_t first = (size_t)cta * slots_per_cta; first < nwords + (size_t)cta * slots_per_cta; first += per_epoch) {
+        for (int k = threadIdx.x; k < slots_per_cta; k += blockDim.x) {
+            const size_t i = first + k;
+            if (i >= nwords) continue;
+            uint32_t w = in[i];
+            if (Mode == LLSync::Sentinel && w == 0xffffffffu) w = 0xfffffffeu;   // never send the sentinel (a NaN either way)
+            buf.template bcast<uint32_t, P>((size_t)rank * slots_per_cta + k, w);        // my row, every rank's region
+            Acc acc;
+            const bool ok = buf.template recvReduce<Acc, uint32_t, P, P, Mode == LLSync::Sentinel>(
+                (size_t)k, (size_t)slots_per_cta, P, [](uint32_t x) { return Acc::widen(x); },
+                [](Acc a, Acc b) { return Acc::add(a, b); }, acc);
+            if (!ok) {
+                atomicExch(fail, 1u);
+                return;
+            }
+            out[i] = acc.narrow();
+        }
+        // sentinel mode: the restored sentinels must be in place before this sub-buffer is used
+        // again two epochs from now (Sec. V "reset": visibility needs a fence)
+        if (Mode == LLSync::Sentinel) __threadfence();
+        buf.advanceEpoch();
+    }
+}
+
+template <LLSync Mode, typename Acc>
+cudaError_t launch(int P, dim3 grid, dim3 block, cudaStream_t s, const char *in0, char *out0, size_t io_stride,
+                   char *scratch0, size_t scratch_stride, size_t nwords, uint64_t epoch, int slots, unsigned *fail)
+{
+    switch (P) {
+        case 1: oneshot_llbuffer_kernel<Mode, 1, Acc><<<grid, block, 0, s>>>(in0, out0, io_stride, scratch0, scratch_stride, nwords, epoch, slots, fail); break;
+        case 2: oneshot_llbuffer_kernel<Mode, 2, Acc><<<grid, block, 0, s>>>(in0, out0, io_stride, scratch0, scratch_stride, nwords, epoch, slots, fail); break;
+        case 4: oneshot_llbuffer_kernel<Mode, 4, Acc><<<grid, block, 0, s>>>(in0, out0, io_stride, scratch0, scratch_stride, nwords, epoch, slots, fail); break;
+        case 8: oneshot_llbuffer_kernel<Mode, 8, Acc><<<grid, block, 0, s>>>(in0, out0, io_stride, scratch0, scratch_stride, nwords, epoch, slots, fail); break;
+        default: return cudaErrorInvalidValue;
+    }
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+extern "C" {
+
+// mode 0 = LL, 1 = sentinel; bf16 0 = fp32 words, 1 = bf16 pairs.  in0 / out0 / scratch0 are rank 0's
+// device addresses, the strides the byte distance to the next rank's copy.  `epoch` is the first
+// epoch this launch may use; *host_epochs_used (may be NULL) receives how many it consumes, so
+// the next launch passes epoch + that.  device_fail: one zeroed u32 that becomes 1 if a wait ran
+// out.  Returns 0 or a negative number for bad arguments / launch failure.
+int llbuffer_oneshot_allreduce(int mode, int P, int bf16, const void *in0, void *out0, size_t io_stride,
+                               void *scratch0, size_t scratch_stride, size_t nwords, unsigned long long epoch,
+                               int ctas, int threads, int slots_per_cta, unsigned *device_fail, void *cuda_stream,
+                               unsigned long long *host_epochs_used)
+{
+    if (!in0 || !out0 || !scratch0 || !device_fail || ctas < 1 || threads < 1 || threads > 1024 || slots_per_cta < 1)
+        return -1;
+    if (epoch == 0) return -1;
+    const size_t per_epoch = (size_t)ctas * slots_per_cta;
+    if (host_epochs_used) *host_epochs_used = (nwords + per_epoch - 1) / per_epoch + 1;   // + 1: a skipped flag value
+    const dim3 grid(ctas, P), block(threads);
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    cudaError_t e;
+    const char *i0 = (const char *)in0;
+    char *o0 = (char *)out0, *s0 = (char *)scratch0;
+    if (mode == 0)
+        e = bf16 ? launch<LLSync::LL, BF16x2Acc>(P, grid, block, s, i0, o0, io_stride, s0, scratch_stride, nwords, epoch, slots_per_cta, device_fail)
+                 : launch<LLSync::LL, F32Acc>(P, grid, block, s, i0, o0, io_stride, s0, scratch_stride, nwords, epoch, slots_per_cta, device_fail);
+    else if (mode == 1)
+        e = bf16 ? launch<LLSync::Sentinel, BF16x2Acc>(P, grid, block, s, i0, o0, io_stride, s0, scratch_stride, nwords, epoch, slots_per_cta, device_fail)
+                 : launch<LLSync::Sentinel, F32Acc>(P, grid, block, s, i0, o0, io_stride, s0, scratch_stride, nwords, epoch, slots_per_cta, device_fail);
+    else
+        return -1;
+    return e == cudaSuccess ? 0 : -3;
+}
+
+}  // extern "C"

@@ -67,6 +67,8 @@ SIGNATURES = [
     ("symar_probe_fence", c_int, [c_int, POINTER(c_double)]),
     ("symar_probe_pingpong", c_int, [c_int, POINTER(c_double)]),
     ("symar_probe_pingpong_pair", c_int, [c_int, c_int, POINTER(c_double), POINTER(c_int)]),
+    ("symar_llbuffer_bytes", c_size_t, [c_int, c_size_t, c_size_t, c_int, c_int]),
+    ("symar_llbuffer_init_sentinel", c_int, [c_void_p, c_size_t, c_void_p]),
     ("symar_probe_pingpong_blocks", c_int, [c_int, c_int, c_int, c_int, POINTER(c_double), POINTER(c_int)]),
 ]
 
@@ -336,6 +338,14 @@ def probe_pingpong(iterations: int = 20000) -> float:
     v = c_double()
     _ck(load().symar_probe_pingpong(iterations, byref(v)), "symar_probe_pingpong")
     return v.value
+
+
+def llbuffer_bytes(sync_mode: int, elem_bytes: int, slots_per_cta: int, ctas: int, round_robin: int) -> int:
+    return int(load().symar_llbuffer_bytes(sync_mode, elem_bytes, slots_per_cta, ctas, round_robin))
+
+
+def llbuffer_init_sentinel(device_ptr: int, nbytes: int, stream: int = 0) -> None:
+    _ck(load().symar_llbuffer_init_sentinel(device_ptr, nbytes, stream), "symar_llbuffer_init_sentinel")
 
 
 def probe_pingpong_blocks(first_block: int, partner_block: int, grid_blocks: int, iterations: int = 20000):
