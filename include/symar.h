@@ -21,8 +21,11 @@
  * with symheap_status) and the kernel returns normally.
  *
  * Environment (read when a heap is created): SYMAR_ALGO = oneshot | twoshot | ll |
- * sentinel replaces SYMAR_AUTO's choice; SYMAR_SPIN_LIMIT_US bounds device-side waits;
- * SYMAR_PDL = 1 enables programmatic dependent launch.
+ * sentinel | twoshot_ll | twoshot_sentinel | twoshot_atomic replaces SYMAR_AUTO's choice;
+ * SYMAR_CTAS_PER_RANK and SYMAR_THREADS fix the launch shape of every algorithm;
+ * SYMAR_SPIN_LIMIT_US bounds device-side waits; SYMAR_PDL = 0 turns programmatic dependent
+ * launch off; SYMAR_DEBUG = 1 logs every call's resolved algorithm and shape to stderr
+ * (nothing is printed otherwise).
  *
  * Threading: a heap may be used from one host thread and one stream at a time
  * (the per-CTA epoch counters live in the heap).  Calls on one stream are

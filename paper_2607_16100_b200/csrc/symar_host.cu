@@ -74,6 +74,7 @@ struct symheap {
     uint64_t  spin_ns = 2000000000ull;
     bool      pdl          = true;    // programmatic dependent launch of every kernel
     int       env_algo     = 0;       // SYMAR_ALGO override of SYMAR_AUTO, 0 = none
+    bool      debug_log    = false;   // SYMAR_DEBUG=1: one stderr line per call
     size_t    scratch_limit = 0;      // push algorithms: payload bytes per rank and iteration, 0 = all there is
     int       dbg_mute     = -1;
     unsigned  dbg_seed     = 0;
@@ -324,6 +325,9 @@ static int run(symheap *h, const void *in, void *out, size_t count, int dtype, i
     h->last_threads = p.cfg.threads;
     h->last_variant = p.args.variant;
     h->last_smem    = p.smem;
+    if (h->debug_log)
+        std::fprintf(stderr, "symar: allreduce count=%zu dtype=%d algo=%d grid=(%d,%d) block=%d variant=%#x smem=%zu pdl=%d\n",
+                     count, dtype, p.algo, p.cfg.ctas, h->P, p.cfg.threads, p.args.variant, p.smem, (int)h->pdl);
     return SYMAR_OK;
 }
 
@@ -619,8 +623,10 @@ static int create_common(symheap_t **heap, int P, size_t bytes_per_rank, void *m
         return cuda_fail(e, "heap initialisation");
     }
     // Environment overrides (read once per heap): SYMAR_SPIN_LIMIT_US bounds every
-    // device-side wait; SYMAR_ALGO = oneshot | twoshot | ll replaces SYMAR_AUTO's choice;
-    // SYMAR_PDL = 1 turns programmatic dependent launch on.
+    // device-side wait; SYMAR_ALGO = oneshot | twoshot | ll | ... replaces SYMAR_AUTO's choice;
+    // SYMAR_PDL = 0 turns programmatic dependent launch off; SYMAR_CTAS_PER_RANK and
+    // SYMAR_THREADS fix the launch shape of every algorithm; SYMAR_DEBUG = 1 logs every
+    // call's resolved algorithm and shape to stderr.
     if (const char *v = std::getenv("SYMAR_SPIN_LIMIT_US")) {
         const long us = std::atol(v);
         if (us > 0) h->spin_ns = (uint64_t)us * 1000ull;
@@ -632,6 +638,17 @@ static int create_common(symheap_t **heap, int P, size_t bytes_per_rank, void *m
                       : a == "twoshot_atomic" ? SYMAR_TWOSHOT_ATOMIC : 0;
     }
     if (const char *v = std::getenv("SYMAR_PDL")) h->pdl = std::atoi(v) != 0;
+    if (const char *v = std::getenv("SYMAR_CTAS_PER_RANK")) {
+        const int c = std::atoi(v);
+        if (c > 0 && c <= kMaxCtas)
+            for (int a = SYMAR_ONESHOT; a <= kLastAlgo; ++a) h->forced[a].ctas = c;
+    }
+    if (const char *v = std::getenv("SYMAR_THREADS")) {
+        const int t = std::atoi(v);
+        if (t > 0 && t <= (int)kMaxThreads)
+            for (int a = SYMAR_ONESHOT; a <= kLastAlgo; ++a) h->forced[a].threads = t;
+    }
+    if (const char *v = std::getenv("SYMAR_DEBUG")) h->debug_log = std::atoi(v) != 0;
     *heap = h;
     return SYMAR_OK;
 }

@@ -50,6 +50,7 @@ def test_binding_constants_match_header():
         assert m and int(m.group(1)) == val
     for name, val in (("SYMAR_AUTO", 0), ("SYMAR_ONESHOT", 1), ("SYMAR_TWOSHOT", 2), ("SYMAR_LL", 3),
                       ("SYMAR_SENTINEL", 4), ("SYMAR_TWOSHOT_LL", 5), ("SYMAR_TWOSHOT_SENTINEL", 6),
+                      ("SYMAR_TWOSHOT_ATOMIC", 7),
                       ("SYMAR_ERR_TIMEOUT", -4)):
         m = re.search(rf"{name}\s*=\s*(-?\d+)", HEADER)
         assert m and int(m.group(1)) == val

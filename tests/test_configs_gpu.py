@@ -138,3 +138,36 @@ def test_speed_of_light_probes_return_plausible_values():
     symar.probe_empty(4, 8, 128, s.cuda_stream)
     symar.probe_empty_pdl(4, 8, 128, s.cuda_stream)
     s.synchronize()
+
+
+def test_environment_overrides_are_read_at_heap_creation(monkeypatch, capfd):
+    monkeypatch.setenv("SYMAR_ALGO", "sentinel")
+    monkeypatch.setenv("SYMAR_CTAS_PER_RANK", "3")
+    monkeypatch.setenv("SYMAR_THREADS", "96")
+    monkeypatch.setenv("SYMAR_PDL", "0")
+    monkeypatch.setenv("SYMAR_DEBUG", "1")
+    h = symar.SymHeap.on_torch(4, 1 << 20)
+    try:
+        x = synth.make_inputs("normal", "bf16", 4, 3000, seed=5)
+        for q in range(4):
+            h.write_rank(q, 0, x[q])
+        h.allreduce(0, 1 << 19, 3000, symar.BF16, symar.AUTO)
+        torch.cuda.synchronize()
+        assert h.status()[0] == symar.OK
+        assert h.last_choice() == (symar.SENTINEL, 3, 96)
+        got = np.stack([h.read_rank(q, 1 << 19, 3000, np.uint16) for q in range(4)])
+        assert np.array_equal(got, O.allreduce(x))
+        err = capfd.readouterr().err
+        assert "symar: allreduce count=3000" in err and "pdl=0" in err and "block=96" in err
+    finally:
+        torch.cuda.synchronize()
+        h.destroy()
+    # and nothing is printed without SYMAR_DEBUG
+    monkeypatch.delenv("SYMAR_DEBUG")
+    h = symar.SymHeap.on_torch(2, 1 << 16)
+    try:
+        h.allreduce(0, 1 << 15, 16, symar.F32, symar.ONESHOT)
+        torch.cuda.synchronize()
+        assert capfd.readouterr().err == ""
+    finally:
+        h.destroy()
