@@ -59,7 +59,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(
-                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100",
+                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "50",
                  "-i", str(self.gpu)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.t = threading.Thread(target=self._pump, daemon=True)
             self.t.start()
@@ -80,7 +80,8 @@ class ClockSampler:
         except Exception:
             self.proc.kill()
         sm, mx, reasons = [], [], set()
-        rows = [l for (t, l) in self.lines if t_begin <= t <= t_end + 0.2] or [l for (_, l) in self.lines]
+        rows = [l for (t, l) in self.lines if t_begin <= t <= t_end + 0.02] or \
+            [l for (t, l) in self.lines if t_begin <= t <= t_end + 0.2] or [l for (_, l) in self.lines]
         for l in rows:
             f = [x.strip() for x in l.split(",")]
             if len(f) < 9:
@@ -474,7 +475,7 @@ def latency_suite(torch, symar, synth, hbm_gbs, quick=False, autotune=True):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=500)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--count", type=int, default=0, help="elements per rank (default: the 64 Mi workload)")
