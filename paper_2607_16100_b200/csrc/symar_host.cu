@@ -222,7 +222,7 @@ static int make_plan(symheap *h, size_t in_off, size_t out_off, size_t count, in
         const uint64_t nl = (ch + kAtLinePayload - 1) / kAtLinePayload;
         if (nl > at_lines_per_half(h->P)) return SYMAR_ERR_UNSUPPORTED;
         if (h->forced[algo].threads <= 0 && !(tuned && tn.cfg[algo][b].ctas > 0))
-            cfg.threads = nl * 8 >= 256 ? 256 : round_threads(std::max<uint64_t>(nl * 8, 32));
+            cfg.threads = nl * 8 >= 8192 ? 512 : (nl * 8 >= 256 ? 256 : round_threads(std::max<uint64_t>(nl * 8, 32)));
         cfg.threads = std::max(32, (cfg.threads + 31) / 32 * 32);
         if (h->forced[algo].ctas <= 0 && !(tuned && tn.cfg[algo][b].ctas > 0))
             cfg.ctas = (int)std::max<uint64_t>(
