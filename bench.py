@@ -291,6 +291,12 @@ def latency_suite(torch, symar, synth, hbm_gbs, quick=False, autotune=True):
                            "numerator and denominator use the same harness",
                 "p50_us": best["p50"], "best": best, "per_algo": row,
                 "twoshot_atomic_not_bit_reproducible": bench_size(8192, (symar.TWOSHOT_ATOMIC,))["twoshot_atomic"],
+                "in_kernel_span_us_p50": {
+                    names[a_]: float(np.median([h.debug_span(0, out_off, 8192, symar.BF16, a_) for _ in range(31)])) / 1e3
+                    for a_ in (symar.ONESHOT, symar.TWOSHOT, symar.LL, symar.SENTINEL)},
+                "in_kernel_span_note": "first CTA in (after its wait for the previous grid) -> last CTA out, device "
+                                       "nanosecond timer (about 32 ns resolution), single stream-launched calls "
+                                       "through the instrumented instantiation of the same kernels",
                 "sol_us": sol,
                 "sol_parts_us": {"empty_launch_same_shape": floor["p50"], "empty_launch_1x1": floor11["p50"],
                                  "flag_round_trip": rt_ns / 1000.0, "bytes_at_peak": t_bytes_us},

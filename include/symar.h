@@ -318,6 +318,15 @@ enum { SYMAR_STATIC_MAX_BYTES = 32768 };
 int allreduce_static(const void *in, void *out, size_t rank_pitch_bytes, int P, size_t count,
                      symar_dtype_t dtype, unsigned int *device_status, void *cuda_stream);
 
+/* Test hook: one allreduce() of the given arguments through the instrumented kernel
+ * instantiation, synchronously; *host_span_ns receives the time from the first CTA's start
+ * (after its wait for the previous grid) to the last CTA's end on the device's nanosecond
+ * timer (resolution about 32 ns): the protocol's own latency without the launch.  Not
+ * capturable.  SYMAR_ERR_UNSUPPORTED for the bulk-copy kernel, which has no test hooks
+ * (messages of 4 MiB per rank and more under SYMAR_TWOSHOT use the register kernel here).  */
+int symar_debug_span(symheap_t *heap, const void *in, void *out, size_t count, symar_dtype_t dtype,
+                     symar_algo_t algo, void *cuda_stream, double *host_span_ns);
+
 /* Text of the last CUDA error seen by the library on this thread (host string). */
 const char *symar_last_cuda_error(void);
 

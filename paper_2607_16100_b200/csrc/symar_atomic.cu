@@ -181,6 +181,7 @@ __global__ void __launch_bounds__(kMaxThreads) twoshot_atomic_kernel(const KArgs
     const bool all_ok = __syncthreads_and(ok);
     flag_exchange<P, true>(a, a.done_off, dcount, r, c, !all_ok, false, dwant);
     if (t == 0) *dcount = dwant;
+    if (DBG) debug_stamp_out(a);
 }
 
 using KernelFn = void (*)(const KArgs);

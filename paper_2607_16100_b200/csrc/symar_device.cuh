@@ -354,9 +354,25 @@ __device__ __forceinline__ void store_result(char *out, uint64_t v, const uint4 
     }
 }
 
-// ---- test hook: seeded start delay -------------------------------------------------
+// ---- test hook: in-kernel span (first CTA in -> last CTA out, nanosecond timer) --------
+__device__ __forceinline__ void debug_stamp_in(const KArgs &a)
+{
+    if (a.dbg_span && threadIdx.x == 0)
+        atomicMin(reinterpret_cast<unsigned long long *>(a.ctl + kCtlSpanIn), (unsigned long long)globaltimer_ns());
+}
+// every thread of the CTA calls it as its last action
+__device__ __forceinline__ void debug_stamp_out(const KArgs &a)
+{
+    if (!a.dbg_span) return;
+    __syncthreads();
+    if (threadIdx.x == 0)
+        atomicMax(reinterpret_cast<unsigned long long *>(a.ctl + kCtlSpanOut), (unsigned long long)globaltimer_ns());
+}
+
+// ---- test hook: seeded start delay (also stamps the CTA's start for the span hook) ----
 __device__ __forceinline__ void debug_delay(const KArgs &a, int rank, int cta)
 {
+    debug_stamp_in(a);
     if (a.dbg_delay_ns == 0) return;
     uint32_t h = a.dbg_seed ^ (uint32_t)(rank * 0x9E3779B1u) ^ (uint32_t)(cta * 0x85EBCA77u);
     h ^= h >> 16;

@@ -79,6 +79,7 @@ struct symheap {
     int       dbg_mute     = -1;
     unsigned  dbg_seed     = 0;
     unsigned  dbg_delay_ns = 0;
+    bool      dbg_span     = false;
     LaunchCfg forced[kAlgos];
     unsigned  variant[kAlgos] = {};
     bool      variant_forced[kAlgos] = {};
@@ -93,7 +94,7 @@ namespace symar {
 
 static size_t elem_size(int dtype) { return dtype == SYMAR_F32 ? 4 : 2; }
 static bool   valid_P(int P) { return P == 1 || P == 2 || P == 4 || P == 8; }
-static bool   dbg_on(const symheap *h) { return h->dbg_mute >= 0 || h->dbg_delay_ns != 0; }
+static bool   dbg_on(const symheap *h) { return h->dbg_mute >= 0 || h->dbg_delay_ns != 0 || h->dbg_span; }
 
 static int bucket_of(size_t bytes)
 {
@@ -265,6 +266,7 @@ static int make_plan(symheap *h, size_t in_off, size_t out_off, size_t count, in
     a.dbg_mute   = h->dbg_mute;
     a.dbg_seed   = h->dbg_seed;
     a.dbg_delay_ns = h->dbg_delay_ns;
+    a.dbg_span   = h->dbg_span ? 1u : 0u;
     if (algo == SYMAR_TWOSHOT) {
         const bool cyclic = nvec >= kCyclicMinVec && !(var & 1u);
         a.blk_log2 = cyclic ? kCyclicLog2 : kOneChunk;
@@ -1016,6 +1018,26 @@ int symar_debug_inject(symheap_t *heap, int mute_rank, unsigned int delay_seed, 
 }
 
 const char *symar_last_cuda_error(void) { return g_last_cuda_error.c_str(); }
+
+int symar_debug_span(symheap_t *heap, const void *in, void *out, size_t count, symar_dtype_t dtype,
+                     symar_algo_t algo, void *cuda_stream, double *host_span_ns)
+{
+    if (!heap || !host_span_ns) return SYMAR_ERR_INVAL;
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    const unsigned long long init[2] = {~0ull, 0ull};
+    CU(cudaMemcpyAsync(heap->ctl + kCtlSpanIn, init, sizeof init, cudaMemcpyHostToDevice, s));
+    CU(cudaStreamSynchronize(s));                       // `init` is on this stack frame
+    heap->dbg_span = true;
+    const int rc = run(heap, in, out, count, (int)dtype, (int)algo, s);
+    heap->dbg_span = false;
+    if (rc != SYMAR_OK) return rc;
+    unsigned long long w[2] = {0, 0};
+    CU(cudaMemcpyAsync(w, heap->ctl + kCtlSpanIn, sizeof w, cudaMemcpyDeviceToHost, s));
+    CU(cudaStreamSynchronize(s));
+    if (w[0] == ~0ull || w[1] < w[0]) return SYMAR_ERR_UNSUPPORTED;     // this kernel carries no stamps
+    *host_span_ns = (double)(w[1] - w[0]);
+    return SYMAR_OK;
+}
 
 size_t symar_llbuffer_bytes(int sync_mode, size_t elem_bytes, size_t slots_per_cta, int ctas, int round_robin)
 {

@@ -76,6 +76,7 @@ __global__ void __launch_bounds__(kMaxThreads) oneshot_kernel(const KArgs a)
             }
         }
     }
+    if (DBG) debug_stamp_out(a);
 }
 
 // The same for two adjacent vectors moved as one 32-byte access per peer.
@@ -159,6 +160,7 @@ __global__ void __launch_bounds__(kMaxThreads) twoshot_kernel(const KArgs a)
         *rcount = rwant;
         *dcount = dwant;
     }
+    if (DBG) debug_stamp_out(a);
 }
 
 // LL with 8 bytes of payload per thread: one 16-byte {w0,f,w1,f} store per peer and
@@ -335,6 +337,7 @@ __global__ void __launch_bounds__(kMaxThreads) ll_kernel(const KArgs a)
     }
     __syncthreads();          // every thread has read the counter before it moves
     if (t == 0) *ep = n0 + a.iters;
+    if (DBG) debug_stamp_out(a);
 }
 
 // One-shot push with sentinel synchronisation (Sec. IV "Sentinel"; Sec. V send / recv with
@@ -427,6 +430,7 @@ __global__ void __launch_bounds__(kMaxThreads) sentinel_kernel(const KArgs a)
     }
     __syncthreads();
     if (t == 0) *ep = n0 + a.iters;
+    if (DBG) debug_stamp_out(a);
 }
 
 // ---- two-shot over the push buffers (the paper's AllReduce_LLBuffer_Twoshot; Table I rows
@@ -598,6 +602,7 @@ __global__ void __launch_bounds__(kPushTwoshotMaxThreads) twoshot_push_kernel(co
     }
     __syncthreads();
     if (t == 0) *ep = n0 + a.iters;
+    if (DBG) debug_stamp_out(a);
 }
 
 // ---- dispatch ---------------------------------------------------------------------

@@ -60,7 +60,8 @@ __host__ __device__ constexpr size_t bulk_smem_bytes(int P, uint32_t tile_vecs, 
 }
 
 // control block words (u32)
-enum : int { kCtlCode = 0, kCtlRank = 1, kCtlPeer = 2, kCtlCta = 3 };
+enum : int { kCtlCode = 0, kCtlRank = 1, kCtlPeer = 2, kCtlCta = 3,
+             kCtlSpanIn = 16, kCtlSpanOut = 18 };   // two u64 (byte 64, 72): first CTA in, last CTA out (test hook)
 
 __host__ __device__ constexpr size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
@@ -147,6 +148,7 @@ struct KArgs {
     int32_t   dbg_mute;      // test hook: rank that stays silent, -1 = none
     uint32_t  dbg_seed;
     uint32_t  dbg_delay_ns;
+    uint32_t  dbg_span;      // test hook: record when the first CTA started and the last one finished
 };
 
 }  // namespace symar

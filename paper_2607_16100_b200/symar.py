@@ -67,6 +67,7 @@ SIGNATURES = [
     ("symar_probe_fence", c_int, [c_int, POINTER(c_double)]),
     ("symar_probe_pingpong", c_int, [c_int, POINTER(c_double)]),
     ("symar_probe_pingpong_pair", c_int, [c_int, c_int, POINTER(c_double), POINTER(c_int)]),
+    ("symar_debug_span", c_int, [c_void_p, c_void_p, c_void_p, c_size_t, c_int, c_int, c_void_p, POINTER(c_double)]),
     ("symar_llbuffer_bytes", c_size_t, [c_int, c_size_t, c_size_t, c_int, c_int]),
     ("symar_llbuffer_init_sentinel", c_int, [c_void_p, c_size_t, c_void_p]),
     ("symar_probe_pingpong_blocks", c_int, [c_int, c_int, c_int, c_int, POINTER(c_double), POINTER(c_int)]),
@@ -302,6 +303,13 @@ class SymHeap:
 
     def set_spin_limit_us(self, us: int) -> None:
         _ck(self._lib.symar_set_spin_limit_us(self._h, us), "symar_set_spin_limit_us")
+
+    def debug_span(self, in_off: int, out_off: int, count: int, dtype: int, algo: int = AUTO, stream: int = 0) -> float:
+        """In-kernel span in ns (first CTA in -> last CTA out) of one synchronous call."""
+        v = c_double()
+        _ck(self._lib.symar_debug_span(self._h, self.rank_ptr(0, in_off), self.rank_ptr(0, out_off), count, dtype,
+                                       algo, stream, byref(v)), "symar_debug_span")
+        return v.value
 
     def debug_inject(self, mute_rank: int = -1, delay_seed: int = 0, delay_max_ns: int = 0) -> None:
         _ck(self._lib.symar_debug_inject(self._h, mute_rank, delay_seed, delay_max_ns), "symar_debug_inject")

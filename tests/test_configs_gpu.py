@@ -171,3 +171,23 @@ def test_environment_overrides_are_read_at_heap_creation(monkeypatch, capfd):
         assert capfd.readouterr().err == ""
     finally:
         h.destroy()
+
+
+def test_in_kernel_span_hook_measures_and_keeps_results():
+    h = symar.SymHeap.on_torch(8, 1 << 20)
+    try:
+        x = synth.make_inputs("normal", "bf16", 8, 8192, seed=2)
+        for q in range(8):
+            h.write_rank(q, 0, x[q])
+        want = O.allreduce(x)
+        for algo in (symar.ONESHOT, symar.TWOSHOT, symar.LL, symar.SENTINEL, symar.TWOSHOT_LL,
+                     symar.TWOSHOT_SENTINEL):
+            spans = [h.debug_span(0, 1 << 19, 8192, symar.BF16, algo) for _ in range(5)]
+            assert all(100.0 <= s <= 200_000.0 for s in spans), (algo, spans)     # 0.1 us ... 0.2 ms
+            got = np.stack([h.read_rank(q, 1 << 19, 8192, np.uint16) for q in range(8)])
+            assert np.array_equal(got, want), algo
+        assert h.debug_span(0, 1 << 19, 8192, symar.BF16, symar.TWOSHOT_ATOMIC) > 0
+        assert h.status()[0] == symar.OK
+    finally:
+        torch.cuda.synchronize()
+        h.destroy()
