@@ -477,6 +477,19 @@ def latency_suite(torch, symar, synth, hbm_gbs, quick=False, autotune=True):
     return out
 
 
+def finite(obj):
+    """JSON has no NaN or Infinity: non-finite numbers become null."""
+    if isinstance(obj, float):
+        return obj if np.isfinite(obj) else None
+    if isinstance(obj, dict):
+        return {k: finite(v) for k, v in obj.items()}
+    if isinstance(obj, (list, tuple)):
+        return [finite(v) for v in obj]
+    if isinstance(obj, np.generic):
+        return finite(obj.item())
+    return obj
+
+
 # ---------------------------------------------------------------------------------
 def main():
     ap = argparse.ArgumentParser()
@@ -525,7 +538,7 @@ def main():
                     "note": "latency section only"}
             line.update(latency_suite(torch, symar, synth, hbm_gbs, quick=args.quick,
                                       autotune=not args.no_autotune))
-            print(json.dumps(line))
+            print(json.dumps(finite(line), allow_nan=False))
         if world > 1:
             dist.barrier()
             dist.destroy_process_group()
@@ -693,13 +706,16 @@ def main():
     del x
 
     if rank == 0 and not args.no_latency:
-        line.update(latency_suite(torch, symar, synth, hbm_gbs, quick=args.quick, autotune=not args.no_autotune))
+        try:
+            line.update(latency_suite(torch, symar, synth, hbm_gbs, quick=args.quick, autotune=not args.no_autotune))
+        except Exception as exc:                      # the bandwidth line above must still be reported
+            line["latency_section_error"] = f"{type(exc).__name__}: {exc}"
 
     if world > 1:
         dist.barrier()
         dist.destroy_process_group()
     if rank == 0:
-        print(json.dumps(line))
+        print(json.dumps(finite(line), allow_nan=False))
 
 
 if __name__ == "__main__":
