@@ -3,18 +3,25 @@
 // rank.  CTAs of different ranks meet only through the symmetric heap, as GPUs
 // of one NVLink domain would.
 //
-//   oneshot_kernel  Sec. III-A.1 (pull): exchange "input ready" signals with
-//                   every peer, read all P inputs, reduce, write the own output.
-//   twoshot_kernel  Sec. III-A.2: the same exchange, reduce only the owned
-//                   vectors, store them into every rank's output (all-gather
-//                   from registers), then hand off with "done" signals.
-//   ll_kernel       Sec. IV "LL" + Sec. V example kernel: push every input word
-//                   to every peer's scratch as {payload, flag} 8-byte stores,
-//                   poll the own scratch, reduce, write the own output; scratch
-//                   is double-buffered by iteration parity.
+//   oneshot_kernel       Sec. III-A.1 (pull): exchange "input ready" signals with
+//                        every peer, read all P inputs, reduce, write the own output.
+//   twoshot_kernel       Sec. III-A.2: the same exchange, reduce only the owned
+//                        vectors, store them into every rank's output (all-gather
+//                        from registers), then hand off with "done" signals.
+//   ll_kernel            Sec. IV "LL" + Sec. V example kernel: push every input word
+//                        to every peer's scratch as {payload, flag} 8-byte stores,
+//                        poll the own scratch, reduce, write the own output; scratch
+//                        is double-buffered by iteration parity.
+//   sentinel_kernel      Sec. IV "Sentinel": the same push with bare payload into
+//                        scratch that holds a sentinel word; the receiver polls
+//                        until every word has changed and restores the sentinel.
+//   twoshot_push_kernel  Table I "Two-shot (LL)" / "Two-shot (Sentinel)": reduce-
+//                        scatter and all-gather both pushed through the scratch,
+//                        synchronised by the data itself.
 //
-// (The two-shot kernel for the bandwidth regime, built on bulk asynchronous
-// copies, lives in symar_bulk.cu.)
+// (Elsewhere: the two-shot kernel of the bandwidth regime on bulk asynchronous
+// copies in symar_bulk.cu, the atomic two-shot in symar_atomic.cu, the sibling
+// collectives in symar_coll.cu.)
 //
 // No kernel contains a grid-wide barrier; every wait is one-directional (a CTA
 // waits for data or a signal FROM each peer) and bounded.
