@@ -50,9 +50,7 @@ __device__ __forceinline__ void oneshot_units(const KArgs &a, char *out, uint64_
 template <typename E, int P, bool DBG>
 __global__ void __launch_bounds__(kMaxThreads) oneshot_kernel(const KArgs a)
 {
-    const bool rank_major = a.variant & 0x800u;
-    const int c = rank_major ? blockIdx.y : blockIdx.x, r = rank_major ? blockIdx.x : blockIdx.y,
-              C = rank_major ? gridDim.y : gridDim.x;
+    const int c = blockIdx.x, r = blockIdx.y, C = gridDim.x;
     const uint32_t t = threadIdx.x, T = blockDim.x;
     char *seg_r = a.seg0 + (size_t)r * a.stride;
     uint32_t *count = reinterpret_cast<uint32_t *>(seg_r + a.epoch_off + ready_count_off(c));
@@ -650,8 +648,7 @@ KernelFn kernel_for(int algo, int dtype, int P, bool dbg)
 cudaError_t launch_kernel(KernelFn fn, int P, int ctas_per_rank, int threads, size_t smem_bytes,
                           const KArgs &args, cudaStream_t stream)
 {
-    const dim3 grid = (args.variant & 0x800u) ? dim3((unsigned)P, (unsigned)ctas_per_rank, 1)
-                                               : dim3((unsigned)ctas_per_rank, (unsigned)P, 1);
+    const dim3 grid((unsigned)ctas_per_rank, (unsigned)P, 1);
     if (!args.pdl) {
         fn<<<grid, dim3((unsigned)threads, 1, 1), smem_bytes, stream>>>(args);
         return cudaGetLastError();
