@@ -689,19 +689,21 @@ def main():
     del heap
 
     if rank == 0 and not args.no_cpu:
-        xs = x if count <= (16 << 20) else np.ascontiguousarray(x[:, :16 << 20])
+        # the oracle as it stands on the whole workload (it needs about 0.1 s per call on 16 cores)
         best, team = 1e30, 1
-        for _ in range(3):
+        t_all = time.perf_counter()
+        for _ in range(5):
             t0 = time.perf_counter()
-            _, team = O.allreduce_timed_team(xs, threads=0)
+            _, team = O.allreduce_timed_team(x, threads=0)
             best = min(best, time.perf_counter() - t0)
         t0 = time.perf_counter()
-        O.allreduce_timed_team(xs, threads=1)
+        O.allreduce_timed_team(x, threads=1)
         one = time.perf_counter() - t0
         line["cpu_baseline"] = {
-            "value": 2 * P * xs.shape[1] * 4 / best / 1e9, "unit": "GB/s", "cores": team, "kind": "oracle",
-            "sample": f"first {xs.shape[1]} of {count} elements per rank, best of 3 full oracle calls "
-                      f"(OpenMP over elements); single-thread: {2 * P * xs.shape[1] * 4 / one / 1e9:.2f} GB/s",
+            "value": 2 * P * count * 4 / best / 1e9, "unit": "GB/s", "cores": team, "kind": "oracle",
+            "sample": f"the whole workload ({count} elements per rank), best of 5 full oracle calls (OpenMP over "
+                      f"elements) + one single-thread call: {2 * P * count * 4 / one / 1e9:.2f} GB/s; "
+                      f"{time.perf_counter() - t_all:.1f} s of CPU time in all",
         }
     del x
 
