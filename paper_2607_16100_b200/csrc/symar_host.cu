@@ -212,7 +212,8 @@ static int make_plan(symheap *h, size_t in_off, size_t out_off, size_t count, in
     const unsigned var = (unsigned)cfg.variant;
 
     cfg.threads = std::min<int>(std::max(32, (cfg.threads + 31) / 32 * 32),
-                                is_twoshot_push(algo) ? (int)kPushTwoshotMaxThreads : (int)kMaxThreads);
+                                is_twoshot_push(algo) ? (int)kPushTwoshotMaxThreads
+                                                      : (algo == SYMAR_LL ? (int)kLLMaxThreads : (int)kMaxThreads));
     KArgs &a = p->args;
     std::memset(&a, 0, sizeof a);
     KernelFn fn = any_kernel_for(algo, dtype, h->P, dbg_on(h));

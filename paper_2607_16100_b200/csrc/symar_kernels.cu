@@ -246,7 +246,7 @@ __device__ __forceinline__ bool ll_iteration_narrow(const KArgs &a, int r, int c
 }
 
 template <typename E, int P, bool DBG>
-__global__ void __launch_bounds__(kMaxThreads) ll_kernel(const KArgs a)
+__global__ void __launch_bounds__(kLLMaxThreads) ll_kernel(const KArgs a)
 {
     const int c = blockIdx.x, r = blockIdx.y, C = gridDim.x;
     const uint32_t t = threadIdx.x, T = blockDim.x;

@@ -32,6 +32,7 @@ constexpr size_t   kCtlBytes    = SYMAR_ALIGN;      // control block at the heap
 constexpr size_t   kFlagGroup   = 32;               // kMaxRanks x u32: one L2 sector per (rank, slot)
 constexpr size_t   kMaxThreads  = 512;
 constexpr size_t   kPushTwoshotMaxThreads = 256;    // that kernel keeps 3 P vectors live per thread: give it registers
+constexpr size_t   kLLMaxThreads = 256;             // the LL poll keeps 2 P flagged vectors live per thread: likewise
 
 // byte offsets of the two u32 exchange counters of slot c, relative to epoch_off
 __host__ __device__ constexpr size_t ready_count_off(int c) { return (size_t)kMaxCtas * 8 + (size_t)c * 4; }

@@ -128,8 +128,8 @@ def test_forced_launch_shapes(heaps, algo, ctas, threads):
     try:
         got = run(h, x, symar.BF16, algo)
         a, c, t = h.last_choice()
-        if algo in (symar.TWOSHOT_LL, symar.TWOSHOT_SENTINEL):
-            # register-heavy kernel: at most 256 threads, and the library clamps the grid to
+        if algo in (symar.LL, symar.TWOSHOT_LL, symar.TWOSHOT_SENTINEL):
+            # register-heavy kernels: at most 256 threads, and the library clamps the grid to
             # what is co-resident (CTAs of different ranks wait for one another)
             assert a == algo and t == min(threads, 256) and 1 <= c <= ctas
         else:
