@@ -78,10 +78,35 @@ def test_c4_full_size_p8_fp32_256MiB():
         assert h.status()[0] == symar.OK
         assert h.last_kernel()[1] > 0                            # the bulk-copy kernel ran
         want_bits = want.view(np.uint32)
-        for r in range(P):
-            got = h.read_rank(r, M, count, np.float32).view(np.uint32)
-            bad = np.flatnonzero(got != want_bits)
-            assert bad.size == 0, f"rank {r}: {bad.size} mismatches, first at {bad[0]}"
+
+        def check_all(what):
+            for r in range(P):
+                got = h.read_rank(r, M, count, np.float32).view(np.uint32)
+                bad = np.flatnonzero(got != want_bits)
+                assert bad.size == 0, f"{what}, rank {r}: {bad.size} mismatches, first at {bad[0]}"
+                h.write_rank(r, M, np.zeros(1 << 20, dtype=np.uint8))      # stale results must not pass the next check
+
+        check_all("default shape")
+        # the register kernel in the shape the tuner tends to pick for this size
+        h.set_launch(symar.TWOSHOT, 15, 512)
+        h.set_variant(symar.TWOSHOT, 4)
+        h.allreduce(0, M, count, symar.F32, symar.TWOSHOT)
+        torch.cuda.synchronize()
+        assert h.last_kernel()[1] == 0 and h.last_choice() == (symar.TWOSHOT, 15, 512)
+        check_all("register kernel 15 x 512")
+        h.set_launch(symar.TWOSHOT, 0, 0)
+        h.set_variant(symar.TWOSHOT, 0)
+        # and exactly what bench.py times: the shape tuned for this size on this GPU (tuning overwrites
+        # the user region, so the inputs go in again)
+        x = synth.make_inputs(w["dist"], "f32", P, count, w["seed"])
+        h.autotune_size(symar.F32, count)
+        for q in range(P):
+            h.write_rank(q, 0, x[q])
+        del x
+        h.allreduce(0, M, count, symar.F32, symar.TWOSHOT)
+        torch.cuda.synchronize()
+        assert h.status()[0] == symar.OK
+        check_all(f"tuned shape {h.last_choice()} kernel {h.last_kernel()}")
     finally:
         h.destroy()
 
