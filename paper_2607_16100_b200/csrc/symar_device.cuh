@@ -162,6 +162,10 @@ __device__ __forceinline__ void pdl_wait_holding(const void *p0, const void *p1,
 }
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;"); }
 
+// L2 prefetch hint.  Safe on memory that an earlier kernel may still be writing: no data
+// is returned, and L2 is the point of coherence, so a later write simply updates the line.
+__device__ __forceinline__ void prefetch_l2(const void *p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
+
 // ---- bounded waiting ------------------------------------------------------------
 // Counts polls in a register; every 256th poll reads the nanosecond timer.  The
 // first reading starts the clock, so the fast path never touches the timer.

@@ -55,7 +55,19 @@ __global__ void __launch_bounds__(kMaxThreads) oneshot_kernel(const KArgs a)
     char *seg_r = a.seg0 + (size_t)r * a.stride;
     uint32_t *count = reinterpret_cast<uint32_t *>(seg_r + a.epoch_off + ready_count_off(c));
     const ExchangePtrs xp = exchange_ptrs<P>(a, a.ready_off, r, c);
-    if (a.pdl) pdl_wait_holding(xp.signal, xp.mine, count);   // the previous call has left the heap
+    if (a.pdl) {
+        // Made resident early, this CTA has time while its predecessor still runs: pull the peers'
+        // input lines of its first passes towards L2 (a hint only -- if a line is still being written,
+        // the write lands in L2 all the same).  One thread per 128-byte line.
+        const uint32_t ub = 16u >> ((a.variant >> 8) & 3u);                    // bytes per thread and pass
+        uint64_t off = ((uint64_t)c * T + t) * ub;
+        for (int pass = 0; pass < 4 && off < a.nvec * 16; ++pass, off += (uint64_t)C * T * ub) {
+            if ((off & 127u) != 0) break;                                       // T * ub is a multiple of 128
+#pragma unroll
+            for (int q = 0; q < P; ++q) prefetch_l2(a.seg0 + (size_t)q * a.stride + a.in_off + off);
+        }
+        pdl_wait_holding(xp.signal, xp.mine, count);   // the previous call has left the heap
+    }
     if (DBG) debug_delay(a, r, c);
     if (DBG && a.dbg_mute == r) return;       // test hook: this rank never joins
 
