@@ -657,9 +657,22 @@ def main():
         line["roofline"]["traffic_source"] = kv["source "].strip()
 
     # end to end through the host-buffer entry point
-    if not args.no_e2e:
-        hin = torch.from_numpy(x).pin_memory()
-        hout = torch.empty_like(hin).pin_memory()
+    e2e_ready = not args.no_e2e
+    if e2e_ready:
+        # 2 x P x M bytes of pinned host memory per rank; if any rank cannot get them, all skip
+        try:
+            hin = torch.from_numpy(x).pin_memory()
+            hout = torch.empty_like(hin).pin_memory()
+        except RuntimeError as exc:
+            e2e_ready = False
+            line["e2e_skipped"] = f"pinned host buffers: {exc}"
+        if world > 1:
+            flag = torch.tensor([1.0 if e2e_ready else 0.0], device="cuda")
+            dist.all_reduce(flag, op=dist.ReduceOp.MIN)
+            if e2e_ready and flag.item() == 0.0:
+                e2e_ready = False
+                line["e2e_skipped"] = "another rank could not allocate its pinned host buffers"
+    if e2e_ready:
         e2e_steps = min(args.steps, 5)
         estep = lambda: heap.allreduce_host(hin.data_ptr(), hout.data_ptr(), in_off, out_off, count,
                                             symar.F32, symar.TWOSHOT, sh)
