@@ -168,8 +168,12 @@ int allreduce(symheap_t *heap, const void *in, void *out, size_t count,
 /* The same collective for HOST buffers (end-to-end path): copies row q of
  * host_in ([P][count] elements, row-major, host memory, ideally pinned) to rank
  * q's `in`, runs allreduce(), copies every rank's `out` to row r of host_out
- * ([P][count]).  All copies and the kernel are enqueued on `cuda_stream`; the
- * host buffers must stay valid until the stream has drained.                   */
+ * ([P][count]).  Ordered on `cuda_stream` like any other call; the host buffers
+ * must stay valid until the stream has drained.  Messages of 32 MiB per rank and
+ * more are cut into 16 MiB chunks (an elementwise sum is a sum of its chunks) that
+ * move on two copy streams of the heap, so that chunk i+1 travels to the device
+ * while chunk i is reduced and chunk i-1 travels back: one kernel per chunk, both
+ * directions of the host link busy at once.  The algorithm is resolved per chunk. */
 int allreduce_host(symheap_t *heap, const void *host_in, void *host_out,
                    const void *in, void *out, size_t count,
                    symar_dtype_t dtype, symar_algo_t algo, void *cuda_stream);

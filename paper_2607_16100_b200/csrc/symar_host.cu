@@ -88,6 +88,9 @@ struct symheap {
     unsigned  last_variant = 0;
     size_t    last_smem = 0;
     std::map<std::tuple<const void *, int>, int> resident;   // (kernel, threads) -> CTAs co-resident
+    // allreduce_host() on large messages: copy streams and events of the chunk pipeline (made on first use)
+    cudaStream_t h2d = nullptr, d2h = nullptr;
+    std::vector<cudaEvent_t> pipe_ev;
 };
 
 namespace symar {
@@ -721,6 +724,9 @@ int symheap_destroy(symheap_t *heap)
         cudaError_t e = cudaFree(heap->mem);
         if (e != cudaSuccess) rc = cuda_fail(e, "cudaFree");
     }
+    for (cudaEvent_t ev : heap->pipe_ev) cudaEventDestroy(ev);
+    if (heap->h2d) cudaStreamDestroy(heap->h2d);
+    if (heap->d2h) cudaStreamDestroy(heap->d2h);
     delete heap;
     return rc;
 }
@@ -778,6 +784,54 @@ int allreduce(symheap_t *heap, const void *in, void *out, size_t count, symar_dt
     return run(heap, in, out, count, (int)dtype, (int)algo, (cudaStream_t)cuda_stream);
 }
 
+// Host-buffer path for large messages: the message is cut into chunks; chunk i+1 travels to the
+// device while chunk i is reduced and chunk i-1 travels back (the AllReduce is elementwise, so a
+// chunk is an AllReduce of its own).  Both directions of the host link are busy at once.
+constexpr size_t kHostChunkBytes = (size_t)16 << 20;      // per rank
+constexpr int    kHostMaxChunks  = 64;
+
+static int host_pipeline(symheap *h, const char *host_in, char *host_out, size_t io, size_t oo, size_t count, int dtype,
+                         int algo, cudaStream_t s)
+{
+    const size_t es = elem_size(dtype), bytes = count * es;
+    size_t chunk = kHostChunkBytes;
+    while ((bytes + chunk - 1) / chunk > (size_t)kHostMaxChunks) chunk *= 2;
+    const int n = (int)((bytes + chunk - 1) / chunk);
+    if (!h->h2d) {
+        CU(cudaStreamCreateWithFlags(&h->h2d, cudaStreamNonBlocking));
+        CU(cudaStreamCreateWithFlags(&h->d2h, cudaStreamNonBlocking));
+    }
+    while (h->pipe_ev.size() < (size_t)(2 * kHostMaxChunks + 2)) {
+        cudaEvent_t ev;
+        CU(cudaEventCreateWithFlags(&ev, cudaEventDisableTiming));
+        h->pipe_ev.push_back(ev);
+    }
+    cudaEvent_t start = h->pipe_ev[0], end = h->pipe_ev[1];
+    CU(cudaEventRecord(start, s));                          // everything enqueued so far comes first
+    CU(cudaStreamWaitEvent(h->h2d, start, 0));
+    for (int i = 0; i < n; ++i) {
+        const size_t off = (size_t)i * chunk, len = std::min(chunk, bytes - off);
+        for (int q = 0; q < h->P; ++q)
+            CU(cudaMemcpyAsync(h->seg0 + (size_t)q * h->L.stride + io + off, host_in + (size_t)q * bytes + off, len,
+                               cudaMemcpyHostToDevice, h->h2d));
+        CU(cudaEventRecord(h->pipe_ev[2 + 2 * i], h->h2d));
+    }
+    for (int i = 0; i < n; ++i) {
+        const size_t off = (size_t)i * chunk, len = std::min(chunk, bytes - off);
+        CU(cudaStreamWaitEvent(s, h->pipe_ev[2 + 2 * i], 0));
+        const int rc = run(h, h->seg0 + io + off, h->seg0 + oo + off, len / es, dtype, algo, s);
+        if (rc != SYMAR_OK) return rc;
+        CU(cudaEventRecord(h->pipe_ev[3 + 2 * i], s));
+        CU(cudaStreamWaitEvent(h->d2h, h->pipe_ev[3 + 2 * i], 0));
+        for (int r = 0; r < h->P; ++r)
+            CU(cudaMemcpyAsync(host_out + (size_t)r * bytes + off, h->seg0 + (size_t)r * h->L.stride + oo + off, len,
+                               cudaMemcpyDeviceToHost, h->d2h));
+    }
+    CU(cudaEventRecord(end, h->d2h));
+    CU(cudaStreamWaitEvent(s, end, 0));                     // the caller's stream sees the results
+    return SYMAR_OK;
+}
+
 int allreduce_host(symheap_t *heap, const void *host_in, void *host_out, const void *in, void *out,
                    size_t count, symar_dtype_t dtype, symar_algo_t algo, void *cuda_stream)
 {
@@ -785,9 +839,12 @@ int allreduce_host(symheap_t *heap, const void *host_in, void *host_out, const v
     int rc = check_buffers(heap, in, out, count, (int)dtype, &io, &oo);
     if (rc != SYMAR_OK) return rc;
     if (!host_in || !host_out) return SYMAR_ERR_INVAL;
+    if ((int)algo < SYMAR_AUTO || (int)algo > kLastAlgo) return SYMAR_ERR_INVAL;
     if (count == 0) return SYMAR_OK;
     cudaStream_t s     = (cudaStream_t)cuda_stream;
     const size_t bytes = count * elem_size((int)dtype);
+    if (bytes >= 2 * kHostChunkBytes && (io % 16 == 0) && (oo % 16 == 0))
+        return host_pipeline(heap, (const char *)host_in, (char *)host_out, io, oo, count, (int)dtype, (int)algo, s);
     for (int q = 0; q < heap->P; ++q)
         CU(cudaMemcpyAsync(heap->seg0 + (size_t)q * heap->L.stride + io, (const char *)host_in + (size_t)q * bytes,
                            bytes, cudaMemcpyHostToDevice, s));
