@@ -695,7 +695,8 @@ def main():
         line["e2e"] = {"value": whole_job_value(algbytes, world, e2e_steps, e_ms) / 1e9, "unit": "GB/s",
                        "h2d_bytes_per_step": P * M, "d2h_bytes_per_step": P * M, "steps": e2e_steps,
                        "ms_per_step": e_ms / e2e_steps, "bit_exact_sampled": e2e_exact,
-                       "note": "allreduce_host(): pinned host inputs -> HBM, kernel, all P outputs -> pinned host"}
+                       "note": "allreduce_host(): pinned host inputs -> HBM, kernels, all P outputs -> pinned host, in 16 MiB "
+                               "chunks on two copy streams (one kernel per chunk; both link directions busy at once)"}
         del hin, hout
 
     heap.destroy()
