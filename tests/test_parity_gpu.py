@@ -579,6 +579,41 @@ def test_host_buffer_entry_point_pipelines_large_messages():
         h.destroy()
 
 
+def test_capture_with_foreign_kernels_copies_and_the_host_pipeline():
+    # every launch carries the programmatic-dependent-launch attribute by default: it must capture
+    # behind kernels of other libraries and behind copy nodes, and the chunked host path must
+    # fork and join its copy streams inside the capture
+    P, count = 2, 9 * (1 << 20) + 77                             # 36 MiB per rank: three chunks
+    M = count * 4
+    out_off = (M + 4095) // 4096 * 4096
+    h = symar.SymHeap.on_torch(P, out_off + M)
+    try:
+        x = synth.make_inputs("uniform", "f32", P, count, seed=23)
+        small = np.ascontiguousarray(x[:, :6000])
+        hin = torch.from_numpy(x).pin_memory()
+        hout = torch.empty_like(hin).pin_memory()
+        other = torch.zeros(1 << 16, device="cuda")
+        s = torch.cuda.Stream()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=s):
+            cs = torch.cuda.current_stream().cuda_stream
+            other.fill_(1.0)                                     # a kernel of another library
+            h.allreduce_host(hin.data_ptr(), hout.data_ptr(), 0, out_off, count, symar.F32, symar.AUTO, cs)
+            other.add_(1.0)
+            h.allreduce(0, out_off, 6000, symar.F32, symar.ONESHOT, cs)     # first 6000 elements again
+        for _ in range(3):
+            hout.zero_()
+            g.replay()
+        torch.cuda.synchronize()
+        assert h.status()[0] == symar.OK and float(other[0]) == 2.0
+        assert_bits(hout.numpy(), O.allreduce(x))
+        got = np.stack([h.read_rank(q, out_off, 6000, np.float32) for q in range(P)])
+        assert_bits(got, O.allreduce(small))
+    finally:
+        torch.cuda.synchronize()
+        h.destroy()
+
+
 def test_library_owned_heap():
     h = symar.SymHeap(2, 1 << 16)
     try:
