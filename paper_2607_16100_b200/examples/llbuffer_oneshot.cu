@@ -8,7 +8,9 @@
 // The P ranks are the rows of the grid (blockIdx.y), as everywhere in this library; all
 // P * ctas CTAs wait for one another and must be co-resident, so keep the grid small.
 // Not a tuned kernel: it shows that a collective is a dozen lines on top of the primitives,
-// and it is the test vehicle of the header (tests/test_llbuffer_gpu.py).
+// and it is the test vehicle of the header (tests/test_llbuffer_gpu.py).  A second kernel
+// further down, an all-gather of 64-bit words, covers 8-byte elements and the single
+// send / recv / reset calls on an undivided buffer.
 #include <cuda_runtime.h>
 #include <cuda_bf16.h>
 
@@ -85,9 +87,69 @@ cudaError_t launch(int P, dim3 grid, dim3 block, cudaStream_t s, const char *in0
     return cudaGetLastError();
 }
 
+// An all-gather of 64-bit words on the same primitives: exercises 8-byte elements (16-byte LL slots),
+// send / recv / reset one at a time, and a buffer that is not subdivided (round_robin = 0: one fixed
+// region per CTA, safe here because a launch is one epoch and a kernel boundary separates epochs).
+template <LLSync Mode, int P>
+__global__ void allgather_u64_kernel(const char *in0, char *out0, size_t io_stride, char *scratch0,
+                                     size_t scratch_stride, size_t nwords, uint64_t epoch, unsigned *fail)
+{
+    const int cta = blockIdx.x, ctas = gridDim.x, rank = blockIdx.y;
+    const size_t per_cta = (nwords + ctas - 1) / ctas;
+    // a region holds P rows of per_cta slots; with round_robin = 0 the object applies no offset, so the
+    // CTA's region is addressed through the slot index
+    LLBuffer<Mode> buf(scratch0, scratch_stride, rank, P, cta, ctas, 0, 0, epoch, 1u << 20);
+    const size_t region = (size_t)cta * P * per_cta;
+    const uint64_t *in = reinterpret_cast<const uint64_t *>(in0 + (size_t)rank * io_stride);
+    uint64_t *out      = reinterpret_cast<uint64_t *>(out0 + (size_t)rank * io_stride);
+    for (size_t k = threadIdx.x; k < per_cta; k += blockDim.x) {
+        const size_t i = (size_t)cta * per_cta + k;
+        if (i >= nwords) continue;
+        uint64_t w = in[i];
+        if (Mode == LLSync::Sentinel && w == ~0ull) w = ~1ull;
+        for (int q = 0; q < P; ++q) buf.template send<uint64_t>(q, region + (size_t)rank * per_cta + k, w);
+        for (int q = 0; q < P; ++q) {
+            uint64_t v;
+            if (!buf.template recv<uint64_t>(region + (size_t)q * per_cta + k, v)) {
+                atomicExch(fail, 1u);
+                return;
+            }
+            if (Mode == LLSync::Sentinel) buf.template reset<uint64_t>(region + (size_t)q * per_cta + k);
+            out[(size_t)q * nwords + i] = v;
+        }
+    }
+}
+
 }  // namespace
 
 extern "C" {
+
+// All-gather of nwords 64-bit words per rank: out[r] = in[0] | in[1] | ... | in[P-1] for every rank r.
+// Scratch per rank: symar_llbuffer_bytes(mode, 8, P * ceil(nwords / ctas), ctas, 0).  mode / epoch /
+// device_fail as for llbuffer_oneshot_allreduce; one epoch per launch.
+int llbuffer_allgather_u64(int mode, int P, const void *in0, void *out0, size_t io_stride, void *scratch0,
+                           size_t scratch_stride, size_t nwords, unsigned long long epoch, int ctas, int threads,
+                           unsigned *device_fail, void *cuda_stream)
+{
+    if (!in0 || !out0 || !scratch0 || !device_fail || ctas < 1 || threads < 1 || threads > 1024 || epoch == 0)
+        return -1;
+    const dim3 grid(ctas, P), block(threads);
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    const char *i0 = (const char *)in0;
+    char *o0 = (char *)out0, *s0 = (char *)scratch0;
+#define SYMAR_EX_LAUNCH(M, N) allgather_u64_kernel<M, N><<<grid, block, 0, s>>>(i0, o0, io_stride, s0, scratch_stride, nwords, epoch, device_fail)
+    if (mode == 0) {
+        if (P == 1) SYMAR_EX_LAUNCH(LLSync::LL, 1); else if (P == 2) SYMAR_EX_LAUNCH(LLSync::LL, 2);
+        else if (P == 4) SYMAR_EX_LAUNCH(LLSync::LL, 4); else if (P == 8) SYMAR_EX_LAUNCH(LLSync::LL, 8); else return -1;
+    } else if (mode == 1) {
+        if (P == 1) SYMAR_EX_LAUNCH(LLSync::Sentinel, 1); else if (P == 2) SYMAR_EX_LAUNCH(LLSync::Sentinel, 2);
+        else if (P == 4) SYMAR_EX_LAUNCH(LLSync::Sentinel, 4); else if (P == 8) SYMAR_EX_LAUNCH(LLSync::Sentinel, 8); else return -1;
+    } else {
+        return -1;
+    }
+#undef SYMAR_EX_LAUNCH
+    return cudaGetLastError() == cudaSuccess ? 0 : -3;
+}
 
 // mode 0 = LL, 1 = sentinel; bf16 0 = fp32 words, 1 = bf16 pairs.  in0 / out0 / scratch0 are rank 0's
 // device addresses, the strides the byte distance to the next rank's copy.  `epoch` is the first

@@ -26,6 +26,17 @@ def example():
     return fn
 
 
+@pytest.fixture(scope="module")
+def allgather():
+    lib = ctypes.CDLL(str(build.build_example()))
+    fn = lib.llbuffer_allgather_u64
+    fn.restype = ctypes.c_int
+    fn.argtypes = [ctypes.c_int, ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p,
+                   ctypes.c_size_t, ctypes.c_size_t, ctypes.c_ulonglong, ctypes.c_int, ctypes.c_int, ctypes.c_void_p,
+                   ctypes.c_void_p]
+    return fn
+
+
 class Rig:
     """Input, output and scratch of every rank inside one symmetric heap's user region."""
 
@@ -124,3 +135,40 @@ def test_size_helper_rejects_bad_arguments():
     assert symar.llbuffer_bytes(2, 4, 100, 3, 2) == 0
     assert symar.llbuffer_bytes(LL, 3, 100, 3, 2) == 0
     assert symar.llbuffer_bytes(LL, 4, 100, 0, 2) == 0
+
+
+@pytest.mark.parametrize("mode", [LL, SENTINEL])
+@pytest.mark.parametrize("P", [2, 8])
+def test_allgather_of_64_bit_words_on_the_primitives(allgather, mode, P):
+    # 8-byte elements (16-byte LL slots), send / recv / reset one at a time, an undivided buffer
+    ctas, nwords = 3, 1000
+    per_cta = (nwords + ctas - 1) // ctas
+    scratch = symar.llbuffer_bytes(mode, 8, P * per_cta, ctas, 0)
+    assert scratch == (2 if mode == LL else 1) * 8 * P * per_cta * ctas
+    io = 1 << 17
+    h = symar.SymHeap.on_torch(P, 2 * io + scratch)
+    fail = torch.zeros(1, dtype=torch.int32, device="cuda")
+    try:
+        stride = h.info().stride
+        for q in range(P):
+            if mode == SENTINEL:
+                symar.llbuffer_init_sentinel(h.rank_ptr(q, 2 * io), scratch)
+            else:
+                h.write_rank(q, 2 * io, np.zeros(scratch, dtype=np.uint8))
+        rng = np.random.default_rng(5)
+        for launch in range(3):                                  # the undivided region is reused every launch
+            x = rng.integers(0, 1 << 63, size=(P, nwords), dtype=np.uint64)
+            x[0, 7] = np.uint64(0xFFFFFFFFFFFFFFFF) if mode == LL else x[0, 7]      # all ones is fine for LL
+            for q in range(P):
+                h.write_rank(q, 0, x[q])
+            rc = allgather(mode, P, h.rank_ptr(0, 0), h.rank_ptr(0, io), stride, h.rank_ptr(0, 2 * io), stride, nwords,
+                           launch + 1, ctas, 128, fail.data_ptr(), 0)
+            assert rc == 0
+            torch.cuda.synchronize()
+            assert int(fail.item()) == 0
+            for q in range(P):
+                got = h.read_rank(q, io, P * nwords, np.uint64)
+                assert np.array_equal(got, x.reshape(-1)), (mode, P, launch, q)
+    finally:
+        torch.cuda.synchronize()
+        h.destroy()
