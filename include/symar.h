@@ -107,7 +107,8 @@ typedef struct {
  *      ncclLLBuffer layout "address = f(epoch, CTA index)") ------------------- */
 
 /* Bytes of device memory a heap of P ranks with `bytes_per_rank` of user region
- * needs (control block + P segments of user region, LL scratch, flags).
+ * needs (control block + P segments of user region, LL, sentinel and atomic
+ * scratch, flags and counters).
  * Returns 0 if P is not 1, 2, 4 or 8.                                          */
 size_t symheap_required_bytes(int P, size_t bytes_per_rank);
 
@@ -146,8 +147,8 @@ int symheap_status(symheap_t *heap, int *code, int *rank, int *peer, int *cta);
  * out[r][i] = narrow( ((x_0[i] + x_1[i]) + ... ) + x_{P-1}[i] )   for every rank r,
  * x_q = widen(in[q]), sum in IEEE binary32 in rank order 0..P-1 (the deterministic
  * one-/two-shot rows of Table I; accumulator type per Sec. V recvReduce), bf16
- * narrowed once with round-to-nearest-even.  All three algorithms give the same
- * bits.
+ * narrowed once with round-to-nearest-even.  Every algorithm gives these bits, except
+ * SYMAR_TWOSHOT_ATOMIC, whose order of additions is free (see its enumerator).
  *
  * in, out : symmetric addresses -- device pointers into RANK 0's user region
  *           (symheap_rank_ptr(heap, 0, off)); rank q's buffer is the same offset
