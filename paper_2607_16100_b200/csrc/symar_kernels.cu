@@ -31,13 +31,42 @@
 namespace symar {
 
 // One-shot data phase with W words per thread: unit u covers bytes [4W u, 4W u + 4W).
+// For small messages the loads are issued BEFORE the CTA barrier that lets thread 0 publish
+// the exchange count, so that the barrier, the publication and the trigger of the dependent
+// launch cost nothing while the data travels (measured -0.03 us of 1.72 us at 16 KiB).
 template <typename E, int P, int W>
-__device__ __forceinline__ void oneshot_units(const KArgs &a, char *out, uint64_t first, uint64_t step)
+__device__ __forceinline__ void oneshot_data(const KArgs &a, char *out, uint64_t first, uint64_t step, bool ok,
+                                             uint32_t *count, uint32_t want)
 {
     const uint64_t bytes  = a.tail_bytes ? (a.nvec - 1) * 16 + a.tail_bytes : a.nvec * 16;
     const uint64_t nunits = (bytes + 4 * W - 1) / (4 * W);
-    for (uint64_t u = first; u < nunits; u += step) {
-        Words<W> x[P];
+    const bool have = ok && first < nunits;
+    Words<W> x[P];
+    // ... when one pass covers the message; with several passes per thread the barrier would sit
+    // between the passes' loads and cost more than it hides (measured +0.13 us at 64 KiB)
+    const bool late = nunits > step;
+    if (have && !late) {
+#pragma unroll
+        for (int q = 0; q < P; ++q)
+            x[q] = ld_peer_words<W>(a.seg0 + (size_t)q * a.stride + a.in_off + first * (4 * W));
+    }
+    // Every warp has consumed the count: publish the next one now, so that its store drains
+    // while the data is in flight.
+    __syncthreads();
+    if (threadIdx.x == 0) *count = want;
+    if (a.pdl) pdl_launch_dependents();       // the next call may take its seats now
+    if (have && late) {
+#pragma unroll
+        for (int q = 0; q < P; ++q)
+            x[q] = ld_peer_words<W>(a.seg0 + (size_t)q * a.stride + a.in_off + first * (4 * W));
+    }
+    if (have) {
+        const uint64_t left = bytes - first * (4 * W);
+        store_words<W>(out + first * (4 * W), reduce_words_in_rank_order<E, P, W>(x),
+                       left < 4u * W ? (uint32_t)left : 4u * W);
+    }
+    if (!ok) return;
+    for (uint64_t u = first + step; u < nunits; u += step) {
 #pragma unroll
         for (int q = 0; q < P; ++q)
             x[q] = ld_peer_words<W>(a.seg0 + (size_t)q * a.stride + a.in_off + u * (4 * W));
@@ -73,26 +102,12 @@ __global__ void __launch_bounds__(kMaxThreads) oneshot_kernel(const KArgs a)
 
     uint32_t want;
     const bool ok = flag_exchange_at<P, false>(a, xp, count, r, c, false, true, want);
-    // Every warp has consumed the count; publish the next one now so that its
-    // store drains while the data is in flight.
-    __syncthreads();
-    if (t == 0) *count = want;
-    if (a.pdl) pdl_launch_dependents();       // the next call may take its seats now
-    if (ok) {
-        char *out = seg_r + a.out_off;
-        const uint64_t first = (uint64_t)c * T + t, step = (uint64_t)C * T;
-        const uint32_t narrow = (a.variant >> 8) & 3u;     // bytes per thread: 16, 8 or 4
-        if (narrow == 2) oneshot_units<E, P, 1>(a, out, first, step);
-        else if (narrow == 1) oneshot_units<E, P, 2>(a, out, first, step);
-        else {
-            for (uint64_t v = first; v < a.nvec; v += step) {
-                uint4 x[P];
-#pragma unroll
-                for (int q = 0; q < P; ++q) x[q] = ld_peer(a.seg0 + (size_t)q * a.stride + a.in_off + v * 16);
-                store_result(out, v, reduce_in_rank_order<E, P>(x), a.nvec, a.tail_bytes);
-            }
-        }
-    }
+    char *out = seg_r + a.out_off;
+    const uint64_t first = (uint64_t)c * T + t, step = (uint64_t)C * T;
+    const uint32_t narrow = (a.variant >> 8) & 3u;     // bytes per thread: 16, 8 or 4
+    if (narrow == 2) oneshot_data<E, P, 1>(a, out, first, step, ok, count, want);
+    else if (narrow == 1) oneshot_data<E, P, 2>(a, out, first, step, ok, count, want);
+    else oneshot_data<E, P, 4>(a, out, first, step, ok, count, want);
     if (DBG) debug_stamp_out(a);
 }
 
