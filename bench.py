@@ -233,6 +233,14 @@ def latency_suite(torch, symar, synth, hbm_gbs, quick=False, autotune=True):
     out["flag_round_trip_pairs"] = {"min_us": rts[0] if rts else None, "median_us": rt_ns / 1000.0,
                                     "max_us": rts[-1] if rts else None, "pairs": pairs}
 
+    # the barrier that the method removes (Sec. III-B), for context: P CTAs, all signal all, all wait for all
+    try:
+        out["barrier_us"] = {f"P{p_}": {"relaxed": symar.probe_barrier(p_, 3000, False) / 1e3,
+                                         "release_acquire": symar.probe_barrier(p_, 3000, True) / 1e3}
+                             for p_ in (2, 4, 8)}
+    except symar.SymarError as exc:
+        out["barrier_us"] = {"error": str(exc)}
+
     def empty_floor(cx, py, T, pdl=True):
         probe = symar.probe_empty_pdl if pdl else symar.probe_empty
         g = graph_of(torch, stream, lambda k, s: probe(cx, py, T, s), K)

@@ -365,6 +365,13 @@ int symar_probe_pingpong_pair(int iterations, int partner_block, double *host_ns
 int symar_probe_pingpong_blocks(int iterations, int first_block, int partner_block, int grid_blocks,
                                 double *host_ns_per_round_trip, int *host_smids);
 
+/* The barrier the method removes (Sec. III-B: "each barrier will incur more than 1 us"): `ranks`
+ * CTAs (2..32, one per rank, all co-resident) signal every peer and wait for every peer,
+ * `iterations` times in a row; *host_ns_per_barrier is the mean as seen by rank 0.  ordered = 0:
+ * relaxed signals and polls, as the paper measured; 1: release signals and acquire polls (a
+ * barrier that also orders memory).  Synchronous; bounded spins (SYMAR_ERR_TIMEOUT).            */
+int symar_probe_barrier(int ranks, int iterations, int ordered, double *host_ns_per_barrier);
+
 /* ---- host side of the thread-level buffer primitives (symar_llbuffer.cuh; Sec. V
  *      "Host-side Functions": a scratch-size helper and the sentinel initialiser) ---- */
 

@@ -88,6 +88,43 @@ __global__ void pingpong_kernel(unsigned *flags, int iters, unsigned long long *
     if (dead) out[1] = 1;
 }
 
+// The barrier the method removes (paper Sec. III-B): every rank signals every peer and waits
+// for every peer, `iters` times in a row.  One CTA per rank, lane q of warp 0 talks to peer q;
+// flags[rank][peer] counts the barriers that `peer` has entered.  mode 0: relaxed signals (the
+// paper's measurement); mode 1: release signals + acquire polls (a barrier that orders memory).
+// out[0] = ns over all iterations as seen by rank 0, out[1] = 1 on timeout.
+__global__ void barrier_kernel(unsigned *flags, int iters, int mode, unsigned long long *out)
+{
+    const int P = gridDim.x, r = blockIdx.x;
+    const unsigned lane = threadIdx.x;
+    if (lane >= 32) return;
+    unsigned *sig        = flags + (size_t)(lane < (unsigned)P ? lane : 0) * 32 + r;    // my word in peer `lane`'s row
+    const unsigned *mine = flags + (size_t)r * 32 + (lane < (unsigned)P ? lane : 0);   // peer `lane`'s word in my row
+    bool dead = false;
+    unsigned long long t0 = 0;
+    for (int i = 1; i <= iters + 1 && !dead; ++i) {
+        if (i == 2) t0 = timer_ns();                    // the first barrier only lines the CTAs up
+        if (lane < (unsigned)P) {
+            if (mode == 1) asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(sig) : "memory");
+            else asm volatile("red.relaxed.gpu.global.add.u32 [%0], 1;" ::"l"(sig) : "memory");
+        }
+        unsigned n = 0;
+        for (;;) {
+            unsigned f;
+            if (mode == 1) asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(f) : "l"(mine) : "memory");
+            else f = ld_relaxed(mine);
+            if (__ballot_sync(0xffffffffu, lane < (unsigned)P && (int)(f - (unsigned)i) < 0) == 0) break;
+            if (++n > kSpinLimit) { dead = true; break; }
+        }
+    }
+    if (r == 0 && lane == 0) {
+        out[0] = timer_ns() - t0;
+        out[1] = dead ? 1 : 0;
+    } else if (dead && lane == 0) {
+        out[1] = 1;
+    }
+}
+
 int sync_and_fetch(unsigned long long *dev, unsigned long long *host, int n)
 {
     if (cudaDeviceSynchronize() != cudaSuccess) return SYMAR_ERR_CUDA;
@@ -135,6 +172,23 @@ int symar_probe_fence(int iterations, double *host_ns_per_fence)
     cudaFree(buf);
     if (rc != SYMAR_OK) return rc;
     *host_ns_per_fence = (double)h[0] / iterations;
+    return SYMAR_OK;
+}
+
+int symar_probe_barrier(int ranks, int iterations, int ordered, double *host_ns_per_barrier)
+{
+    if (ranks < 2 || ranks > 32 || iterations < 1 || !host_ns_per_barrier) return SYMAR_ERR_INVAL;
+    unsigned char *buf = nullptr;
+    const size_t flag_bytes = 32 * 32 * sizeof(unsigned);                   // one 128-byte row per rank
+    if (cudaMalloc(&buf, flag_bytes + 256) != cudaSuccess) return SYMAR_ERR_NOMEM;
+    cudaMemset(buf, 0, flag_bytes + 256);
+    unsigned long long h[2] = {0, 0};
+    barrier_kernel<<<ranks, 32>>>((unsigned *)buf, iterations, ordered ? 1 : 0, (unsigned long long *)(buf + flag_bytes));
+    int rc = sync_and_fetch((unsigned long long *)(buf + flag_bytes), h, 2);
+    cudaFree(buf);
+    if (rc != SYMAR_OK) return rc;
+    if (h[1] != 0) return SYMAR_ERR_TIMEOUT;
+    *host_ns_per_barrier = (double)h[0] / iterations;
     return SYMAR_OK;
 }
 

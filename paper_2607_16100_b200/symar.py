@@ -68,6 +68,7 @@ SIGNATURES = [
     ("symar_probe_pingpong", c_int, [c_int, POINTER(c_double)]),
     ("symar_probe_pingpong_pair", c_int, [c_int, c_int, POINTER(c_double), POINTER(c_int)]),
     ("symar_debug_span", c_int, [c_void_p, c_void_p, c_void_p, c_size_t, c_int, c_int, c_void_p, POINTER(c_double)]),
+    ("symar_probe_barrier", c_int, [c_int, c_int, c_int, POINTER(c_double)]),
     ("symar_llbuffer_bytes", c_size_t, [c_int, c_size_t, c_size_t, c_int, c_int]),
     ("symar_llbuffer_init_sentinel", c_int, [c_void_p, c_size_t, c_void_p]),
     ("symar_probe_pingpong_blocks", c_int, [c_int, c_int, c_int, c_int, POINTER(c_double), POINTER(c_int)]),
@@ -354,6 +355,13 @@ def llbuffer_bytes(sync_mode: int, elem_bytes: int, slots_per_cta: int, ctas: in
 
 def llbuffer_init_sentinel(device_ptr: int, nbytes: int, stream: int = 0) -> None:
     _ck(load().symar_llbuffer_init_sentinel(device_ptr, nbytes, stream), "symar_llbuffer_init_sentinel")
+
+
+def probe_barrier(ranks: int, iterations: int = 5000, ordered: bool = False) -> float:
+    """ns per all-to-all flag barrier among `ranks` CTAs (the barrier the method removes)."""
+    v = c_double()
+    _ck(load().symar_probe_barrier(ranks, iterations, 1 if ordered else 0, byref(v)), "symar_probe_barrier")
+    return v.value
 
 
 def probe_pingpong_blocks(first_block: int, partner_block: int, grid_blocks: int, iterations: int = 20000):

@@ -159,6 +159,10 @@ def test_speed_of_light_probes_return_plausible_values():
         symar.probe_pingpong_blocks(5, 5, nsm, 100)              # a block cannot play against itself
     with pytest.raises(symar.SymarError):
         symar.probe_pingpong_blocks(0, nsm, nsm, 100)            # partner outside the launch
+    for ordered in (False, True):
+        assert 50.0 < symar.probe_barrier(8, 500, ordered) < 20_000.0
+    with pytest.raises(symar.SymarError):
+        symar.probe_barrier(1, 10)
     s = torch.cuda.Stream()
     symar.probe_empty(4, 8, 128, s.cuda_stream)
     symar.probe_empty_pdl(4, 8, 128, s.cuda_stream)
