@@ -285,6 +285,17 @@ def latency_suite(torch, symar, synth, hbm_gbs, quick=False, autotune=True):
                 row[names[algo]] = r
             return row
 
+        def prior_art_row():
+            """The same one-shot kernel with the two memory-ordering barriers of the prior-art form (Sec. III-B)."""
+            a_, c_, t_ = h.query_choice(8192, symar.BF16, symar.ONESHOT)
+            h.set_launch(symar.ONESHOT, c_, t_)
+            h.set_variant(symar.ONESHOT, 0x4000 | 0x100)
+            r_ = bench_size(8192, (symar.ONESHOT,))["oneshot"]
+            h.set_variant(symar.ONESHOT, 0)
+            h.set_launch(symar.ONESHOT, 0, 0)
+            return {"p50_us": r_["p50"], "bit_exact": r_["bit_exact"], "ctas_per_rank": r_["ctas_per_rank"],
+                    "threads": r_["threads"], "note": "8 bytes per thread; release signals + a second barrier before exit"}
+
         # C2: 16 KiB per rank
         if P == 8:
             row = bench_size(8192, ALL, stream_too=True)
@@ -299,6 +310,7 @@ def latency_suite(torch, symar, synth, hbm_gbs, quick=False, autotune=True):
                            "numerator and denominator use the same harness",
                 "p50_us": best["p50"], "best": best, "per_algo": row,
                 "twoshot_atomic_not_bit_reproducible": bench_size(8192, (symar.TWOSHOT_ATOMIC,))["twoshot_atomic"],
+                "prior_art_two_barrier_oneshot": prior_art_row(),
                 "in_kernel_span_us_p50": {
                     names[a_]: float(np.median([h.debug_span(0, out_off, 8192, symar.BF16, a_) for _ in range(31)])) / 1e3
                     for a_ in (symar.ONESHOT, symar.TWOSHOT, symar.LL, symar.SENTINEL)},

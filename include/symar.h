@@ -252,7 +252,8 @@ int symar_set_launch(symheap_t *heap, symar_algo_t algo, int ctas_per_rank, int 
 /* Implementation variant of one algorithm's kernel, for performance experiments;
  * every variant computes the same bits.  0 = back to the table/default choice;
  * bit 31 alone forces the plain variant (all other bits 0).  One-shot: bits 8-9 = bytes
- * per thread (0: 16, 1: 8, 2: 4); LL: bit 8 = 8 instead of 16 payload bytes per thread;
+ * per thread (0: 16, 1: 8, 2: 4), bit 14 = the prior-art form with a memory-ordering barrier
+ * before the data phase and another before returning (what Sec. III-B removes; for comparison); LL: bit 8 = 8 instead of 16 payload bytes per thread;
  * two-shot: bit 0 = contiguous chunks also for large messages (no block-cyclic
  * ownership), bit 1 = 16-byte instead of 32-byte accesses for large messages,
  * bit 2 = never use the bulk-copy kernel, bits 8-10 = its pipeline depth (0:

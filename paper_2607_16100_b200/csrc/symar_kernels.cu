@@ -100,14 +100,26 @@ __global__ void __launch_bounds__(kMaxThreads) oneshot_kernel(const KArgs a)
     if (DBG) debug_delay(a, r, c);
     if (DBG && a.dbg_mute == r) return;       // test hook: this rank never joins
 
+    // Variant bit 14: the prior-art form that the method replaces (Sec. III-B), for comparison only --
+    // a memory-ordering barrier before the data phase (release signals) and a second one before
+    // returning, as a pull kernel needs when nothing else keeps inputs from being overwritten.
+    const bool prior_art = a.variant & 0x4000u;
     uint32_t want;
-    const bool ok = flag_exchange_at<P, false>(a, xp, count, r, c, false, true, want);
+    const bool ok = prior_art ? flag_exchange_at<P, true>(a, xp, count, r, c, false, true, want)
+                              : flag_exchange_at<P, false>(a, xp, count, r, c, false, true, want);
     char *out = seg_r + a.out_off;
     const uint64_t first = (uint64_t)c * T + t, step = (uint64_t)C * T;
     const uint32_t narrow = (a.variant >> 8) & 3u;     // bytes per thread: 16, 8 or 4
     if (narrow == 2) oneshot_data<E, P, 1>(a, out, first, step, ok, count, want);
     else if (narrow == 1) oneshot_data<E, P, 2>(a, out, first, step, ok, count, want);
     else oneshot_data<E, P, 4>(a, out, first, step, ok, count, want);
+    if (prior_art) {
+        uint32_t *dcount = reinterpret_cast<uint32_t *>(seg_r + a.epoch_off + done_count_off(c));
+        uint32_t dwant;
+        __syncthreads();
+        flag_exchange<P, true>(a, a.done_off, dcount, r, c, !ok, false, dwant);
+        if (t == 0) *dcount = dwant;
+    }
     if (DBG) debug_stamp_out(a);
 }
 

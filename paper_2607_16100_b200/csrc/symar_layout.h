@@ -39,7 +39,8 @@ __host__ __device__ constexpr size_t ready_count_off(int c) { return (size_t)kMa
 __host__ __device__ constexpr size_t done_count_off(int c) { return (size_t)kMaxCtas * 12 + (size_t)c * 4; }
 
 // Variant bits carried in KArgs::variant (every variant computes the same bits):
-//   one-shot : bits 8-9 = bytes per thread (0: 16, 1: 8, 2: 4)
+//   one-shot : bits 8-9 = bytes per thread (0: 16, 1: 8, 2: 4); bit 14 = prior-art form with two
+//              memory-ordering barriers (comparison only, never chosen)
 //   LL       : bit 8    = 8 instead of 16 payload bytes per thread
 //   two-shot : bit 0 = contiguous chunks for large messages, bit 1 = 16-byte accesses,
 //              bit 2 = never the bulk-copy kernel, bits 8-10 = bulk pipeline depth,

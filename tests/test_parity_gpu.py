@@ -622,3 +622,18 @@ def test_library_owned_heap():
         assert h.rank_ptr(1, 0) - h.rank_ptr(0, 0) == info.stride
     finally:
         h.destroy()
+
+
+def test_prior_art_two_barrier_oneshot_gives_the_same_bits(heaps):
+    # variant bit 14: the barrier-based form the method replaces, kept for comparison in the bench
+    h = heaps[8]
+    x = synth.make_inputs("normal", "bf16", 8, 8192, seed=14)
+    try:
+        for var in (0x4000, 0x4100, 0x4200):
+            h.set_variant(symar.ONESHOT, var)
+            for _ in range(3):
+                assert_bits(run(h, x, symar.BF16, symar.ONESHOT, poison=False), O.allreduce(x), hex(var))
+        h.set_variant(symar.ONESHOT, 0)
+        assert_bits(run(h, x, symar.BF16, symar.TWOSHOT), O.allreduce(x))      # shares the done flags
+    finally:
+        h.set_variant(symar.ONESHOT, 0)
