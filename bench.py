@@ -254,6 +254,20 @@ def latency_suite(torch, symar, synth, hbm_gbs, quick=False, autotune=True):
         tune_s = time.time() - t0
         out_off = 12 << 20
         res = {"autotune_seconds": tune_s}
+        if autotune:
+            # what the tuner measured (graphs of back-to-back calls, warm): per size the time of every
+            # bit-reproducible algorithm at its best shape -- the selector's whole landscape
+            table = []
+            for log2 in range(5, 24):
+                us = {}
+                for a_ in (symar.ONESHOT, symar.TWOSHOT, symar.LL, symar.SENTINEL, symar.TWOSHOT_LL,
+                           symar.TWOSHOT_SENTINEL):
+                    e_ = h.tuned_entry(symar.BF16, log2, a_)
+                    if e_ and e_[0] > 0 and e_[2] < 1e29:
+                        us[names[a_]] = round(e_[2], 3)
+                if us:
+                    table.append({"bytes_per_rank": 1 << log2, "us": us, "best": min(us, key=us.get)})
+            out.setdefault("tuner_table_bf16", {})[f"P{P}"] = table
 
         def bench_size(count, algos, stream_too=False):
             x = synth.make_inputs("normal", "bf16", P, count, synth.seed_for_config(2))
