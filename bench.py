@@ -1,19 +1,23 @@
 #!/usr/bin/env python
 """Benchmark of the barrier-free symmetric-memory AllReduce on B200.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--out-dir DIR]
 
-One JSON line on stdout (rank 0).  A "step" is one AllReduce of the bandwidth
-workload: P = 8 emulated ranks, fp32, 64 Mi elements (256 MiB) per rank,
-inputs U(-1, 1), two-shot algorithm.  `value` is algorithmic bytes (every input
-byte read once + every output byte written once = 2 P M) per second with the
-inputs resident in HBM.  The latency half of the metric (P = 8, bf16, 16 KiB per
-rank, p50 against the speed-of-light bound measured in the same process), the
-16 KiB..1 MiB sweep with the selector's choice and the 160-call decode-step
-graph ride along in the same line under `latency_16KB`, `sweep`, `decode_trace`.
+ONE short JSON line on stdout (rank 0), fewer than 2000 characters.  A "step" is one AllReduce of
+the bandwidth workload: P = 8 emulated ranks, fp32, 64 Mi elements (256 MiB) per rank, inputs
+U(-1, 1), two-shot algorithm.  `value` is algorithmic bytes (every input byte read once + every
+output byte written once = 2 P M) per second with the inputs resident in HBM.  The latency half of
+the metric (P = 8, bf16, 16 KiB per rank, p50 against the speed-of-light bound measured in the same
+process) and the 160-call decode-step graph ride in the same line as a handful of numbers under
+`latency_16KB` and `decode_trace`.
 
-N > 1 runs N independent replicas (one process and one heap per GPU; the path
-itself is a single-GPU emulation and has no exchange between GPUs).
+Everything else -- per-algorithm rows, the 16 KiB..1 MiB sweep with the selector's choice, the
+sampled flag round trips, phase stamps, the tuner's table, the context measurements -- goes to one
+file per workload in DIR (default gpurun_out/): results_c2.json, results_c3.json, results_c4.json,
+results_c5.json.  The line names them under `details`.
+
+N > 1 runs N independent replicas (one process and one heap per GPU; the path itself is a
+single-GPU emulation and has no exchange between GPUs).
 """
 from __future__ import annotations
 
@@ -196,23 +200,11 @@ def time_stream(torch, stream, enqueue, n, warm=50):
     return float(np.percentile(us, 50))
 
 
-def latency_suite(torch, symar, synth, hbm_gbs, quick=False, autotune=True):
-    """C2 (16 KiB vs SoL), C3 (sweep + selector), C5 (decode-step graph)."""
-    from oracle import allreduce_oracle as O
-    out = {}
-    stream = torch.cuda.Stream()
-    K, reps = 64, (60 if quick else 300)
-    names = dict(symar.ALGO_NAMES)
-    ALL = (symar.ONESHOT, symar.TWOSHOT, symar.LL, symar.SENTINEL, symar.TWOSHOT_LL, symar.TWOSHOT_SENTINEL,
-           symar.AUTO)
-
-    # speed-of-light parts (paper Sec. VI), measured here
-    fence_ns = symar.probe_fence(20000)
-    # The flag round trip depends on which SMs the two CTAs sit on (measured: mostly on
-    # the one that sends first; 0.5-0.7 us from some SMs, 0.9-1.1 us from others), and the
-    # ranks of the AllReduce are spread over the whole chip.  Sample pairs with both ends
-    # spread over a one-CTA-per-SM launch and use the median pair for the bound (min and
-    # max are reported).
+def sample_flag_round_trips(torch, symar):
+    """The flag round trip depends on which SMs the two CTAs sit on (measured: mostly on the one
+    that sends first; 0.5-0.7 us from some SMs, 0.9-1.1 us from others), and the ranks of the
+    AllReduce are spread over the whole chip.  Sample pairs with both ends spread over a
+    one-CTA-per-SM launch; the bound uses the median pair, min and max are reported."""
     pairs = []
     nsm = torch.cuda.get_device_properties(0).multi_processor_count
     firsts = [int(round(i * (nsm - 1) / 11)) for i in range(12)]
@@ -228,10 +220,95 @@ def latency_suite(torch, symar, synth, hbm_gbs, quick=False, autotune=True):
             except symar.SymarError:
                 pass
     rts = sorted(p["round_trip_us"] for p in pairs)
-    rt_ns = 1000.0 * (rts[len(rts) // 2] if rts else float("nan"))
-    rt_min_ns = 1000.0 * (rts[0] if rts else float("nan"))
-    out["flag_round_trip_pairs"] = {"min_us": rts[0] if rts else None, "median_us": rt_ns / 1000.0,
-                                    "max_us": rts[-1] if rts else None, "pairs": pairs}
+    nan = float("nan")
+    return {"min_us": rts[0] if rts else nan, "median_us": rts[len(rts) // 2] if rts else nan,
+            "max_us": rts[-1] if rts else nan, "pairs": pairs}
+
+
+def spread(values):
+    v = [x for x in values if x == x]
+    if not v:
+        return {"median": None, "min": None, "max": None, "n": 0}
+    return {"median": float(np.median(v)), "min": float(min(v)), "max": float(max(v)), "n": len(v)}
+
+
+def oracle_us(O, x):
+    """The CPU oracle on one message, in microseconds: single thread and all host cores (best of 5)."""
+    one = all_ = 1e30
+    team = 1
+    for _ in range(5):
+        t0 = time.perf_counter()
+        O.allreduce_timed_team(x, threads=1)
+        one = min(one, time.perf_counter() - t0)
+        t0 = time.perf_counter()
+        _, team = O.allreduce_timed_team(x, threads=0)
+        all_ = min(all_, time.perf_counter() - t0)
+    return {"single_thread_us": one * 1e6, "all_cores_us": all_ * 1e6, "cores": team}
+
+
+def sys_scope_numbers(shapes, quick):
+    """16 KiB one-shot and LL from the build whose flags, signals and data+flag accesses are at
+    system scope (what an NVLink domain needs), in a child process that loads that library."""
+    try:
+        from paper_2607_16100_b200 import build as B
+        lib = B.build_lib_sys()
+        env = dict(os.environ, SYMAR_LIB=str(lib))
+        r = subprocess.run([sys.executable, str(ROOT / "bench.py"), "--scope-probe", json.dumps(shapes)] +
+                           (["--quick"] if quick else []), capture_output=True, text=True, env=env, timeout=300)
+        if r.returncode != 0:
+            return {"error": (r.stderr or r.stdout)[-300:]}
+        return json.loads(r.stdout.strip().splitlines()[-1])
+    except Exception as exc:
+        return {"error": f"{type(exc).__name__}: {exc}"}
+
+
+def scope_probe(shapes_json, quick):
+    """Child of sys_scope_numbers(): times the given (algorithm, variant, shape) rows at 16 KiB, P = 8."""
+    import torch
+    from oracle import allreduce_oracle as O
+    from paper_2607_16100_b200 import symar, synth
+    shapes = json.loads(shapes_json)
+    stream = torch.cuda.Stream()
+    P, count, out_off = 8, 8192, 1 << 20
+    h = symar.SymHeap.on_torch(P, 2 << 20)
+    x = synth.make_inputs("normal", "bf16", P, count, synth.seed_for_config(2))
+    for q in range(P):
+        h.write_rank(q, 0, x[q])
+    want = O.allreduce(x)
+    out = {"library": str(symar.LIB_PATH.name)}
+    for name, (algo, variant, ctas, threads) in shapes.items():
+        h.set_variant(algo, variant if variant else 1 << 31)
+        h.set_launch(algo, ctas, threads)
+        enq = lambda k, s: h.allreduce(0, out_off, count, symar.BF16, algo, s)
+        enq(0, stream.cuda_stream)
+        stream.synchronize()
+        got = np.stack([h.read_rank(q, out_off, count, np.uint16) for q in range(P)])
+        g = graph_of(torch, stream, enq, 64)
+        r = time_graph(torch, g, stream, 64, 60 if quick else 200)
+        out[name] = {"p50_us": r["p50"], "bit_exact": bool(np.array_equal(got, want)) and h.status()[0] == 0}
+        h.set_variant(algo, 0)
+        h.set_launch(algo, 0, 0)
+    h.destroy()
+    print(json.dumps(out))
+
+
+def latency_suite(torch, symar, synth, hbm_gbs, quick=False, autotune=True):
+    """C2 (16 KiB vs SoL), C3 (sweep + selector), C5 (decode-step graph)."""
+    from oracle import allreduce_oracle as O
+    out = {}
+    stream = torch.cuda.Stream()
+    K, reps = 64, (60 if quick else 300)
+    REPEATS = 3 if quick else 5
+    names = dict(symar.ALGO_NAMES)
+    ALL = (symar.ONESHOT, symar.TWOSHOT, symar.LL, symar.SENTINEL, symar.TWOSHOT_LL, symar.TWOSHOT_SENTINEL,
+           symar.AUTO)
+
+    # speed-of-light parts (paper Sec. VI), measured here
+    fence_ns = symar.probe_fence(20000)
+    rt0 = sample_flag_round_trips(torch, symar)
+    rt_ns, rt_min_ns = 1000.0 * rt0["median_us"], 1000.0 * rt0["min_us"]
+    out["flag_round_trip_pairs"] = rt0
+    bytes_us = lambda nbytes, P_: 2 * P_ * nbytes / (hbm_gbs * 1e9) * 1e6      # "bytes at peak": the measured copy rate
 
     # the barrier that the method removes (Sec. III-B), for context: P CTAs, all signal all, all wait for all
     try:
@@ -241,10 +318,10 @@ def latency_suite(torch, symar, synth, hbm_gbs, quick=False, autotune=True):
     except symar.SymarError as exc:
         out["barrier_us"] = {"error": str(exc)}
 
-    def empty_floor(cx, py, T, pdl=True):
+    def empty_floor(cx, py, T, pdl=True, n=None):
         probe = symar.probe_empty_pdl if pdl else symar.probe_empty
         g = graph_of(torch, stream, lambda k, s: probe(cx, py, T, s), K)
-        return time_graph(torch, g, stream, K, reps)
+        return time_graph(torch, g, stream, K, n or reps)
 
     for P in (8, 4):
         h = symar.SymHeap.on_torch(P, 24 << 20)
@@ -269,10 +346,14 @@ def latency_suite(torch, symar, synth, hbm_gbs, quick=False, autotune=True):
                     table.append({"bytes_per_rank": 1 << log2, "us": us, "best": min(us, key=us.get)})
             out.setdefault("tuner_table_bf16", {})[f"P{P}"] = table
 
-        def bench_size(count, algos, stream_too=False):
+        def load_inputs(count):
             x = synth.make_inputs("normal", "bf16", P, count, synth.seed_for_config(2))
             for q in range(P):
                 h.write_rank(q, 0, x[q])
+            return x
+
+        def bench_size(count, algos, stream_too=False, n=None):
+            x = load_inputs(count)
             want = O.allreduce(x)
             row = {}
             for algo in algos:
@@ -283,8 +364,9 @@ def latency_suite(torch, symar, synth, hbm_gbs, quick=False, autotune=True):
                 got = np.stack([h.read_rank(q, out_off, count, np.uint16) for q in range(P)])
                 exact = bool(np.array_equal(got, want)) and h.status()[0] == 0
                 g = graph_of(torch, stream, enq, K)
-                r = time_graph(torch, g, stream, K, reps)
-                r.update({"algo": names[a], "ctas_per_rank": c, "threads": t, "bit_exact": exact})
+                r = time_graph(torch, g, stream, K, n or reps)
+                r.update({"algo": names[a], "ctas_per_rank": c, "threads": t, "variant": h.last_kernel()[0],
+                          "bit_exact": exact})
                 if algo == symar.TWOSHOT_ATOMIC:
                     # order of the atomic adds is free: all ranks identical, values within one bf16 ulp
                     # of the oracle plus 1e-6 * sum|x| (bit_exact is reported as seen, not required)
@@ -299,16 +381,15 @@ def latency_suite(torch, symar, synth, hbm_gbs, quick=False, autotune=True):
                 row[names[algo]] = r
             return row
 
-        def prior_art_row():
-            """The same one-shot kernel with the two memory-ordering barriers of the prior-art form (Sec. III-B)."""
-            a_, c_, t_ = h.query_choice(8192, symar.BF16, symar.ONESHOT)
-            h.set_launch(symar.ONESHOT, c_, t_)
-            h.set_variant(symar.ONESHOT, 0x4000 | 0x100)
-            r_ = bench_size(8192, (symar.ONESHOT,))["oneshot"]
-            h.set_variant(symar.ONESHOT, 0)
-            h.set_launch(symar.ONESHOT, 0, 0)
-            return {"p50_us": r_["p50"], "bit_exact": r_["bit_exact"], "ctas_per_rank": r_["ctas_per_rank"],
-                    "threads": r_["threads"], "note": "8 bytes per thread; release signals + a second barrier before exit"}
+        def with_variant(algo, variant, ctas, threads, count=8192):
+            """One row of `algo` with the given variant bits and launch shape."""
+            h.set_launch(algo, ctas, threads)
+            h.set_variant(algo, variant if variant else 1 << 31)
+            try:
+                return bench_size(count, (algo,))[names[algo]]
+            finally:
+                h.set_variant(algo, 0)
+                h.set_launch(algo, 0, 0)
 
         # C2: 16 KiB per rank
         if P == 8:
@@ -316,21 +397,65 @@ def latency_suite(torch, symar, synth, hbm_gbs, quick=False, autotune=True):
             best = min(row.values(), key=lambda r: r["p50"])
             floor = empty_floor(best["ctas_per_rank"], P, best["threads"])
             floor11 = empty_floor(1, 1, 1)
-            t_bytes_us = 2 * P * 16384 / (hbm_gbs * 1e9) * 1e6
+            t_bytes_us = bytes_us(16384, P)
             sol = floor["p50"] + rt_ns / 1000.0 + t_bytes_us
+            # the whole comparison again, bound and kernel interleaved in this process, REPEATS times
+            rep_rows = []
+            for _ in range(REPEATS):
+                rt_i = sample_flag_round_trips(torch, symar)
+                fl_i = empty_floor(best["ctas_per_rank"], P, best["threads"])["p50"]
+                p_i = bench_size(8192, (symar.AUTO,))["auto"]["p50"]
+                sol_i = fl_i + rt_i["median_us"] + t_bytes_us
+                rep_rows.append({"p50_us": p_i, "empty_launch_us": fl_i, "flag_round_trip_median_us": rt_i["median_us"],
+                                 "flag_round_trip_min_us": rt_i["min_us"], "sol_us": sol_i, "ratio_to_sol": p_i / sol_i,
+                                 "ratio_to_sol_fastest_pair": p_i / (fl_i + rt_i["min_us"] + t_bytes_us)})
+            o_a, o_c, o_t = h.query_choice(8192, symar.BF16, symar.ONESHOT)
+            o_var = row["oneshot"]["variant"]
+            release = with_variant(symar.ONESHOT, o_var | 0x8000, o_c, o_t)
+            prior = with_variant(symar.ONESHOT, 0x4000 | 0x100, o_c, o_t)
+            phases = {}
+            for a_ in (symar.ONESHOT, symar.LL, symar.TWOSHOT):
+                try:
+                    load_inputs(8192)
+                    ph = [h.debug_phases(0, out_off, 8192, symar.BF16, a_) for _ in range(31)]
+                    phases[names[a_]] = {str(k): {f: float(np.median([p_[k][f] for p_ in ph])) / 1e3
+                                                  for f in ("first", "mean", "last")} for k in sorted(ph[0])}
+                except symar.SymarError as exc:
+                    phases[names[a_]] = {"error": str(exc)}
+            l_var = row["ll"]["variant"]
+            sys_scope = sys_scope_numbers(
+                {"oneshot": [symar.ONESHOT, o_var, o_c, o_t],
+                 "oneshot_release_signal": [symar.ONESHOT, o_var | 0x8000, o_c, o_t],
+                 "ll": [symar.LL, l_var, row["ll"]["ctas_per_rank"], row["ll"]["threads"]]}, quick)
             out["latency_16KB"] = {
                 "workload": "c2: P=8, bf16, 8192 elements (16 KiB) per rank, N(0,1); buffers L2-resident (warm)",
                 "harness": f"{K} back-to-back calls in one CUDA graph, one replay = one sample, {reps} samples; "
                            "numerator and denominator use the same harness",
                 "p50_us": best["p50"], "best": best, "per_algo": row,
+                "repeats": rep_rows,
+                "ratio_to_sol_over_repeats": spread([r_["ratio_to_sol"] for r_ in rep_rows]),
+                "p50_us_over_repeats": spread([r_["p50_us"] for r_ in rep_rows]),
                 "twoshot_atomic_not_bit_reproducible": bench_size(8192, (symar.TWOSHOT_ATOMIC,))["twoshot_atomic"],
-                "prior_art_two_barrier_oneshot": prior_art_row(),
+                "prior_art_two_barrier_oneshot": {
+                    "p50_us": prior["p50"], "bit_exact": prior["bit_exact"], "ctas_per_rank": prior["ctas_per_rank"],
+                    "threads": prior["threads"],
+                    "note": "8 bytes per thread; release signals + a second barrier before exit"},
+                "oneshot_release_signal": {
+                    "p50_us": release["p50"], "bit_exact": release["bit_exact"], "ctas_per_rank": release["ctas_per_rank"],
+                    "threads": release["threads"], "ratio_to_sol": release["p50"] / sol,
+                    "note": "the selector's one-shot with red.release on the ready signal and nothing else changed: "
+                            "the form a system needs whose ranks do not share a kernel boundary"},
+                "system_scope_build": sys_scope,
                 "in_kernel_span_us_p50": {
                     names[a_]: float(np.median([h.debug_span(0, out_off, 8192, symar.BF16, a_) for _ in range(31)])) / 1e3
                     for a_ in (symar.ONESHOT, symar.TWOSHOT, symar.LL, symar.SENTINEL)},
                 "in_kernel_span_note": "first CTA in (after its wait for the previous grid) -> last CTA out, device "
                                        "nanosecond timer (about 32 ns resolution), single stream-launched calls "
                                        "through the instrumented instantiation of the same kernels",
+                "phase_stamps_us": phases,
+                "phase_stamps_note": "per phase {first, mean, last} over all CTAs (thread 0 of each), us since the first "
+                                     "CTA's start; median of 31 instrumented calls; phases as in symar_debug_phases",
+                "oracle_cpu": oracle_us(O, load_inputs(8192)),
                 "sol_us": sol,
                 "sol_parts_us": {"empty_launch_same_shape": floor["p50"], "empty_launch_1x1": floor11["p50"],
                                  "flag_round_trip": rt_ns / 1000.0, "bytes_at_peak": t_bytes_us},
@@ -364,10 +489,12 @@ def latency_suite(torch, symar, synth, hbm_gbs, quick=False, autotune=True):
             for nbytes in (128, 1024, 4096):
                 row = bench_size(nbytes // 2, ALL)
                 fl = empty_floor(row["auto"]["ctas_per_rank"], P, row["auto"]["threads"])
-                s_ol = fl["p50"] + rt_ns / 1000.0 + 2 * P * nbytes / (hbm_gbs * 1e9) * 1e6
+                s_ol = fl["p50"] + rt_ns / 1000.0 + bytes_us(nbytes, P)
                 small.append({"bytes_per_rank": nbytes, "p50_us": {k: v["p50"] for k, v in row.items()},
                               "selector": row["auto"]["algo"],
                               "selector_shape": [row["auto"]["ctas_per_rank"], row["auto"]["threads"]],
+                              "ll_shape": [row["ll"]["ctas_per_rank"], row["ll"]["threads"], row["ll"]["variant"]],
+                              "ll_minus_oneshot_us": row["ll"]["p50"] - row["oneshot"]["p50"],
                               "sol_us": s_ol, "ratio_to_sol": row["auto"]["p50"] / s_ol,
                               "bit_exact": all(v["bit_exact"] for v in row.values())})
             out["small_messages"] = small
@@ -458,6 +585,8 @@ def latency_suite(torch, symar, synth, hbm_gbs, quick=False, autotune=True):
                 named = {k: v["p50"] for k, v in row.items() if k != "auto"}
                 best_name = min(named, key=named.get)
                 ra = bench_size(8192 * B, (symar.TWOSHOT_ATOMIC,))["twoshot_atomic"]
+                fl = empty_floor(row["auto"]["ctas_per_rank"], P, row["auto"]["threads"], n=100)
+                s_ol = fl["p50"] + rt_ns / 1000.0 + bytes_us(16384 * B, P)
                 sweep.append({"bytes_per_rank": 16384 * B, "p50_us": {k: v["p50"] for k, v in row.items()},
                               "twoshot_atomic_p50_us": ra["p50"], "twoshot_atomic_within_tolerance":
                                   ra["within_tolerance"],
@@ -465,8 +594,16 @@ def latency_suite(torch, symar, synth, hbm_gbs, quick=False, autotune=True):
                                   [row["auto"]["ctas_per_rank"], row["auto"]["threads"]],
                               "best": best_name,
                               "selector_within_5pct": bool(row["auto"]["p50"] <= 1.05 * named[best_name]),
+                              "sol_us": s_ol, "ratio_to_sol": row["auto"]["p50"] / s_ol,
+                              "sol_parts_us": {"empty_launch_same_shape": fl["p50"], "flag_round_trip": rt_ns / 1000.0,
+                                               "bytes_at_measured_hbm_copy_rate": bytes_us(16384 * B, P)},
+                              "oracle_cpu": oracle_us(O, synth.make_inputs("normal", "bf16", P, 8192 * B,
+                                                                           synth.seed_for_config(2))),
                               "bit_exact": all(v["bit_exact"] for v in row.values())})
             out["sweep"] = sweep
+            out["sweep_note"] = "sol_us = empty launch of the selector's shape + median flag round trip + 2*P*M bytes at " \
+                                "the measured HBM copy rate (the messages are L2-resident, so the byte term is an upper " \
+                                "estimate of what the bound allows); oracle_cpu = the CPU oracle on the same message"
         # C5: 160 calls in one graph
         calls, count = 160, 8192 * 4
         nb = count * 2
@@ -486,12 +623,24 @@ def latency_suite(torch, symar, synth, hbm_gbs, quick=False, autotune=True):
                 got = np.stack([h.read_rank(q, base_out + k * nb, count, np.uint16) for q in range(P)])
                 exact = exact and bool(np.array_equal(got, O.allreduce(xs[k])))
         a, c, t = h.last_choice()
-        r = time_graph(torch, g, stream, calls, 60 if quick else 200)
+        n_dec = 60 if quick else 200
+        r = time_graph(torch, g, stream, calls, n_dec)
         floor = empty_floor(c, P, t)
-        t_bytes_us = 2 * P * nb / (hbm_gbs * 1e9) * 1e6
+        t_bytes_us = bytes_us(nb, P)
         sol = floor["p50"] + rt_ns / 1000.0 + t_bytes_us
+        dec_rows = []
+        for _ in range(REPEATS):
+            rt_i = sample_flag_round_trips(torch, symar)
+            fl_i = empty_floor(c, P, t)["p50"]
+            p_i = time_graph(torch, g, stream, calls, n_dec)["p50"]
+            sol_i = fl_i + rt_i["median_us"] + t_bytes_us
+            dec_rows.append({"per_call_us": p_i, "empty_launch_us": fl_i,
+                             "flag_round_trip_median_us": rt_i["median_us"], "sol_us": sol_i,
+                             "ratio_to_sol": p_i / sol_i})
         res.update({"step_total_us_p50": r["p50"] * calls, "per_call_us": r, "sol_per_call_us": sol,
                     "ratio_to_sol": r["p50"] / sol, "algo": names[a], "ctas_per_rank": c, "threads": t,
+                    "repeats": dec_rows, "ratio_to_sol_over_repeats": spread([d_["ratio_to_sol"] for d_ in dec_rows]),
+                    "oracle_cpu_one_call": oracle_us(O, xs[0]),
                     "bit_exact": exact, "calls": calls, "bytes_per_rank": nb,
                     "cache_state": "every call has its own input and output (%d MiB touched per step): "
                                    "mostly HBM-cold, unlike the warm 16 KiB number" % (2 * P * calls * nb >> 20)})
@@ -524,6 +673,146 @@ def finite(obj):
     return obj
 
 
+
+# ---------------------------------------------------------------------------------
+# output: one short line for the driver, one file per workload for the reader
+# ---------------------------------------------------------------------------------
+MAX_LINE_CHARS = 2000
+
+
+def _r(x, nd=4):
+    """Numbers of the short line: a few significant decimals are all the clocks justify."""
+    if isinstance(x, bool) or x is None:
+        return x
+    if isinstance(x, (float, np.floating)):
+        x = float(x)
+        return round(x, nd) if np.isfinite(x) else None
+    if isinstance(x, np.integer):
+        return int(x)
+    return x
+
+
+def compact_line(bw, lat, details):
+    """The line rank 0 prints: the base contract's keys, `roofline`, `cpu_baseline`, `e2e`, and a
+    handful of numbers for the latency half of the metric.  `bw` is the bandwidth workload's full
+    record (or None), `lat` the latency suite's (or None), `details` the files that hold the rest."""
+    line = {}
+    if bw:
+        for k in ("metric", "value", "unit", "n_gpus", "steps", "warmup", "ms_per_step", "higher_is_better", "scaling",
+                  "vs_baseline", "dtype", "data", "impl"):
+            line[k] = _r(bw.get(k))
+        cfg = bw.get("config", {})
+        line["config"] = {"workload": "c4: P=8 emulated ranks, fp32, %s el/rank, U(-1,1), two-shot; value=2PM bytes/time; "
+                                      "4 GiB per step >> L2" % cfg.get("elements_per_rank"),
+                          "kernel": cfg.get("kernel"),
+                          "ctas_per_rank": cfg.get("ctas_per_rank"), "threads": cfg.get("threads"),
+                          "multi_gpu": "replicas"}
+        ck = bw.get("clocks") or {}
+        line["clocks"] = {"sm_mhz": _r(ck.get("sm_mhz"), 0), "sm_max_mhz": _r(ck.get("sm_max_mhz"), 0),
+                          "reasons": ck.get("reasons", [])}
+        line["gpu_launches"] = bw.get("gpu_launches")
+        line["bit_exact_sampled"] = bw.get("bit_exact_sampled")
+        rf = bw.get("roofline") or {}
+        line["roofline"] = {"bound": rf.get("bound"), "achieved": _r(rf.get("achieved"), 1), "peak": _r(rf.get("peak"), 1),
+                            "unit": rf.get("unit"), "frac": _r(rf.get("frac")), "peak_source": "measured"
+                            if str(rf.get("peak_source", "")).startswith("measured") else "fallback",
+                            "frac_nominal_8TBs": _r(rf.get("frac_of_nominal_8TBps")),
+                            "algorithmic_bytes": rf.get("algorithmic_bytes_per_launch"),
+                            "launch_ms": _r((rf.get("launch_ms") or {}).get("mean")), "traffic": rf.get("traffic")}
+        if bw.get("cpu_baseline"):
+            cb = bw["cpu_baseline"]
+            line["cpu_baseline"] = {"value": _r(cb["value"], 2), "unit": cb["unit"], "cores": cb["cores"],
+                                    "kind": cb["kind"], "sample": "whole workload, best of 5"}
+        if bw.get("e2e"):
+            e = bw["e2e"]
+            line["e2e"] = {"value": _r(e["value"], 2), "unit": e["unit"], "h2d_bytes_per_step": e["h2d_bytes_per_step"],
+                           "d2h_bytes_per_step": e["d2h_bytes_per_step"], "ms_per_step": _r(e.get("ms_per_step"), 2),
+                           "bit_exact_sampled": e.get("bit_exact_sampled")}
+        elif bw.get("e2e_skipped"):
+            line["e2e_skipped"] = str(bw["e2e_skipped"])[:80]
+    else:
+        line.update({"metric": METRIC, "impl": "ours", "data": "synthetic", "dtype": "bf16", "note": "latency section only"})
+    if lat and "latency_section_error" in lat:
+        line["latency_section_error"] = str(lat["latency_section_error"])[:160]
+    if lat and "latency_16KB" in lat:
+        c2 = lat["latency_16KB"]
+        best = c2.get("best", {})
+        rs = c2.get("ratio_to_sol_over_repeats", {})
+        sysb = c2.get("system_scope_build") or {}
+        line["latency_16KB"] = {
+            "p50_us": _r(c2.get("p50_us"), 3), "algo": best.get("algo"),
+            "shape": [best.get("ctas_per_rank"), best.get("threads")],
+            "sol_us": _r(c2.get("sol_us"), 3), "ratio_to_sol": _r(c2.get("ratio_to_sol"), 3),
+            "repeats": rs.get("n"), "ratio_median": _r(rs.get("median"), 3), "ratio_min": _r(rs.get("min"), 3),
+            "ratio_max": _r(rs.get("max"), 3),
+            "sol_fastest_pair_us": _r(c2.get("sol_fastest_pair_us"), 3),
+            "ratio_to_sol_fastest_pair": _r(c2.get("ratio_to_sol_fastest_pair"), 3),
+            "bit_exact": all(v.get("bit_exact") for v in c2.get("per_algo", {}).values()),
+            "ll_p50_us": _r((c2.get("per_algo", {}).get("ll") or {}).get("p50"), 3),
+            "oneshot_release_p50_us": _r((c2.get("oneshot_release_signal") or {}).get("p50_us"), 3),
+            "sys_scope_p50_us": {k: _r((sysb.get(k) or {}).get("p50_us"), 3) for k in ("oneshot", "ll")}
+            if "error" not in sysb else None,
+            "oracle_cpu_us": _r((c2.get("oracle_cpu") or {}).get("all_cores_us"), 1),
+        }
+    if lat and "decode_trace" in lat:
+        line["decode_trace"] = {}
+        for key, d in lat["decode_trace"].items():
+            rs = d.get("ratio_to_sol_over_repeats", {})
+            line["decode_trace"][key] = {
+                "us_per_call": _r((d.get("per_call_us") or {}).get("p50"), 3), "ratio_to_sol": _r(d.get("ratio_to_sol"), 3),
+                "ratio_min": _r(rs.get("min"), 3), "ratio_max": _r(rs.get("max"), 3), "algo": d.get("algo"),
+                "bit_exact": d.get("bit_exact")}
+    if lat and "sweep" in lat:
+        line["sweep_ok"] = {"selector_within_5pct": all(r_.get("selector_within_5pct") for r_ in lat["sweep"]),
+                            "bit_exact": all(r_.get("bit_exact") for r_ in lat["sweep"])}
+    names = sorted(Path(d_).name for d_ in details)
+    line["details"] = (str(Path(details[0]).parent) + "/{" + ",".join(names) + "}") if details else None
+    return finite(line)
+
+
+def write_results(out_dir, bw, lat):
+    """One JSON file per workload: c4 (bandwidth), c2 (16 KiB and below, the bound's parts), c3 (sweep,
+    tuner table, context), c5 (decode trace).  Returns the paths written, relative to the repository."""
+    out_dir = Path(out_dir)
+    paths = []
+    try:
+        out_dir.mkdir(parents=True, exist_ok=True)
+    except OSError:
+        return paths
+    lat = lat or {}
+    parts = {
+        "results_c4.json": bw,
+        "results_c2.json": {k: lat[k] for k in ("latency_16KB", "small_messages", "flag_round_trip_pairs", "barrier_us")
+                            if k in lat},
+        "results_c3.json": {k: lat[k] for k in ("sweep", "sweep_note", "tuner_table_bf16", "sibling_collectives_16KB",
+                                                "scratch_sweep_32MiB") if k in lat},
+        "results_c5.json": {k: lat[k] for k in ("decode_trace",) if k in lat},
+    }
+    for name, body in parts.items():
+        if not body:
+            continue
+        try:
+            (out_dir / name).write_text(json.dumps(finite(body), allow_nan=False, indent=1) + "\n")
+            p_ = out_dir / name
+            paths.append(str(p_.relative_to(ROOT)) if p_.is_relative_to(ROOT) else str(p_))
+        except OSError:
+            pass
+    return paths
+
+
+def emit(line):
+    """Prints the one line; if it ever outgrew the limit, drops the optional parts rather than the contract's."""
+    text = json.dumps(line, allow_nan=False, separators=(",", ":"))
+    for k in ("sweep_ok", "decode_trace", "latency_16KB", "details"):
+        if len(text) < MAX_LINE_CHARS:
+            break
+        line.pop(k, None)
+        line["truncated"] = True
+        text = json.dumps(line, allow_nan=False, separators=(",", ":"))
+    print(text, flush=True)
+    return text
+
+
 # ---------------------------------------------------------------------------------
 def main():
     ap = argparse.ArgumentParser()
@@ -541,11 +830,16 @@ def main():
     ap.add_argument("--ctas", type=int, default=0)
     ap.add_argument("--threads", type=int, default=0)
     ap.add_argument("--variant", type=lambda v: int(v, 0), default=0, help="two-shot kernel variant bits")
+    ap.add_argument("--out-dir", default=str(ROOT / "gpurun_out"), help="where the per-workload result files go")
+    ap.add_argument("--scope-probe", default=None, help=argparse.SUPPRESS)     # child process of the latency section
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
     if args.impl == "reference":
         run_reference(args)
+        return
+    if args.scope_probe:
+        scope_probe(args.scope_probe, args.quick)
         return
 
     import torch
@@ -568,11 +862,8 @@ def main():
     hbm_gbs, peak_src = peaks()
     if args.latency_only:
         if rank == 0:
-            line = {"metric": METRIC, "impl": "ours", "n_gpus": world, "data": "synthetic", "dtype": "bf16",
-                    "note": "latency section only"}
-            line.update(latency_suite(torch, symar, synth, hbm_gbs, quick=args.quick,
-                                      autotune=not args.no_autotune))
-            print(json.dumps(finite(line), allow_nan=False))
+            lat = latency_suite(torch, symar, synth, hbm_gbs, quick=args.quick, autotune=not args.no_autotune)
+            emit(compact_line(None, lat, write_results(args.out_dir, None, lat)))
         if world > 1:
             dist.barrier()
             dist.destroy_process_group()
@@ -755,17 +1046,18 @@ def main():
         }
     del x
 
+    lat = None
     if rank == 0 and not args.no_latency:
         try:
-            line.update(latency_suite(torch, symar, synth, hbm_gbs, quick=args.quick, autotune=not args.no_autotune))
+            lat = latency_suite(torch, symar, synth, hbm_gbs, quick=args.quick, autotune=not args.no_autotune)
         except Exception as exc:                      # the bandwidth line above must still be reported
-            line["latency_section_error"] = f"{type(exc).__name__}: {exc}"
+            lat = {"latency_section_error": f"{type(exc).__name__}: {exc}"}
 
     if world > 1:
         dist.barrier()
         dist.destroy_process_group()
     if rank == 0:
-        print(json.dumps(finite(line), allow_nan=False))
+        emit(compact_line(line, lat, write_results(args.out_dir, line, lat)))
 
 
 if __name__ == "__main__":
