@@ -30,6 +30,8 @@
 // streams, or two host threads) race on it and must be serialised by the caller.
 #include <cuda_runtime.h>
 
+#include <atomic>
+
 #include "symar_device.cuh"
 
 namespace symar {
@@ -171,25 +173,37 @@ StaticFn pick_static(int P)
 }
 
 // Device address of the scratch, looked up once per device.  cudaGetSymbolAddress
-// answers for the CURRENT device, so the cache is indexed by it.
+// answers for the CURRENT device, so the cache is indexed by it.  Two host threads
+// may make their first call on a device at the same time: both look the address up,
+// both store the same value, and the atomic makes either store safe to read.
 constexpr int kMaxDevices = 64;
-unsigned char *g_scratch_addr[kMaxDevices];
-bool           g_scratch_known[kMaxDevices];
+std::atomic<unsigned char *> g_scratch_addr[kMaxDevices];
 
+// All CTAs of a call wait for one another, so the largest launch (kStaticSlots CTAs for
+// each of kMaxRanks ranks) must fit on the device at once; checked with the address.
 int scratch_for_current_device(unsigned char **addr)
 {
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return SYMAR_ERR_CUDA;
-    if (!g_scratch_known[dev]) {
+    unsigned char *known = g_scratch_addr[dev].load(std::memory_order_acquire);
+    if (known == nullptr) {
+        int sms = 0, per_sm = 0;
+        if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
+            cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, ll_static_kernel<BF16, kMaxRanks>, (int)kStaticThreads,
+                                                          0) != cudaSuccess) {
+            cudaGetLastError();
+            return SYMAR_ERR_CUDA;
+        }
+        if ((long)sms * per_sm < (long)kStaticSlots * kMaxRanks) return SYMAR_ERR_UNSUPPORTED;
         void *p = nullptr;
         if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || p == nullptr) {
             cudaGetLastError();
             return SYMAR_ERR_CUDA;
         }
-        g_scratch_addr[dev]  = static_cast<unsigned char *>(p);
-        g_scratch_known[dev] = true;
+        known = static_cast<unsigned char *>(p);
+        g_scratch_addr[dev].store(known, std::memory_order_release);
     }
-    *addr = g_scratch_addr[dev];
+    *addr = known;
     return SYMAR_OK;
 }
 
@@ -232,7 +246,7 @@ extern "C" int allreduce_static(const void *in, void *out, size_t rank_pitch_byt
     a.nvec       = (bytes + 15) / 16;
     a.scratch    = scratch;
     a.status     = device_status;
-    a.spin_ns    = 2000000000ull;
+    a.spin_ns    = 200000000ull;       // 0.2 s: far beyond any call, short enough not to hold a shared GPU
     a.tail_bytes = (uint32_t)(bytes % 16);
     StaticFn fn  = dtype == SYMAR_F32 ? pick_static<F32>(P) : pick_static<BF16>(P);
     const unsigned ctas = (unsigned)((a.nvec + kStaticThreads - 1) / kStaticThreads);
