@@ -6,8 +6,8 @@
  * DEVICE address.
  *
  * Model.  P ranks are emulated on one GPU as disjoint CTA partitions of ONE
- * kernel launch.  They share a symmetric heap (paper Sec. II-B, "symmetric
- * objects ... identical type, size, and layout on each processing element"):
+ * kernel launch.  They share a symmetric heap (paper Sec. II-B: every rank holds
+ * an object of the same type, size and layout at the same offset):
  * P equally laid-out rank segments, so that the object at byte offset `o` of
  * rank q is always  base + q * stride + o.  Ranks meet only through that memory,
  * exactly as GPUs of one NVLink domain meet through load/store-accessible
@@ -25,11 +25,22 @@
  * SYMAR_CTAS_PER_RANK and SYMAR_THREADS fix the launch shape of every algorithm;
  * SYMAR_SPIN_LIMIT_US bounds device-side waits; SYMAR_PDL = 0 turns programmatic dependent
  * launch off; SYMAR_DEBUG = 1 logs every call's resolved algorithm and shape to stderr
- * (nothing is printed otherwise).
+ * (nothing is printed otherwise); SYMAR_TUNE = exhaustive makes allreduce_autotune time every
+ * algorithm and shape at every size instead of pruning by the previous size's result.
  *
  * Threading: a heap may be used from one host thread and one stream at a time
  * (the per-CTA epoch counters live in the heap).  Calls on one stream are
  * ordered by the stream.
+ *
+ * What a call needs from the GPU: the CTAs of the P ranks wait for one another, so
+ * all P x C CTAs of a launch must be resident at the same time.  The library sizes
+ * every launch to what fits on the IDLE device; it cannot see other work.  Kernels
+ * of other streams or processes that hold SMs while a call runs (a second heap, a
+ * compute kernel of the caller, allreduce_static next to a heap call) can keep part
+ * of the grid from starting; the resident CTAs then wait until the bound expires
+ * (default 0.2 s), the call reports SYMAR_ERR_TIMEOUT and `out` is undefined.  Give
+ * the collective the device for its few microseconds: order it after the work
+ * before it on one stream, as a tensor-parallel layer does anyway.
  */
 #ifndef SYMAR_H
 #define SYMAR_H
@@ -46,8 +57,8 @@ typedef struct symheap symheap_t;            /* opaque; owned by the library */
 typedef enum { SYMAR_F32 = 0, SYMAR_BF16 = 1 } symar_dtype_t;
 
 typedef enum {
-    SYMAR_AUTO    = 0,   /* per-size selector (Sec. VIII: "select the best-performing
-                            low-latency algorithm based on the collected empirical results") */
+    SYMAR_AUTO    = 0,   /* per-size selector (Sec. VIII: the fastest low-latency algorithm for
+                            a size is chosen from measurements taken beforehand)              */
     SYMAR_ONESHOT = 1,   /* Sec. III-A.1, pull form: every rank reads all P inputs           */
     SYMAR_TWOSHOT = 2,   /* Sec. III-A.2: reduce-scatter, then all-gather with flag handoff  */
     SYMAR_LL      = 3,   /* Sec. IV "LL" + Sec. V example: one-shot push, data+flag stores   */
@@ -205,11 +216,14 @@ int symar_reduce(symheap_t *heap, const void *in, void *out, size_t count,
 
 /* ---- selector (Sec. VIII kernel selection; Sec. IX: selection is empirical) --
  *
- * Times every algorithm and launch shape over a power-of-two grid of message
+ * Times the algorithms and their launch shapes over a power-of-two grid of message
  * sizes (16 B ... min(bytes_per_rank / 2, 64 MiB) per rank) on an internal
  * stream, and fills the (P, dtype) table that SYMAR_AUTO and the default launch
- * shapes consult.  Synchronous; takes seconds.  OVERWRITES the user region of
- * every rank.  Before it is called, built-in default thresholds apply.         */
+ * shapes consult.  Going up the grid, an algorithm that moves more bytes than the
+ * winner and lost by more than 1.5 x one size down is not timed again, and shapes
+ * are searched around the previous size's winner (SYMAR_TUNE = exhaustive in the
+ * environment searches everything).  Synchronous; takes seconds.  OVERWRITES the
+ * user region of every rank.  Before it is called, built-in defaults apply.     */
 int allreduce_autotune(symheap_t *heap, symar_dtype_t dtype);
 
 /* The same for ONE message size: times every algorithm, shape and variant on messages
@@ -253,7 +267,12 @@ int symar_set_launch(symheap_t *heap, symar_algo_t algo, int ctas_per_rank, int 
  * every variant computes the same bits.  0 = back to the table/default choice;
  * bit 31 alone forces the plain variant (all other bits 0).  One-shot: bits 8-9 = bytes
  * per thread (0: 16, 1: 8, 2: 4), bit 14 = the prior-art form with a memory-ordering barrier
- * before the data phase and another before returning (what Sec. III-B removes; for comparison); LL: bit 8 = 8 instead of 16 payload bytes per thread;
+ * before the data phase and another before returning (what Sec. III-B removes; for comparison),
+ * bit 15 = release ordering on the "input ready" signal and nothing else changed (what the
+ * exchange costs where no kernel boundary publishes the inputs; for comparison).  LL: bit 8 = 8
+ * instead of 16 payload bytes per thread, bit 9 = the general (looping) kernel even where the
+ * single-iteration kernel covers the message, bits 12-15 = cycles / 64 by which the
+ * single-iteration kernel holds back its first poll;
  * two-shot: bit 0 = contiguous chunks also for large messages (no block-cyclic
  * ownership), bit 1 = 16-byte instead of 32-byte accesses for large messages,
  * bit 2 = never use the bulk-copy kernel, bits 8-10 = its pipeline depth (0:
@@ -275,7 +294,9 @@ int symar_set_pdl(symheap_t *heap, int enabled);
  * the scratch (1 MiB of payload per rank and iteration for the one-shot forms).       */
 int symar_set_scratch_limit(symheap_t *heap, size_t payload_bytes_per_iteration);
 
-/* Upper bound of any device-side wait, in microseconds (default 2 000 000). */
+/* Upper bound of any device-side wait, in microseconds.  Default 200 000 (0.2 s: hundreds of
+ * times the longest call, and short enough not to hold a shared GPU when a wait can never end);
+ * SYMAR_SPIN_LIMIT_US in the environment or this call change it.                      */
 int symar_set_spin_limit_us(symheap_t *heap, unsigned int microseconds);
 
 /* Test hooks; all off by default and free when off (separate kernel
@@ -309,7 +330,12 @@ int symar_debug_inject(symheap_t *heap, int mute_rank, unsigned int delay_seed,
  *           0 is a no-op.  The result is the same bits as allreduce() gives.
  * device_status : optional device word (may be NULL), owned by the caller; it is
  *           cleared on the stream before the launch and set to SYMAR_ERR_TIMEOUT
- *           if a bounded wait inside the kernel gave up.
+ *           if a bounded wait (0.2 s) inside the kernel gave up.  It is the ONLY report
+ *           of a timeout: with NULL, a wait that gave up leaves `out` incomplete and
+ *           nothing says so.  All CTAs of a call (at most 16 per rank) wait for one
+ *           another and must be resident together: a GPU whose SMs are held by other
+ *           kernels at that moment makes the waits run out.  SYMAR_ERR_UNSUPPORTED if
+ *           the device could not hold the largest launch even when idle.
  * cuda_stream : the copy-free call enqueues one small memset (only if
  *           device_status is given) and one kernel.
  *
@@ -332,6 +358,18 @@ int allreduce_static(const void *in, void *out, size_t rank_pitch_bytes, int P, 
  * (messages of 4 MiB per rank and more under SYMAR_TWOSHOT use the register kernel here).  */
 int symar_debug_span(symheap_t *heap, const void *in, void *out, size_t count, symar_dtype_t dtype,
                      symar_algo_t algo, void *cuda_stream, double *host_span_ns);
+
+/* Test hook: as symar_debug_span, with a stamp at every phase of the kernel.  Thread 0 of each
+ * CTA stamps the device timer when it reaches phase k; host_ns (24 host doubles) receives, for
+ * k = 0..7, {earliest, mean, latest} over all CTAs in nanoseconds since the earliest phase-0
+ * stamp (-1 where the kernel has no such phase); host_stamps (8 host ints) the number of CTAs
+ * that stamped phase k.  Phases: 0 = CTA in (after its wait for the previous grid); 7 = CTA out;
+ * one-shot: 1 = every peer's signal seen, 2 = thread 0's loads back, reduced, store issued;
+ * two-shot: 1 as one-shot, 2 = thread 0's share stored, 3 = the CTA's stores issued, 5 = release
+ * fence done and "done" signal sent, 4 = every peer's "done" seen; LL: 1 = counter and input
+ * back, stores issued, 3 = every peer's row seen, 4 = result stored.  Timer resolution ~32 ns.   */
+int symar_debug_phases(symheap_t *heap, const void *in, void *out, size_t count, symar_dtype_t dtype,
+                       symar_algo_t algo, void *cuda_stream, double *host_ns, int *host_stamps);
 
 /* Text of the last CUDA error seen by the library on this thread (host string). */
 const char *symar_last_cuda_error(void);
@@ -366,7 +404,7 @@ int symar_probe_pingpong_pair(int iterations, int partner_block, double *host_ns
 int symar_probe_pingpong_blocks(int iterations, int first_block, int partner_block, int grid_blocks,
                                 double *host_ns_per_round_trip, int *host_smids);
 
-/* The barrier the method removes (Sec. III-B: "each barrier will incur more than 1 us"): `ranks`
+/* The barrier the method removes (Sec. III-B puts each such barrier above a microsecond): `ranks`
  * CTAs (2..32, one per rank, all co-resident) signal every peer and wait for every peer,
  * `iterations` times in a row; *host_ns_per_barrier is the mean as seen by rank 0.  ordered = 0:
  * relaxed signals and polls, as the paper measured; 1: release signals and acquire polls (a

@@ -14,6 +14,9 @@ LIB = PKG / "libsymar.so"
 SOURCES = ["symar_kernels.cu", "symar_bulk.cu", "symar_host.cu", "symar_probe.cu", "symar_static.cu", "symar_coll.cu",
            "symar_atomic.cu"]
 
+LIB_SYS = PKG / "libsymar_sys.so"
+LIB_CHECK = PKG / "libsymar_check.so"
+
 EXAMPLE_SRC = PKG / "examples" / "llbuffer_oneshot.cu"
 EXAMPLE_LIB = PKG / "libsymar_example.so"
 
@@ -23,6 +26,7 @@ NVCC_FLAGS = [
     "-Xcompiler", "-fPIC", "-shared",
     "--ftz=false", "--prec-div=true", "--prec-sqrt=true", "--fmad=false",
     "-cudart", "static",
+    "--threads", "0",
 ]
 
 
@@ -50,6 +54,34 @@ def build_lib(force: bool = False, verbose: bool = False) -> Path:
     return LIB
 
 
+def _build_flavour(lib: Path, define: str, force: bool) -> Path:
+    deps = list(CSRC.iterdir()) + [ROOT / "include" / "symar.h", Path(__file__)]
+    if not force and lib.exists() and all(d.stat().st_mtime <= lib.stat().st_mtime for d in deps):
+        return lib
+    nvcc = os.environ.get("NVCC", "nvcc")
+    tmp = lib.with_suffix(f".so.tmp{os.getpid()}")
+    cmd = [nvcc, *NVCC_FLAGS, define, "-I", str(ROOT / "include"), "-I", str(CSRC),
+           "-o", str(tmp), *[str(CSRC / s) for s in SOURCES]]
+    subprocess.run(cmd, check=True)
+    os.replace(tmp, lib)
+    return lib
+
+
+def build_lib_sys(force: bool = False) -> Path:
+    """The same library with every flag, signal and data+flag access at SYSTEM scope (what ranks on
+    several GPUs of one NVLink domain need), for timing beside the default.  Load it by setting
+    SYMAR_LIB to its path before importing the binding."""
+    return _build_flavour(LIB_SYS, "-DSYMAR_SCOPE_SYS", force)
+
+
+def build_lib_check(force: bool = False) -> Path:
+    """The bounds-checking debug build: every heap address a kernel computes is checked against the
+    region it must lie in before it is used; a violation records SYMAR_ERR_INVAL with the rank, the
+    CTA slot and the region in the status word and skips the access.  Slower; for tests.  Load it by
+    setting SYMAR_LIB to its path before importing the binding."""
+    return _build_flavour(LIB_CHECK, "-DSYMAR_CHECK", force)
+
+
 def build_example(force: bool = False) -> Path:
     """The one-shot AllReduce of examples/llbuffer_oneshot.cu: uses include/symar_llbuffer.cuh only."""
     deps = [EXAMPLE_SRC, ROOT / "include" / "symar_llbuffer.cuh", Path(__file__)]
@@ -66,3 +98,7 @@ def build_example(force: bool = False) -> Path:
 if __name__ == "__main__":
     print(build_lib(force="--force" in sys.argv, verbose="-v" in sys.argv))
     print(build_example(force="--force" in sys.argv))
+    if "--sys" in sys.argv:
+        print(build_lib_sys(force="--force" in sys.argv))
+    if "--check" in sys.argv:
+        print(build_lib_check(force="--force" in sys.argv))

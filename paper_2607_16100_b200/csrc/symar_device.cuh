@@ -13,8 +13,14 @@ namespace symar {
 
 // ---- memory operations -------------------------------------------------------
 // On one device `.gpu` scope is sufficient; a multi-GPU build of the same
-// protocol would use `.sys`.
+// protocol would use `.sys`.  Compiling with -DSYMAR_SCOPE_SYS gives that build
+// (every flag, signal and data+flag access at system scope), so that its cost
+// can be timed beside the default.
+#ifdef SYMAR_SCOPE_SYS
+#define SYMAR_SCOPE "sys"
+#else
 #define SYMAR_SCOPE "gpu"
+#endif
 
 __device__ __forceinline__ uint32_t ld_acquire_u32(const uint32_t *p)
 {
@@ -373,6 +379,22 @@ __device__ __forceinline__ void debug_stamp_out(const KArgs &a)
         atomicMax(reinterpret_cast<unsigned long long *>(a.ctl + kCtlSpanOut), (unsigned long long)globaltimer_ns());
 }
 
+// ---- test hook: phase stamps ------------------------------------------------------------
+// Thread 0 of every CTA stamps the device's nanosecond timer when it reaches phase k; the
+// control block keeps, per phase, the earliest and the latest stamp over all CTAs and the
+// (wrapping) sum, from which the host derives the mean.  A warp issues in order, so a stamp
+// placed after an instruction that consumes a load's result is taken after that load returned.
+__device__ __forceinline__ void debug_phase(const KArgs &a, int k)
+{
+    if (!a.dbg_span || threadIdx.x != 0) return;
+    const unsigned long long now = globaltimer_ns();
+    unsigned long long *w = reinterpret_cast<unsigned long long *>(a.ctl);
+    atomicMin(w + kCtlPhaseMin / 2 + k, now);
+    atomicMax(w + kCtlPhaseMax / 2 + k, now);
+    atomicAdd(w + kCtlPhaseSum / 2 + k, now);
+    atomicAdd(w + kCtlPhaseCnt / 2 + k, 1ull);
+}
+
 // ---- test hook: seeded start delay (also stamps the CTA's start for the span hook) ----
 __device__ __forceinline__ void debug_delay(const KArgs &a, int rank, int cta)
 {
@@ -424,7 +446,9 @@ __device__ __forceinline__ ExchangePtrs exchange_ptrs(const KArgs &a, uint64_t f
     return p;
 }
 
-template <int P, bool RELEASE>
+// STAMP >= 0 (instrumented instantiations only): phase stamp once this thread's signal is issued,
+// i.e. for a release signal once its fence has completed.
+template <int P, bool RELEASE, int STAMP = -1>
 __device__ __forceinline__ bool flag_exchange_at(const KArgs &a, const ExchangePtrs &p, const uint32_t *count, int r,
                                                  int c, bool silent, bool all_warps, uint32_t &want)
 {
@@ -434,6 +458,7 @@ __device__ __forceinline__ bool flag_exchange_at(const KArgs &a, const ExchangeP
         if (RELEASE) red_release_inc_u32(p.signal);
         else red_relaxed_inc_u32(p.signal);
     }
+    if (STAMP >= 0) debug_phase(a, STAMP);
     const uint32_t n = ld_relaxed_u32(count);
     if (!all_warps && t >= 32) {
         want = n + 1;
@@ -453,11 +478,12 @@ __device__ __forceinline__ bool flag_exchange_at(const KArgs &a, const ExchangeP
     }
 }
 
-template <int P, bool RELEASE>
+template <int P, bool RELEASE, int STAMP = -1>
 __device__ __forceinline__ bool flag_exchange(const KArgs &a, uint64_t flags_off, const uint32_t *count,
                                               int r, int c, bool silent, bool all_warps, uint32_t &want)
 {
-    return flag_exchange_at<P, RELEASE>(a, exchange_ptrs<P>(a, flags_off, r, c), count, r, c, silent, all_warps, want);
+    return flag_exchange_at<P, RELEASE, STAMP>(a, exchange_ptrs<P>(a, flags_off, r, c), count, r, c, silent, all_warps,
+                                               want);
 }
 
 // Reduce-scatter + all-gather of one 16-byte vector: P loads, the rank-ordered

@@ -71,10 +71,11 @@ struct symheap {
     int       device  = 0;
     int       num_sms = 0;
     int       max_smem = 48 * 1024;   // opt-in dynamic shared memory per CTA
-    uint64_t  spin_ns = 2000000000ull;
+    uint64_t  spin_ns = 200000000ull;    // 200 ms: hundreds of times the longest call (a 256 MiB message takes 0.65 ms)
     bool      pdl          = true;    // programmatic dependent launch of every kernel
     int       env_algo     = 0;       // SYMAR_ALGO override of SYMAR_AUTO, 0 = none
     bool      debug_log    = false;   // SYMAR_DEBUG=1: one stderr line per call
+    bool      tune_exhaustive = false;   // SYMAR_TUNE=exhaustive: the tuner prunes nothing
     size_t    scratch_limit = 0;      // push algorithms: payload bytes per rank and iteration, 0 = all there is
     int       dbg_mute     = -1;
     unsigned  dbg_seed     = 0;
@@ -131,6 +132,21 @@ static int round_threads(uint64_t want)
 // Variant bits of the bulk two-shot kernel: pipeline depth and tile size.
 static int bulk_variant(int stages, int tile_log2_over_4k) { return (stages << 8) | (tile_log2_over_4k << 12); }
 
+// LL, single-iteration kernel: the largest message it covers (64 slots x 256 threads x 8 bytes), and
+// the default hold-back of the first poll in steps of 64 cycles.  The hold-back pays once the P (P - 1)
+// rows in flight are enough to make polls and stores compete in L2 (measured at P = 8, 4 and 2: none
+// below about 100 KiB in flight, one store-to-poll hop -- 768 cycles -- from a megabyte up).
+constexpr uint64_t kLLSmallMaxBytes = (uint64_t)kLLSlots * kLLMaxThreads * 8;
+static unsigned ll_default_gap(int P, uint64_t bytes)
+{
+    const uint64_t in_flight = (uint64_t)P * (P - 1) * 2 * bytes;     // payload + flags, all ranks
+    if (in_flight < (96u << 10)) return 0;
+    if (in_flight < (192u << 10)) return 2;
+    if (in_flight < (384u << 10)) return 8;
+    if (in_flight < (1u << 20)) return 10;
+    return 12;
+}
+
 // Launch shape when neither the caller nor the tuner fixed one.
 static LaunchCfg default_cfg(const symheap *h, int algo, uint64_t nvec)
 {
@@ -159,9 +175,14 @@ static LaunchCfg default_cfg(const symheap *h, int algo, uint64_t nvec)
         const int narrow = bytes <= (8u << 10) ? 2 : (bytes <= (128u << 10) ? 1 : 0);
         c.variant = narrow << 8;
         units     = work << narrow;
-    } else if (algo == SYMAR_LL && nvec * 16 <= (8u << 10)) {
-        c.variant = 0x100;
+    } else if (algo == SYMAR_LL && nvec * 16 <= kLLSmallMaxBytes) {
+        // the single-iteration kernel with 8 bytes of payload per thread (measured ahead of 16 bytes
+        // per thread at every size it covers), first poll held back by the default for this traffic
+        c.variant = 0x100 | (ll_default_gap(h->P, nvec * 16) << 12);
         units     = work * 2;
+        c.threads = units <= 256 ? round_threads(units) : (units < 2048 ? 64 : (units <= 8192 ? 128 : 256));
+        c.ctas    = (int)std::min<uint64_t>((units + c.threads - 1) / c.threads, (uint64_t)kLLSlots);
+        return c;
     }
     c.threads = units >= 2048 ? 128 : round_threads(std::max<uint64_t>(units / 16, 32));
     uint64_t ctas = (units + c.threads - 1) / c.threads;
@@ -170,13 +191,15 @@ static LaunchCfg default_cfg(const symheap *h, int algo, uint64_t nvec)
     return c;
 }
 
-// Before autotuning.  Measured on B200 (P = 8 and 4): with ranks that share one
-// L2 the pull one-shot wins from 128 B up to 256 KiB per rank, two-shot above;
-// LL's extra stores cost more than the round trip it saves (they pay off across
-// NVLink, which this emulation does not have), so AUTO picks LL only when the
-// tuner has measured it to be faster.
-static int default_algo(size_t bytes)
+// Before autotuning.  Measured on B200: with ranks that share one L2 the pull
+// one-shot wins from about 1 KiB up to 256 KiB per rank, two-shot above; LL saves
+// one dependent round trip and pays for it with P - 1 flagged stores and polls per
+// thread, which is a gain only while those are few.
+static int default_algo(int P, size_t bytes)
 {
+    // the data+flag protocol leads at the smallest sizes (Sec. VII Obs. 1); measured here: up to
+    // 16 KiB between two ranks, up to a few hundred bytes among eight, nowhere among four
+    if ((P == 2 && bytes <= (16u << 10)) || (P == 8 && bytes <= 512)) return SYMAR_LL;
     if (bytes <= (256u << 10)) return SYMAR_ONESHOT;
     return SYMAR_TWOSHOT;
 }
@@ -204,7 +227,7 @@ static int make_plan(symheap *h, size_t in_off, size_t out_off, size_t count, in
         tuned = true;
     }
 
-    if (algo == SYMAR_AUTO) algo = h->env_algo ? h->env_algo : (tuned ? tn.best_algo[b] : default_algo(bytes));
+    if (algo == SYMAR_AUTO) algo = h->env_algo ? h->env_algo : (tuned ? tn.best_algo[b] : default_algo(h->P, bytes));
 
     LaunchCfg cfg = default_cfg(h, algo, nvec);
     if (tuned && tn.cfg[algo][b].ctas > 0) cfg = tn.cfg[algo][b];
@@ -247,6 +270,19 @@ static int make_plan(symheap *h, size_t in_off, size_t out_off, size_t count, in
     }
     if (!fn) return SYMAR_ERR_INVAL;
     const int cap_slots = (is_push(algo) || algo == SYMAR_TWOSHOT_ATOMIC) ? kLLSlots : kMaxCtas;
+    // LL: a message that the launch covers with one unit per thread takes the straight-line
+    // single-iteration kernel (variant bit 9 keeps the general one)
+    if (algo == SYMAR_LL && !(var & 0x200u) && !h->scratch_limit) {
+        const int words      = (var & 0x100u) ? 2 : 4;
+        const uint64_t units = (bytes + 4 * words - 1) / (4 * words);
+        const uint64_t need  = (units + cfg.threads - 1) / cfg.threads;
+        KernelFn sfn = ll_small_kernel_for(dtype, h->P, words, dbg_on(h));
+        if (sfn && need <= (uint64_t)cfg.ctas && need <= (uint64_t)cap_slots &&
+            need <= (uint64_t)std::max(1, max_resident(h, sfn, cfg.threads, 0) / h->P)) {
+            fn       = sfn;
+            cfg.ctas = (int)need;
+        }
+    }
     const int cap_res   = std::max(1, max_resident(h, fn, cfg.threads, p->smem) / h->P);
     cfg.ctas = std::max(1, std::min({cfg.ctas, cap_slots, cap_res}));
 
@@ -397,8 +433,10 @@ static int run_collective(symheap *h, int op, const void *in, void *out, size_t 
 // ---- autotuner ---------------------------------------------------------------------
 
 // Median per-call time (us) of K back-to-back calls captured in one graph.
+// `give_up_us` > 0: a candidate whose first two replays both take longer than that is not worth
+// the remaining replays (its faster replay is returned).
 static int time_calls(symheap *h, cudaStream_t s, size_t count, int dtype, int algo, int K, int reps,
-                      double *us_out)
+                      double *us_out, double give_up_us = 0.0)
 {
     const size_t bytes = count * elem_size(dtype);
     const void *in = h->seg0;
@@ -430,6 +468,10 @@ static int time_calls(symheap *h, cudaStream_t s, size_t count, int dtype, int a
         cudaEventRecord(e1, s);
         cudaEventSynchronize(e1);
         cudaEventElapsedTime(&ms[i], e0, e1);
+        if (i == 1 && give_up_us > 0.0 && (double)std::min(ms[0], ms[1]) * 1000.0 / K > give_up_us) {
+            ms.assign(reps, std::min(ms[0], ms[1]));
+            break;
+        }
     }
     cudaEventDestroy(e0);
     cudaEventDestroy(e1);
@@ -442,9 +484,21 @@ static int time_calls(symheap *h, cudaStream_t s, size_t count, int dtype, int a
     return SYMAR_OK;
 }
 
-// Times every algorithm, launch shape and kernel variant on messages of `bytes` per rank
-// and records the winners in bucket b of `tn`.
-static int tune_bucket(symheap *h, int dtype, int b, size_t bytes, cudaStream_t s, Tuned &tn)
+// Times algorithms, launch shapes and kernel variants on messages of `bytes` per rank and records
+// the winners in bucket b of `tn`.
+//
+// With `prev` >= 0 (the bucket tuned just before, one size step down) the search is pruned by
+// what that bucket showed, unless the heap asks for the exhaustive search:
+//   * an algorithm that moves more bytes per rank than the winner does (the push forms: 2 to 4 times
+//     the payload through scratch; above 1 MiB also one-shot: P times the reads) and that lost by
+//     more than 1.5 x one step down is not timed again -- its traffic grows as fast as the winner's
+//     or faster, so it cannot come back (Table I's volume column); its row reads "not timed";
+//   * above 256 KiB the launch shapes of an algorithm are searched around its winner one step down
+//     (CTA counts from half to four times, block sizes from half to twice), since a message twice
+//     as large wants the same shape or the next larger one;
+//   * a shape whose first two replays are a quarter slower than the algorithm's best so far is
+//     not replayed further.
+static int tune_bucket(symheap *h, int dtype, int b, size_t bytes, cudaStream_t s, Tuned &tn, int prev = -1)
 {
     static const int kThreads[] = {64, 128, 256, 512};
     static const int kCtas[]    = {1, 2, 4, 8, 10, 12, 15, 16, 18, 24, 32, 37, 48, 64, 74};
@@ -453,6 +507,7 @@ static int tune_bucket(symheap *h, int dtype, int b, size_t bytes, cudaStream_t 
     const uint64_t nvec = (bytes + 15) / 16;
     const int K    = bytes <= (1u << 20) ? 24 : (bytes <= (16u << 20) ? 6 : 2);
     const int reps = 7;
+    const bool prune = prev >= 0 && !h->tune_exhaustive;
     LaunchCfg saved[kAlgos];
     unsigned saved_variant[kAlgos];
     bool saved_forced[kAlgos];
@@ -464,11 +519,17 @@ static int tune_bucket(symheap *h, int dtype, int b, size_t bytes, cudaStream_t 
     int rc = SYMAR_OK;
     double best_us = 1e30;
     tn.best_algo[b] = SYMAR_ONESHOT;
+    double prev_best = 1e30;
+    if (prune)
+        for (int a = SYMAR_ONESHOT; a <= kLastTuned; ++a) prev_best = std::min(prev_best, tn.us[a][prev]);
     for (int algo = SYMAR_ONESHOT; algo <= kLastTuned && rc == SYMAR_OK; ++algo) {
         tn.us[algo][b]  = 1e30;
         tn.cfg[algo][b] = LaunchCfg{};
         if (is_push(algo) && bytes > (4u << 20)) continue;   // scratch traffic through L2: hopeless there
         if (algo != SYMAR_TWOSHOT && bytes > (32u << 20)) continue;   // only two-shot moves the minimum of bytes
+        if (prune && bytes > (64u << 10) && (is_push(algo) || (algo == SYMAR_ONESHOT && bytes > (1u << 20))) &&
+            tn.us[algo][prev] > 1.5 * prev_best)
+            continue;                                        // lost one step down, and its traffic grows at least as fast
         const uint64_t work = (algo == SYMAR_TWOSHOT || is_twoshot_push(algo)) ? (nvec + h->P - 1) / h->P : nvec;
         // kernel variants worth timing: the default; for two-shot in the bandwidth
         // regime the bulk kernel's tile sizes and depths, and the register kernel
@@ -479,21 +540,38 @@ static int tune_bucket(symheap *h, int dtype, int b, size_t bytes, cudaStream_t 
                         bulk_variant(4, 0), 4};
         else if (algo == SYMAR_ONESHOT && bytes <= (1u << 20))
             variants = {0, 0x100, 0x200};            // 16, 8 or 4 bytes per thread
-        else if (algo == SYMAR_LL && bytes <= (256u << 10))
-            variants = {0, 0x100};                   // 16 or 8 bytes of payload per thread
+        else if (algo == SYMAR_LL && bytes <= kLLSmallMaxBytes) {
+            // 8 bytes of payload per thread with the first poll held back by the default for this
+            // traffic, by a quarter of a hop less and more, and not at all; 16 bytes per thread
+            const int g = (int)ll_default_gap(h->P, bytes);
+            variants = {0x100 | (g << 12)};
+            for (int alt : {g - 4, g + 3, 0})
+                if (alt >= 0 && alt <= 15 && alt != g &&
+                    std::find(variants.begin(), variants.end(), 0x100 | (alt << 12)) == variants.end())
+                    variants.push_back(0x100 | (alt << 12));
+            if (bytes >= 4096) variants.push_back(g << 12);
+        } else if (algo == SYMAR_LL && bytes <= (256u << 10))
+            variants = {0, 0x100};                   // general kernel: 16 or 8 bytes of payload per thread
         struct Cand { double us; LaunchCfg cfg; };
         std::vector<Cand> cands;                     // bandwidth regime: the first pass's shapes, for a second look
+        // the neighbourhood of this algorithm's winner one step down
+        // (above 256 KiB only: below, few shapes are valid, calls are short, and the best shape still moves
+        // between the unit widths from one size to the next)
+        const LaunchCfg near =
+            (prune && bytes > (256u << 10) && tn.cfg[algo][prev].ctas > 0) ? tn.cfg[algo][prev] : LaunchCfg{};
         for (int var : variants) {
             // threads a shape needs: one per unit of this variant
             const uint64_t units = bulk ? work : work << ((var >> 8) & 3);
             for (int T : kThreads) {
                 if (bulk && var != 4 && T != 128 && T != 256) continue;
+                if (near.ctas > 0 && (2 * T < near.threads || T > 2 * near.threads)) continue;
                 for (int C : kCtas) {
                     // skip shapes with far more threads than vectors, except the smallest
                     if ((uint64_t)C * T > 2 * units && !(C == 1 && T == 64)) continue;
                     // and shapes that would leave each thread hundreds of units
                     if (!bulk && units / ((uint64_t)C * T) > 4096) continue;
                     if (bulk && (C * h->P < 48)) continue;
+                    if (near.ctas > 0 && (2 * C < near.ctas || C > 4 * near.ctas)) continue;
                     h->forced[algo]         = LaunchCfg{C, T, var};
                     h->variant[algo]        = (unsigned)var;
                     h->variant_forced[algo] = true;
@@ -501,7 +579,9 @@ static int tune_bucket(symheap *h, int dtype, int b, size_t bytes, cudaStream_t 
                     if (make_plan(h, 0, round_up(bytes, kAlign), count, dtype, algo, &p) != SYMAR_OK) continue;
                     if (p.cfg.ctas != C || p.cfg.threads != T) continue;   // clamped: a duplicate of another shape
                     double us = 0;
-                    rc = time_calls(h, s, count, dtype, algo, K, reps, &us);
+                    // a shape a quarter slower than this algorithm's best so far is dropped after two replays
+                    rc = time_calls(h, s, count, dtype, algo, K, reps, &us,
+                                    h->tune_exhaustive || tn.us[algo][b] > 1e29 ? 0.0 : 1.25 * tn.us[algo][b]);
                     if (rc != SYMAR_OK) break;
                     if (bulk) cands.push_back(Cand{us, LaunchCfg{C, T, var}});
                     // a larger launch must win by more than the timing noise (1.5 %) to displace a smaller one
@@ -588,7 +668,7 @@ static int autotune(symheap *h, int dtype, size_t only_bytes)
     h->tuned[dtype].valid = false;
     std::memset(h->tuned[dtype].have, 0, sizeof h->tuned[dtype].have);
     for (int b = tn.lo_bucket; b <= tn.hi_bucket && rc == SYMAR_OK; ++b)
-        rc = tune_bucket(h, dtype, b, (size_t)1 << b, s, tn);
+        rc = tune_bucket(h, dtype, b, (size_t)1 << b, s, tn, b > tn.lo_bucket ? b - 1 : -1);
     cudaStreamSynchronize(s);
     cudaStreamDestroy(s);
     if (rc != SYMAR_OK) {
@@ -655,7 +735,8 @@ static int create_common(symheap_t **heap, int P, size_t bytes_per_rank, void *m
     // device-side wait; SYMAR_ALGO = oneshot | twoshot | ll | ... replaces SYMAR_AUTO's choice;
     // SYMAR_PDL = 0 turns programmatic dependent launch off; SYMAR_CTAS_PER_RANK and
     // SYMAR_THREADS fix the launch shape of every algorithm; SYMAR_DEBUG = 1 logs every
-    // call's resolved algorithm and shape to stderr.
+    // call's resolved algorithm and shape to stderr; SYMAR_TUNE = exhaustive makes
+    // allreduce_autotune time every algorithm and shape at every size (no pruning).
     if (const char *v = std::getenv("SYMAR_SPIN_LIMIT_US")) {
         const long us = std::atol(v);
         if (us > 0) h->spin_ns = (uint64_t)us * 1000ull;
@@ -678,6 +759,7 @@ static int create_common(symheap_t **heap, int P, size_t bytes_per_rank, void *m
             for (int a = SYMAR_ONESHOT; a <= kLastAlgo; ++a) h->forced[a].threads = t;
     }
     if (const char *v = std::getenv("SYMAR_DEBUG")) h->debug_log = std::atoi(v) != 0;
+    if (const char *v = std::getenv("SYMAR_TUNE")) h->tune_exhaustive = std::string(v) == "exhaustive";
     *heap = h;
     return SYMAR_OK;
 }
@@ -1094,6 +1176,42 @@ int symar_debug_span(symheap_t *heap, const void *in, void *out, size_t count, s
     CU(cudaStreamSynchronize(s));
     if (w[0] == ~0ull || w[1] < w[0]) return SYMAR_ERR_UNSUPPORTED;     // this kernel carries no stamps
     *host_span_ns = (double)(w[1] - w[0]);
+    return SYMAR_OK;
+}
+
+int symar_debug_phases(symheap_t *heap, const void *in, void *out, size_t count, symar_dtype_t dtype,
+                       symar_algo_t algo, void *cuda_stream, double *host_ns, int *host_stamps)
+{
+    if (!heap || !host_ns || !host_stamps) return SYMAR_ERR_INVAL;
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    unsigned long long w[4 * kPhases];
+    for (int k = 0; k < kPhases; ++k) {
+        w[k]               = ~0ull;     // earliest
+        w[kPhases + k]     = 0ull;      // latest
+        w[2 * kPhases + k] = 0ull;      // wrapping sum
+        w[3 * kPhases + k] = 0ull;      // stamps
+    }
+    CU(cudaMemcpyAsync(heap->ctl + kCtlPhaseMin, w, sizeof w, cudaMemcpyHostToDevice, s));
+    CU(cudaStreamSynchronize(s));                       // `w` is on this stack frame
+    heap->dbg_span = true;
+    const int rc = run(heap, in, out, count, (int)dtype, (int)algo, s);
+    heap->dbg_span = false;
+    if (rc != SYMAR_OK) return rc;
+    CU(cudaMemcpyAsync(w, heap->ctl + kCtlPhaseMin, sizeof w, cudaMemcpyDeviceToHost, s));
+    CU(cudaStreamSynchronize(s));
+    if (w[3 * kPhases] == 0) return SYMAR_ERR_UNSUPPORTED;             // this kernel carries no stamps
+    const unsigned long long t0 = w[0];
+    for (int k = 0; k < kPhases; ++k) {
+        const unsigned long long n = w[3 * kPhases + k];
+        host_stamps[k] = (int)n;
+        if (n == 0) {
+            host_ns[3 * k] = host_ns[3 * k + 1] = host_ns[3 * k + 2] = -1.0;
+            continue;
+        }
+        host_ns[3 * k]     = (double)(long long)(w[k] - t0);
+        host_ns[3 * k + 1] = (double)(long long)(w[2 * kPhases + k] - n * t0) / (double)n;   // sums wrap; the difference does not
+        host_ns[3 * k + 2] = (double)(long long)(w[kPhases + k] - t0);
+    }
     return SYMAR_OK;
 }
 

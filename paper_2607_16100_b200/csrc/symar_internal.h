@@ -12,6 +12,9 @@ using KernelFn = void (*)(const KArgs);
 // variant that honours the test hooks.  nullptr for unsupported combinations.
 KernelFn kernel_for(int algo, int dtype, int P, bool dbg);
 
+// LL for messages that one iteration covers with one unit of `words` (2 or 4) 32-bit words per thread.
+KernelFn ll_small_kernel_for(int dtype, int P, int words, bool dbg);
+
 // Two-shot kernel of the bandwidth regime (bulk asynchronous copies through
 // shared memory); needs bulk_smem_bytes() of dynamic shared memory.
 KernelFn bulk_kernel_for(int dtype, int P);

@@ -12,6 +12,8 @@
 //                        to every peer's scratch as {payload, flag} 8-byte stores,
 //                        poll the own scratch, reduce, write the own output; scratch
 //                        is double-buffered by iteration parity.
+//   ll_small_kernel      the same for messages that one iteration covers with one
+//                        unit per thread: straight-line code, all peers polled at once.
 //   sentinel_kernel      Sec. IV "Sentinel": the same push with bare payload into
 //                        scratch that holds a sentinel word; the receiver polls
 //                        until every word has changed and restores the sentinel.
@@ -34,7 +36,9 @@ namespace symar {
 // For small messages the loads are issued BEFORE the CTA barrier that lets thread 0 publish
 // the exchange count, so that the barrier, the publication and the trigger of the dependent
 // launch cost nothing while the data travels (measured -0.03 us of 1.72 us at 16 KiB).
-template <typename E, int P, int W>
+// (Measured and dropped: two units per thread in half as many CTAs, +0.1 to +0.3 us at 16 KiB;
+// leaving the trigger of the dependent launch to the kernel's end, +0.1 us at every size.)
+template <typename E, int P, int W, bool DBG>
 __device__ __forceinline__ void oneshot_data(const KArgs &a, char *out, uint64_t first, uint64_t step, bool ok,
                                              uint32_t *count, uint32_t want)
 {
@@ -65,6 +69,7 @@ __device__ __forceinline__ void oneshot_data(const KArgs &a, char *out, uint64_t
         store_words<W>(out + first * (4 * W), reduce_words_in_rank_order<E, P, W>(x),
                        left < 4u * W ? (uint32_t)left : 4u * W);
     }
+    if (DBG) debug_phase(a, 2);               // this thread's loads are back, reduced and on their way out
     if (!ok) return;
     for (uint64_t u = first + step; u < nunits; u += step) {
 #pragma unroll
@@ -99,20 +104,28 @@ __global__ void __launch_bounds__(kMaxThreads) oneshot_kernel(const KArgs a)
     }
     if (DBG) debug_delay(a, r, c);
     if (DBG && a.dbg_mute == r) return;       // test hook: this rank never joins
+    if (DBG) debug_phase(a, 0);
 
     // Variant bit 14: the prior-art form that the method replaces (Sec. III-B), for comparison only --
     // a memory-ordering barrier before the data phase (release signals) and a second one before
     // returning, as a pull kernel needs when nothing else keeps inputs from being overwritten.
+    // Variant bit 15: release on the "input ready" signal and nothing else changed -- what the
+    // exchange costs when the signal itself has to publish the input, as it must where no kernel
+    // boundary common to all ranks does (Sec. II-B: remote writes visible to polling); comparison only.
+    // (Measured and dropped: only warp 0 polls while the other warps wait at a CTA barrier, +0.03 to
+    // +0.06 us: the barrier costs more than three more warps' polls of the same sector.)
     const bool prior_art = a.variant & 0x4000u;
+    const bool release   = prior_art || (a.variant & 0x8000u);
     uint32_t want;
-    const bool ok = prior_art ? flag_exchange_at<P, true>(a, xp, count, r, c, false, true, want)
-                              : flag_exchange_at<P, false>(a, xp, count, r, c, false, true, want);
+    const bool ok = release ? flag_exchange_at<P, true>(a, xp, count, r, c, false, true, want)
+                            : flag_exchange_at<P, false>(a, xp, count, r, c, false, true, want);
+    if (DBG) debug_phase(a, 1);
     char *out = seg_r + a.out_off;
     const uint64_t first = (uint64_t)c * T + t, step = (uint64_t)C * T;
     const uint32_t narrow = (a.variant >> 8) & 3u;     // bytes per thread: 16, 8 or 4
-    if (narrow == 2) oneshot_data<E, P, 1>(a, out, first, step, ok, count, want);
-    else if (narrow == 1) oneshot_data<E, P, 2>(a, out, first, step, ok, count, want);
-    else oneshot_data<E, P, 4>(a, out, first, step, ok, count, want);
+    if (narrow == 2) oneshot_data<E, P, 1, DBG>(a, out, first, step, ok, count, want);
+    else if (narrow == 1) oneshot_data<E, P, 2, DBG>(a, out, first, step, ok, count, want);
+    else oneshot_data<E, P, 4, DBG>(a, out, first, step, ok, count, want);
     if (prior_art) {
         uint32_t *dcount = reinterpret_cast<uint32_t *>(seg_r + a.epoch_off + done_count_off(c));
         uint32_t dwant;
@@ -120,7 +133,10 @@ __global__ void __launch_bounds__(kMaxThreads) oneshot_kernel(const KArgs a)
         flag_exchange<P, true>(a, a.done_off, dcount, r, c, !ok, false, dwant);
         if (t == 0) *dcount = dwant;
     }
-    if (DBG) debug_stamp_out(a);
+    if (DBG) {
+        debug_stamp_out(a);
+        debug_phase(a, 7);
+    }
 }
 
 // The same for two adjacent vectors moved as one 32-byte access per peer.
@@ -157,8 +173,10 @@ __global__ void __launch_bounds__(kMaxThreads) twoshot_kernel(const KArgs a)
 
     // reduce-scatter: which vectors rank r owns
     uint32_t rwant, dwant;
+    if (DBG) debug_phase(a, 0);
     bool ok = flag_exchange<P, false>(a, a.ready_off, rcount, r, c, false, true, rwant);
     if (a.pdl) pdl_launch_dependents();
+    if (DBG) debug_phase(a, 1);               // every peer's input is ready
     if (ok) {
         const uint64_t step = (uint64_t)C * T;
         if (a.blk_log2 == kOneChunk) {
@@ -198,13 +216,20 @@ __global__ void __launch_bounds__(kMaxThreads) twoshot_kernel(const KArgs a)
     }
     // handoff: this CTA's part of rank r's vectors has landed everywhere -> tell
     // every peer; then wait until every peer's CTA c has delivered its part here.
+    if (DBG) debug_phase(a, 2);               // thread 0's share reduced, its stores issued
     __syncthreads();
-    flag_exchange<P, true>(a, a.done_off, dcount, r, c, !ok, false, dwant);
+    if (DBG) debug_phase(a, 3);               // the whole CTA's stores issued
+    if (DBG) flag_exchange<P, true, 5>(a, a.done_off, dcount, r, c, !ok, false, dwant);   // 5: release fence done, signal sent
+    else flag_exchange<P, true>(a, a.done_off, dcount, r, c, !ok, false, dwant);
+    if (DBG) debug_phase(a, 4);               // every peer's part has landed here
     if (t == 0) {
         *rcount = rwant;
         *dcount = dwant;
     }
-    if (DBG) debug_stamp_out(a);
+    if (DBG) {
+        debug_stamp_out(a);
+        debug_phase(a, 7);
+    }
 }
 
 // LL with 8 bytes of payload per thread: one 16-byte {w0,f,w1,f} store per peer and
@@ -298,6 +323,7 @@ __global__ void __launch_bounds__(kLLMaxThreads) ll_kernel(const KArgs a)
     const uint64_t n0 = ld_relaxed_u64(ep);
     if (DBG) debug_delay(a, r, c);
     if (DBG && a.dbg_mute == r) return;       // test hook: this rank never joins
+    if (DBG) debug_phase(a, 0);
 
     const char *in = seg_r + a.in_off;
     char *out      = seg_r + a.out_off;
@@ -332,6 +358,7 @@ __global__ void __launch_bounds__(kLLMaxThreads) ll_kernel(const KArgs a)
                 st_relaxed_v2u64(dst + (size_t)kLLSlotVecs * 16, d2, d3);
             }
         }
+        if (DBG && it == 0) debug_phase(a, 1);     // counter and input were back, first trip's stores issued
         // recvReduce: poll the P-1 peer rows together; a row that has arrived is
         // not polled again
         for (uint32_t k = t; k < cnt && !failed; k += T) {
@@ -373,6 +400,7 @@ __global__ void __launch_bounds__(kLLMaxThreads) ll_kernel(const KArgs a)
                 if (q == r) x[q] = own;
             store_result(out, v0 + k, reduce_in_rank_order<E, P>(x), a.nvec, a.tail_bytes);
         }
+        if (DBG && it == 0) debug_phase(a, 4);     // first iteration received, reduced and stored
         // No CTA barrier between iterations: position k is sent and received by
         // the same thread index on every rank, and a thread sends iteration i+1
         // only after its own receive of iteration i, which needed the peer
@@ -381,7 +409,146 @@ __global__ void __launch_bounds__(kLLMaxThreads) ll_kernel(const KArgs a)
     }
     __syncthreads();          // every thread has read the counter before it moves
     if (t == 0) *ep = n0 + a.iters;
-    if (DBG) debug_stamp_out(a);
+    if (DBG) {
+        debug_stamp_out(a);
+        debug_phase(a, 7);
+    }
+}
+
+// LL for a message that one iteration covers with ONE unit of W words per thread (Sec. V example
+// kernel; Sec. VII Obs. 1: LL owes its small-message lead to compile-time unrolling and to polling
+// all peers in parallel): no loop over units or iterations, no run-time choice of the unit width,
+// the counter load and the input load in flight together, P - 1 stores, then polls of all P - 1 rows
+// at once.  Unit t of CTA c sits at byte t * 16 of the sender's row (W = 2: {w0,f,w1,f}) and, for
+// W = 4, also in the second plane of the row ({w2,f,w3,f}); the flag is the slot's own
+// iteration counter, so this kernel and ll_kernel can alternate on one heap.
+//
+// Polling.  A poll of a line that a peer has just written returns after several hundred cycles, and
+// a poll that reaches L2 a moment before the data costs that round trip again while it competes
+// with the peers' stores for L2.  The first poll is therefore held back by `gap` cycles (64 cycles x
+// variant bits 12-15; a default per size, refined by the tuner): measured at P = 8, 2.8 -> 2.3 us at
+// 16 KiB with 768 cycles (about one store-to-poll hop), no gain below 1 KiB.  Keeping two polls per
+// row in flight instead (a second one issued half a round trip after the first) was measured
+// slower at every size (+0.4 us).
+//
+// Dependent launch.  The kernel never triggers its dependent early: the next call then starts when
+// this grid has drained, overlapping only its launch with this grid's completion.  Measured against
+// a trigger before the stores, after them or after the polls: 1.56 instead of 1.81 us at 128 B,
+// equal or better at every size up to 64 KiB (an early-resident successor only sits in its wait).
+template <int W> struct LLRaw { U64x2 v[W / 2]; };
+
+template <int W>
+__device__ __forceinline__ LLRaw<W> ll_row_load(const char *p)
+{
+    LLRaw<W> d;
+    d.v[0] = ld_relaxed_v2u64(p);
+    if (W == 4) d.v[W / 2 - 1] = ld_relaxed_v2u64(p + (size_t)kLLSlotVecs * 16);
+    return d;
+}
+template <int W>
+__device__ __forceinline__ bool ll_row_take(const LLRaw<W> &d, uint32_t e, Words<W> &x)
+{
+    bool here = (uint32_t)(d.v[0].a >> 32) == e && (uint32_t)(d.v[0].b >> 32) == e;
+    if (W == 4) here = here && (uint32_t)(d.v[W / 2 - 1].a >> 32) == e && (uint32_t)(d.v[W / 2 - 1].b >> 32) == e;
+    if (here) {
+        x.w[0] = (uint32_t)d.v[0].a;
+        x.w[1] = (uint32_t)d.v[0].b;
+        if (W == 4) {
+            x.w[W - 2] = (uint32_t)d.v[W / 2 - 1].a;
+            x.w[W - 1] = (uint32_t)d.v[W / 2 - 1].b;
+        }
+    }
+    return here;
+}
+__device__ __forceinline__ void idle_cycles(uint32_t cycles)
+{
+    if (cycles == 0) return;
+    const uint32_t c0 = (uint32_t)clock();
+    while ((uint32_t)clock() - c0 < cycles) { /* bounded by `cycles` */ }
+}
+
+template <typename E, int P, int W, bool DBG>
+__global__ void __launch_bounds__(kLLMaxThreads) ll_small_kernel(const KArgs a)
+{
+    const int c = blockIdx.x, r = blockIdx.y;
+    const uint32_t t = threadIdx.x, T = blockDim.x;
+    char *seg_r  = a.seg0 + (size_t)r * a.stride;
+    uint64_t *ep = reinterpret_cast<uint64_t *>(seg_r + a.epoch_off) + c;
+    const uint64_t bytes = a.tail_bytes ? (a.nvec - 1) * 16 + a.tail_bytes : a.nvec * 16;
+    const uint64_t lo    = ((uint64_t)c * T + t) * (4 * W);
+    const uint32_t valid = lo < bytes ? (bytes - lo < 4u * W ? (uint32_t)(bytes - lo) : 4u * W) : 0u;
+    const char *in  = seg_r + a.in_off + lo;
+    const size_t pos = (size_t)t * 16;
+    const uint32_t gap = ((a.variant >> 12) & 15u) * 64u;
+    if (a.pdl) pdl_wait_holding(ep, in, seg_r);       // the previous call has left the heap
+    const uint64_t n = ld_relaxed_u64(ep) + 1;        // advanceEpoch: flag value and sub-buffer
+    Words<W> own;
+#pragma unroll
+    for (int i = 0; i < W; ++i) own.w[i] = 0u;
+    if (valid) {
+        // the last 16-byte vector of a message lies inside the user region even when it is partial
+        if (W == 2)
+            asm volatile("ld.global.nc.L1::no_allocate.v2.u32 {%0, %1}, [%2];"
+                         : "=r"(own.w[0]), "=r"(own.w[1])
+                         : "l"(in));
+        else
+            asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];"
+                         : "=r"(own.w[0]), "=r"(own.w[1]), "=r"(own.w[W - 2]), "=r"(own.w[W - 1])
+                         : "l"(in));
+    }
+    if (DBG) debug_delay(a, r, c);
+    if (DBG && a.dbg_mute == r) return;       // test hook: this rank never joins
+    if (DBG) debug_phase(a, 0);
+
+    const uint32_t e      = flag_of(n);
+    const uint64_t region = a.ll_off + ((uint64_t)(n & 1) * kLLSlots + c) * P * kLLSenderBytes;
+    bool failed = false;
+    if (valid) {
+        const uint64_t hi_e = (uint64_t)e << 32;
+        char *dst = a.seg0 + region + (size_t)r * kLLSenderBytes + pos;      // my row in rank 0's region
+#pragma unroll
+        for (int q = 0; q < P; ++q) {
+            if (q != r) {
+                st_relaxed_v2u64(dst, hi_e | own.w[0], hi_e | own.w[1]);
+                if (W == 4) st_relaxed_v2u64(dst + (size_t)kLLSlotVecs * 16, hi_e | own.w[W - 2], hi_e | own.w[W - 1]);
+            }
+            dst += a.stride;
+        }
+        if (DBG) debug_phase(a, 1);           // counter and input were back, all stores issued
+        const char *src = seg_r + region + pos;                              // row q of my region: + q * kLLSenderBytes
+        Words<W> x[P];
+        unsigned need = ((1u << P) - 1u) & ~(1u << r);
+        Spin spin;
+        idle_cycles(gap);
+        while (need != 0) {
+            LLRaw<W> d[P];
+#pragma unroll
+            for (int q = 0; q < P; ++q)
+                if (need >> q & 1u) d[q] = ll_row_load<W>(src + (size_t)q * kLLSenderBytes);
+#pragma unroll
+            for (int q = 0; q < P; ++q)
+                if ((need >> q & 1u) && ll_row_take<W>(d[q], e, x[q])) need &= ~(1u << q);
+            if (need != 0 && spin.due() && spin.expired(a.spin_ns)) {
+                report_timeout(a.ctl, r, __ffs(need) - 1, c);
+                failed = true;
+                break;
+            }
+        }
+        if (DBG) debug_phase(a, 3);           // every peer's row seen
+        if (!failed) {
+#pragma unroll
+            for (int q = 0; q < P; ++q)
+                if (q == r) x[q] = own;
+            store_words<W>(seg_r + a.out_off + lo, reduce_words_in_rank_order<E, P, W>(x), valid);
+        }
+        if (DBG) debug_phase(a, 4);
+    }
+    __syncthreads();          // every thread has read the counter before it moves
+    if (t == 0) *ep = n;
+    if (DBG) {
+        debug_stamp_out(a);
+        debug_phase(a, 7);
+    }
 }
 
 // One-shot push with sentinel synchronisation (Sec. IV "Sentinel"; Sec. V send / recv with
@@ -474,7 +641,10 @@ __global__ void __launch_bounds__(kMaxThreads) sentinel_kernel(const KArgs a)
     }
     __syncthreads();
     if (t == 0) *ep = n0 + a.iters;
-    if (DBG) debug_stamp_out(a);
+    if (DBG) {
+        debug_stamp_out(a);
+        debug_phase(a, 7);
+    }
 }
 
 // ---- two-shot over the push buffers (the paper's AllReduce_LLBuffer_Twoshot; Table I rows
@@ -646,7 +816,10 @@ __global__ void __launch_bounds__(kPushTwoshotMaxThreads) twoshot_push_kernel(co
     }
     __syncthreads();
     if (t == 0) *ep = n0 + a.iters;
-    if (DBG) debug_stamp_out(a);
+    if (DBG) {
+        debug_stamp_out(a);
+        debug_phase(a, 7);
+    }
 }
 
 // ---- dispatch ---------------------------------------------------------------------
@@ -681,6 +854,25 @@ KernelFn kernel_for(int algo, int dtype, int P, bool dbg)
 {
     if (dtype == SYMAR_F32) return dbg ? pick_ranks<F32, true>(algo, P) : pick_ranks<F32, false>(algo, P);
     if (dtype == SYMAR_BF16) return dbg ? pick_ranks<BF16, true>(algo, P) : pick_ranks<BF16, false>(algo, P);
+    return nullptr;
+}
+
+template <typename E, bool DBG>
+static KernelFn pick_ll_small_ranks(int P, int words)
+{
+    switch (P) {
+        case 1: return words == 2 ? ll_small_kernel<E, 1, 2, DBG> : ll_small_kernel<E, 1, 4, DBG>;
+        case 2: return words == 2 ? ll_small_kernel<E, 2, 2, DBG> : ll_small_kernel<E, 2, 4, DBG>;
+        case 4: return words == 2 ? ll_small_kernel<E, 4, 2, DBG> : ll_small_kernel<E, 4, 4, DBG>;
+        case 8: return words == 2 ? ll_small_kernel<E, 8, 2, DBG> : ll_small_kernel<E, 8, 4, DBG>;
+    }
+    return nullptr;
+}
+
+KernelFn ll_small_kernel_for(int dtype, int P, int words, bool dbg)
+{
+    if (dtype == SYMAR_F32) return dbg ? pick_ll_small_ranks<F32, true>(P, words) : pick_ll_small_ranks<F32, false>(P, words);
+    if (dtype == SYMAR_BF16) return dbg ? pick_ll_small_ranks<BF16, true>(P, words) : pick_ll_small_ranks<BF16, false>(P, words);
     return nullptr;
 }
 

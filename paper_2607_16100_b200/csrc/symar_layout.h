@@ -40,8 +40,10 @@ __host__ __device__ constexpr size_t done_count_off(int c) { return (size_t)kMax
 
 // Variant bits carried in KArgs::variant (every variant computes the same bits):
 //   one-shot : bits 8-9 = bytes per thread (0: 16, 1: 8, 2: 4); bit 14 = prior-art form with two
-//              memory-ordering barriers (comparison only, never chosen)
-//   LL       : bit 8    = 8 instead of 16 payload bytes per thread
+//              memory-ordering barriers, bit 15 = release on the ready signal (comparison only,
+//              never chosen)
+//   LL       : bit 8    = 8 instead of 16 payload bytes per thread; bit 9 = never the single-iteration
+//              kernel; bits 12-15 = cycles / 64 the single-iteration kernel holds back its first poll
 //   two-shot : bit 0 = contiguous chunks for large messages, bit 1 = 16-byte accesses,
 //              bit 2 = never the bulk-copy kernel, bits 8-10 = bulk pipeline depth,
 //              bits 12-13 = log2(bulk tile size / 4 KiB)
@@ -63,7 +65,10 @@ __host__ __device__ constexpr size_t bulk_smem_bytes(int P, uint32_t tile_vecs, 
 
 // control block words (u32)
 enum : int { kCtlCode = 0, kCtlRank = 1, kCtlPeer = 2, kCtlCta = 3,
-             kCtlSpanIn = 16, kCtlSpanOut = 18 };   // two u64 (byte 64, 72): first CTA in, last CTA out (test hook)
+             kCtlSpanIn = 16, kCtlSpanOut = 18,     // two u64 (byte 64, 72): first CTA in, last CTA out (test hook)
+             // phase stamps (test hook): kPhases u64 each -- earliest, latest, wrapping sum, number of stamps
+             kCtlPhaseMin = 64, kCtlPhaseMax = 80, kCtlPhaseSum = 96, kCtlPhaseCnt = 112 };
+constexpr int kPhases = 8;
 
 __host__ __device__ constexpr size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 

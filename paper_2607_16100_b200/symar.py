@@ -7,11 +7,14 @@ or fails to load this module raises -- there is no fallback of any kind.
 from __future__ import annotations
 
 import ctypes
+import os
 from ctypes import POINTER, byref, c_char_p, c_double, c_int, c_size_t, c_uint, c_void_p
 from pathlib import Path
 
 _PKG = Path(__file__).resolve().parent
-LIB_PATH = _PKG / "libsymar.so"
+# SYMAR_LIB selects another build of the same library (the system-scope or the bounds-checking
+# flavour of paper_2607_16100_b200/build.py); by default the regular one.
+LIB_PATH = Path(os.environ["SYMAR_LIB"]) if os.environ.get("SYMAR_LIB") else _PKG / "libsymar.so"
 
 F32, BF16 = 0, 1
 AUTO, ONESHOT, TWOSHOT, LL, SENTINEL, TWOSHOT_LL, TWOSHOT_SENTINEL, TWOSHOT_ATOMIC = 0, 1, 2, 3, 4, 5, 6, 7
@@ -68,6 +71,8 @@ SIGNATURES = [
     ("symar_probe_pingpong", c_int, [c_int, POINTER(c_double)]),
     ("symar_probe_pingpong_pair", c_int, [c_int, c_int, POINTER(c_double), POINTER(c_int)]),
     ("symar_debug_span", c_int, [c_void_p, c_void_p, c_void_p, c_size_t, c_int, c_int, c_void_p, POINTER(c_double)]),
+    ("symar_debug_phases", c_int, [c_void_p, c_void_p, c_void_p, c_size_t, c_int, c_int, c_void_p, POINTER(c_double),
+                                   POINTER(c_int)]),
     ("symar_probe_barrier", c_int, [c_int, c_int, c_int, POINTER(c_double)]),
     ("symar_llbuffer_bytes", c_size_t, [c_int, c_size_t, c_size_t, c_int, c_int]),
     ("symar_llbuffer_init_sentinel", c_int, [c_void_p, c_size_t, c_void_p]),
@@ -311,6 +316,16 @@ class SymHeap:
         _ck(self._lib.symar_debug_span(self._h, self.rank_ptr(0, in_off), self.rank_ptr(0, out_off), count, dtype,
                                        algo, stream, byref(v)), "symar_debug_span")
         return v.value
+
+    def debug_phases(self, in_off: int, out_off: int, count: int, dtype: int, algo: int = AUTO, stream: int = 0):
+        """Per phase k = 0..7 of one synchronous call: (earliest, mean, latest) ns since the first CTA's
+        start, and how many CTAs stamped it; phases the kernel does not have are left out."""
+        ns = (c_double * 24)()
+        n = (c_int * 8)()
+        _ck(self._lib.symar_debug_phases(self._h, self.rank_ptr(0, in_off), self.rank_ptr(0, out_off), count, dtype,
+                                         algo, stream, ns, n), "symar_debug_phases")
+        return {k: {"first": ns[3 * k], "mean": ns[3 * k + 1], "last": ns[3 * k + 2], "ctas": n[k]}
+                for k in range(8) if n[k] > 0}
 
     def debug_inject(self, mute_rank: int = -1, delay_seed: int = 0, delay_max_ns: int = 0) -> None:
         _ck(self._lib.symar_debug_inject(self._h, mute_rank, delay_seed, delay_max_ns), "symar_debug_inject")

@@ -25,7 +25,7 @@ def lib():
     return symar.load()
 
 
-def test_header_declares_the_three_north_star_calls():
+def test_header_declares_the_three_core_calls():
     names = declared_functions()
     for must in ("symheap_create", "allreduce", "allreduce_autotune"):
         assert must in names

@@ -62,6 +62,40 @@ def test_c2_and_c3_message_sweep_p8_bf16():
         h.destroy()
 
 
+def test_pruned_tuner_is_quick_and_finds_what_the_exhaustive_search_finds(monkeypatch):
+    # The tuner skips algorithms that lost clearly one size down and searches shapes around the previous
+    # winner.  It must stay within seconds, and at every c3 size its choice must be as fast as the best
+    # entry of a search that prunes nothing (each tuner's own timings; 8 % covers their run-to-run noise).
+    import time
+    w = synth.WORKLOADS["c3"]
+    h = symar.SymHeap.on_torch(8, 24 << 20)
+    monkeypatch.setenv("SYMAR_TUNE", "exhaustive")
+    g = symar.SymHeap.on_torch(8, 24 << 20)
+    monkeypatch.delenv("SYMAR_TUNE")
+    try:
+        t0 = time.perf_counter()
+        h.autotune(symar.BF16)
+        quick = time.perf_counter() - t0
+        t0 = time.perf_counter()
+        g.autotune(symar.BF16)
+        full = time.perf_counter() - t0
+        assert quick < 5.0, (quick, full)
+        for B in w["batch"]:
+            count = w["count"] * B
+            log2 = (count * 2 - 1).bit_length()
+            algo = h.query_choice(count, symar.BF16)[0]
+            mine = h.tuned_entry(symar.BF16, log2, algo)[2]
+            best = min(g.tuned_entry(symar.BF16, log2, a)[2] for a in ALGOS[:-1])
+            assert mine <= 1.08 * best, (B, algo, mine, best)
+            # and it is the same algorithm, unless two are within that noise of each other
+            theirs = g.query_choice(count, symar.BF16)[0]
+            assert algo == theirs or g.tuned_entry(symar.BF16, log2, algo)[2] <= 1.08 * best, (B, algo, theirs)
+    finally:
+        torch.cuda.synchronize()
+        h.destroy()
+        g.destroy()
+
+
 def test_c4_full_size_p8_fp32_256MiB():
     w = synth.WORKLOADS["c4"]
     P, count = w["P"], w["count"]

@@ -203,11 +203,17 @@ FORCE_PLAIN = 1 << 31
 @pytest.mark.parametrize("P,dtype,dist", [(8, "bf16", "normal"), (4, "f32", "uniform"), (2, "bf16", "normal"),
                                           (1, "f32", "uniform")])
 @pytest.mark.parametrize("algo,variant", [(symar.ONESHOT, FORCE_PLAIN), (symar.ONESHOT, 0x100),
-                                          (symar.ONESHOT, 0x200), (symar.LL, FORCE_PLAIN), (symar.LL, 0x100),
+                                          (symar.ONESHOT, 0x200),
+                                          # release on the ready signal (comparison variant)
+                                          (symar.ONESHOT, 0x8100), (symar.ONESHOT, 0x8000),
+                                          # LL: single-iteration kernel where it fits (16 / 8 payload bytes per
+                                          # thread, first poll held back), and the general kernel (bit 9)
+                                          (symar.LL, FORCE_PLAIN), (symar.LL, 0x100), (symar.LL, 0x3100),
+                                          (symar.LL, 0xC000), (symar.LL, 0x200), (symar.LL, 0x300),
                                           (symar.SENTINEL, FORCE_PLAIN), (symar.TWOSHOT_LL, FORCE_PLAIN),
                                           (symar.TWOSHOT_SENTINEL, FORCE_PLAIN)])
 def test_unit_width_variants(heaps, algo, variant, P, dtype, dist, count):
-    # 16, 8 or 4 bytes per thread: same bits, whatever the ragged tail
+    # every implementation variant of a kernel gives the same bits, whatever the ragged tail
     h = heaps[P]
     x = synth.make_inputs(dist, dtype, P, count, seed=31 * count + P)
     h.set_variant(algo, variant)
@@ -538,6 +544,29 @@ def test_bounded_wait_reports_timeout_and_heap_recovers(algo):
         h.reset()
         got = run(h, x, symar.BF16, algo)
         assert_bits(got, O.allreduce(x))
+    finally:
+        torch.cuda.synchronize()
+        h.destroy()
+
+
+@pytest.mark.parametrize("algo", [symar.ONESHOT, symar.LL, symar.TWOSHOT])
+def test_default_wait_bound_is_a_fraction_of_a_second(algo):
+    # With the library's default bound, a wait that can never end gives up well within a second
+    # (a GPU that other work shares must not be held for long) and says so in the status word.
+    import time
+    h = symar.SymHeap.on_torch(4, 1 << 20)
+    try:
+        x = synth.make_inputs("normal", "bf16", 4, 4096, seed=9)
+        for q in range(4):
+            h.write_rank(q, 0, x[q])
+        h.debug_inject(1, 0, 0)
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        h.allreduce(0, 65536, 4096, symar.BF16, algo)
+        torch.cuda.synchronize()
+        took = time.perf_counter() - t0
+        assert h.status()[0] == symar.ERR_TIMEOUT
+        assert 0.05 < took < 0.9, took
     finally:
         torch.cuda.synchronize()
         h.destroy()
