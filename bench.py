@@ -292,6 +292,50 @@ def scope_probe(shapes_json, quick):
     print(json.dumps(out))
 
 
+def run_case(spec, steps, warmup):
+    """`--case ALGO:BYTES[:P[:VARIANT[:CTAS:THREADS]]]`: a few stream-launched calls of ONE algorithm on a
+    bf16 message of BYTES per rank, checked against the oracle -- a small, self-ending command for
+    profilers (a few MiB on the device, `warmup` + `steps` launches)."""
+    import torch
+    from oracle import allreduce_oracle as O
+    from paper_2607_16100_b200 import symar, synth
+    f = spec.split(":")
+    algo = {v: k for k, v in symar.ALGO_NAMES.items()}[f[0]]
+    nbytes = int(f[1])
+    P = int(f[2]) if len(f) > 2 else 8
+    variant = int(f[3], 0) if len(f) > 3 else 0
+    ctas, threads = (int(f[4]), int(f[5])) if len(f) > 5 else (0, 0)
+    count = nbytes // 2
+    out_off = (nbytes + 4095) // 4096 * 4096
+    h = symar.SymHeap.on_torch(P, max(2 * out_off, 1 << 16))
+    x = synth.make_inputs("normal", "bf16", P, count, synth.seed_for_config(2))
+    for q in range(P):
+        h.write_rank(q, 0, x[q])
+    if variant:
+        h.set_variant(algo, variant)
+    if ctas or threads:
+        h.set_launch(algo, ctas, threads)
+    stream = torch.cuda.Stream()
+    call = lambda: h.allreduce(0, out_off, count, symar.BF16, algo, stream.cuda_stream)
+    for _ in range(max(1, warmup)):
+        call()
+    stream.synchronize()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with torch.cuda.stream(stream):
+        a.record(stream)
+        for _ in range(steps):
+            call()
+        b.record(stream)
+    stream.synchronize()
+    got = np.stack([h.read_rank(q, out_off, count, np.uint16) for q in range(P)])
+    al, c, t = h.last_choice()
+    print(json.dumps({"case": spec, "algo": symar.ALGO_NAMES[al], "ctas_per_rank": c, "threads": t,
+                      "variant": h.last_kernel()[0], "launches": max(1, warmup) + steps,
+                      "stream_launched_us_per_call": a.elapsed_time(b) * 1000.0 / steps,
+                      "bit_exact": bool(np.array_equal(got, O.allreduce(x))) and h.status()[0] == 0}))
+    h.destroy()
+
+
 def latency_suite(torch, symar, synth, hbm_gbs, quick=False, autotune=True):
     """C2 (16 KiB vs SoL), C3 (sweep + selector), C5 (decode-step graph)."""
     from oracle import allreduce_oracle as O
@@ -832,6 +876,8 @@ def main():
     ap.add_argument("--variant", type=lambda v: int(v, 0), default=0, help="two-shot kernel variant bits")
     ap.add_argument("--out-dir", default=str(ROOT / "gpurun_out"), help="where the per-workload result files go")
     ap.add_argument("--scope-probe", default=None, help=argparse.SUPPRESS)     # child process of the latency section
+    ap.add_argument("--case", default=None, help="ALGO:BYTES[:P[:VARIANT[:CTAS:THREADS]]] -- a few calls of one "
+                                                 "algorithm on a bf16 message (for profilers); --steps calls, default 5")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -840,6 +886,11 @@ def main():
         return
     if args.scope_probe:
         scope_probe(args.scope_probe, args.quick)
+        return
+    if args.case:
+        import __graft_entry__ as ge
+        ge.build()
+        run_case(args.case, args.steps if args.steps != 500 else 5, args.warmup)
         return
 
     import torch

@@ -371,6 +371,19 @@ int symar_debug_span(symheap_t *heap, const void *in, void *out, size_t count, s
 int symar_debug_phases(symheap_t *heap, const void *in, void *out, size_t count, symar_dtype_t dtype,
                        symar_algo_t algo, void *cuda_stream, double *host_ns, int *host_stamps);
 
+/* Self-test of the bounds-checking build of the library (libsymar_check.so, compiled with
+ * -DSYMAR_CHECK: every heap address a kernel computes is checked against the region it must
+ * lie in -- this call's input or output range, the LL, sentinel or atomic scratch, the flag
+ * arrays, the counters -- and an access outside is recorded as SYMAR_ERR_INVAL in the status
+ * word (rank, CTA slot, and in place of the peer the bit mask of the regions it was meant for:
+ * 1 input, 2 output, 4 LL, 8 sentinel, 16 atomic scratch, 32 ready flags, 64 done flags,
+ * 128 counters) and SKIPPED).  One CTA stores once inside a 64-byte output range and once
+ * 64 bytes beyond it, at an address that is still inside the heap's user region (bytes 1024..1151
+ * of rank 0; the heap needs 4 KiB per rank), so nothing can fault either way.  SYMAR_OK: the
+ * first store landed, the second was recorded and kept out; SYMAR_ERR_UNSUPPORTED: this is
+ * the regular build, which checks nothing.  Synchronous; clears the status word.          */
+int symar_check_selftest(symheap_t *heap, void *cuda_stream);
+
 /* Text of the last CUDA error seen by the library on this thread (host string). */
 const char *symar_last_cuda_error(void);
 

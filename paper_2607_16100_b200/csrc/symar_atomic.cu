@@ -46,6 +46,7 @@ namespace {
 
 __device__ __forceinline__ void red_add_v4_f32(void *p, float a, float b, float c, float d)
 {
+    p = SYMAR_PTR(p, 16, kRegAt);
     asm volatile("red.relaxed." SYMAR_SCOPE ".global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(p), "f"(a), "f"(b),
                  "f"(c), "f"(d)
                  : "memory");
@@ -54,19 +55,22 @@ __device__ __forceinline__ void red_add_v4_f32(void *p, float a, float b, float 
 template <typename E> struct Elem;
 template <> struct Elem<F32> {
     using T = float;
-    __device__ static __forceinline__ float load(const char *p) { return __ldg(reinterpret_cast<const float *>(p)); }
-    __device__ static __forceinline__ void store(char *p, float v) { *reinterpret_cast<float *>(p) = v; }
+    __device__ static __forceinline__ float load(const char *p)
+    {
+        return __ldg(SYMAR_PTR(reinterpret_cast<const float *>(p), 4, kRegIn));
+    }
+    __device__ static __forceinline__ void store(char *p, float v) { *SYMAR_PTR(reinterpret_cast<float *>(p), 4, kRegOut) = v; }
 };
 template <> struct Elem<BF16> {
     using T = uint16_t;
     __device__ static __forceinline__ float load(const char *p)
     {
-        return __uint_as_float((uint32_t)__ldg(reinterpret_cast<const unsigned short *>(p)) << 16);
+        return __uint_as_float((uint32_t)__ldg(SYMAR_PTR(reinterpret_cast<const unsigned short *>(p), 2, kRegIn)) << 16);
     }
     __device__ static __forceinline__ void store(char *p, float v)
     {
         __nv_bfloat16 h = __float2bfloat16_rn(v);
-        *reinterpret_cast<uint16_t *>(p) = *reinterpret_cast<uint16_t *>(&h);
+        *SYMAR_PTR(reinterpret_cast<uint16_t *>(p), 2, kRegOut) = *reinterpret_cast<uint16_t *>(&h);
     }
 };
 
@@ -77,12 +81,13 @@ __global__ void __launch_bounds__(kMaxThreads) twoshot_atomic_kernel(const KArgs
 {
     using El = Elem<E>;
     constexpr uint32_t es = sizeof(typename El::T);
+    SYMAR_CHECK_BEGIN(a, P, a.count * es, a.count * es);
     const int c = blockIdx.x, r = blockIdx.y, C = gridDim.x;
     const uint32_t t = threadIdx.x, T = blockDim.x;
     const uint32_t j = t & 7u;                       // position in the 8-thread group of a line
     const uint32_t g = t >> 3, G = T >> 3;           // group index, groups per CTA
     char *seg_r      = a.seg0 + (size_t)r * a.stride;
-    uint32_t *dcount = reinterpret_cast<uint32_t *>(seg_r + a.epoch_off + done_count_off(c));
+    uint32_t *dcount = SYMAR_PTR(reinterpret_cast<uint32_t *>(seg_r + a.epoch_off + done_count_off(c)), 4, kRegCtr);
     if (a.pdl) {
         pdl_wait();                                  // the previous call has left the heap
         pdl_launch_dependents();

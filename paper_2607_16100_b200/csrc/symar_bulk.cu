@@ -79,6 +79,7 @@ template <typename E, int P>
 __global__ void __launch_bounds__(kMaxThreads) twoshot_bulk_kernel(const KArgs a)
 {
     extern __shared__ __align__(128) unsigned char smem[];
+    SYMAR_CHECK_BEGIN_ALLREDUCE(a, P);
     const int c = blockIdx.x, r = blockIdx.y, C = gridDim.x;
     const uint32_t t = threadIdx.x, T = blockDim.x;
     const uint32_t S = a.stages, TV = a.tile_vecs, TB = TV * 16u;
@@ -87,8 +88,8 @@ __global__ void __launch_bounds__(kMaxThreads) twoshot_bulk_kernel(const KArgs a
     unsigned char *out_tiles = in_tiles + (size_t)S * P * TB;               // [kBulkOutBufs][TB]
 
     char *seg_r = a.seg0 + (size_t)r * a.stride;
-    uint32_t *rcount = reinterpret_cast<uint32_t *>(seg_r + a.epoch_off + ready_count_off(c));
-    uint32_t *dcount = reinterpret_cast<uint32_t *>(seg_r + a.epoch_off + done_count_off(c));
+    uint32_t *rcount = SYMAR_PTR(reinterpret_cast<uint32_t *>(seg_r + a.epoch_off + ready_count_off(c)), 4, kRegCtr);
+    uint32_t *dcount = SYMAR_PTR(reinterpret_cast<uint32_t *>(seg_r + a.epoch_off + done_count_off(c)), 4, kRegCtr);
 
     if (t == 0) {
         for (uint32_t s = 0; s < S; ++s) mbar_init(&full[s], 1);
@@ -115,11 +116,17 @@ __global__ void __launch_bounds__(kMaxThreads) twoshot_bulk_kernel(const KArgs a
         const uint32_t s   = (uint32_t)(i % S);
         const uint64_t v0  = tile_first(i);
         const uint32_t nb  = tile_count(v0) * 16u;
-        mbar_expect_tx(&full[s], nb * P);
+        // (checking build: a tile outside the call's input range is not copied, and not waited for)
+        uint32_t good = 0;
 #pragma unroll
         for (int q = 0; q < P; ++q)
-            bulk_load(in_tiles + ((size_t)s * P + q) * TB, a.seg0 + (size_t)q * a.stride + a.in_off + v0 * 16, nb,
-                      &full[s]);
+            good += SYMAR_RANGE_OK(a.seg0 + (size_t)q * a.stride + a.in_off + v0 * 16, nb, kRegIn) ? 1u : 0u;
+        mbar_expect_tx(&full[s], nb * good);
+#pragma unroll
+        for (int q = 0; q < P; ++q)
+            if (good == (uint32_t)P || SYMAR_RANGE_OK(a.seg0 + (size_t)q * a.stride + a.in_off + v0 * 16, nb, kRegIn))
+                bulk_load(in_tiles + ((size_t)s * P + q) * TB, a.seg0 + (size_t)q * a.stride + a.in_off + v0 * 16, nb,
+                          &full[s]);
     };
 
     if (ok && t == 0)
@@ -162,7 +169,8 @@ __global__ void __launch_bounds__(kMaxThreads) twoshot_bulk_kernel(const KArgs a
             // all-gather: the reduced tile leaves shared memory once per rank
 #pragma unroll
             for (int q = 0; q < P; ++q)
-                bulk_store(a.seg0 + (size_t)q * a.stride + a.out_off + v0 * 16, ot, nvt * 16u);
+                if (SYMAR_RANGE_OK(a.seg0 + (size_t)q * a.stride + a.out_off + v0 * 16, nvt * 16u, kRegOut))
+                    bulk_store(a.seg0 + (size_t)q * a.stride + a.out_off + v0 * 16, ot, nvt * 16u);
             bulk_commit();
             // The output tile written two trips from now is the one stored in the
             // previous trip: let all but the newest store finish reading.

@@ -29,6 +29,7 @@ template <> struct Unit<2> {
     __device__ static __forceinline__ Unit ld(const char *p)
     {
         Unit u;
+        p = SYMAR_PTR(p, 2, kRegIn);
         asm volatile("ld.relaxed." SYMAR_SCOPE ".global.u16 %0, [%1];" : "=h"(u.v) : "l"(p) : "memory");
         return u;
     }
@@ -47,7 +48,7 @@ __device__ __forceinline__ void st_unit(char *p, const Unit<4> &u, uint32_t vali
 }
 __device__ __forceinline__ void st_unit(char *p, const Unit<2> &u, uint32_t)
 {
-    *reinterpret_cast<uint16_t *>(p) = u.v;
+    *SYMAR_PTR(reinterpret_cast<uint16_t *>(p), 2, kRegOut) = u.v;
 }
 
 template <typename E, int P>
@@ -118,11 +119,13 @@ __device__ __forceinline__ void coll_body(const CollArgs &a, int r, uint64_t fir
 template <typename E, int P, int OP>
 __global__ void __launch_bounds__(kMaxThreads) coll_kernel(const CollArgs a)
 {
+    // input and output sizes per rank: ReduceScatter reads P chunks, AllGather writes P
+    SYMAR_CHECK_BEGIN(a.k, P, OP == kOpReduceScatter ? a.bytes * P : a.bytes, OP == kOpAllGather ? a.bytes * P : a.bytes);
     const int c = blockIdx.x, r = blockIdx.y, C = gridDim.x;
     const uint32_t t = threadIdx.x, T = blockDim.x;
     const KArgs &k = a.k;
     char *seg_r = k.seg0 + (size_t)r * k.stride;
-    uint32_t *count = reinterpret_cast<uint32_t *>(seg_r + k.epoch_off + ready_count_off(c));
+    uint32_t *count = SYMAR_PTR(reinterpret_cast<uint32_t *>(seg_r + k.epoch_off + ready_count_off(c)), 4, kRegCtr);
     if (k.pdl) pdl_wait();
 
     uint32_t want;

@@ -11,6 +11,105 @@
 
 namespace symar {
 
+// ---- bounds-checking debug build (-DSYMAR_CHECK) -------------------------------------
+// Every global-memory helper below passes its address through SYMAR_PTR(p, bytes, regions):
+// in the regular build that is `p`; in the checking build the access must lie wholly inside one
+// of the named regions of some rank's segment (for the user region: inside THIS call's input
+// or output range), else the violation is recorded -- SYMAR_ERR_INVAL in the heap's status word
+// with the rank, the CTA slot and the regions the access was meant for -- and the access is
+// SKIPPED: it is redirected to a small sink array, so that nothing outside the sink is read or
+// written.  Stands in for a memory checker where none can be run.
+enum : uint32_t { kRegIn = 1, kRegOut = 2, kRegLL = 4, kRegSn = 8, kRegAt = 16, kRegReady = 32, kRegDone = 64,
+                  kRegCtr = 128 };
+#ifdef SYMAR_CHECK
+struct CheckCtx {
+    const char *base;            // rank 0's segment (nullptr: no heap); the ranges below repeat every `stride`
+    uint64_t    stride;
+    uint32_t    nranks, nreg, nabs;
+    uint64_t    lo[8], hi[8];    // segment-relative byte ranges
+    uint32_t    kind[8];
+    const char *alo[4], *ahi[4]; // absolute ranges (buffers outside a heap)
+    uint32_t    akind[4];
+    uint32_t   *ctl;             // heap status words, or nullptr
+    uint32_t   *status;          // a caller's status word, or nullptr
+};
+static __device__ __align__(32) unsigned char g_check_sink[64 * 32];
+__device__ __forceinline__ CheckCtx &check_ctx()
+{
+    __shared__ CheckCtx ctx;
+    return ctx;
+}
+static __device__ __noinline__ void check_fail(const CheckCtx &c, uint32_t allowed)
+{
+    if (c.ctl && atomicCAS(&c.ctl[kCtlCode], 0u, (uint32_t)SYMAR_ERR_INVAL) == 0u) {
+        c.ctl[kCtlRank] = blockIdx.y;
+        c.ctl[kCtlPeer] = allowed;
+        c.ctl[kCtlCta]  = blockIdx.x;
+        __threadfence();
+    }
+    if (c.status) atomicCAS(c.status, 0u, (uint32_t)SYMAR_ERR_INVAL);
+}
+static __device__ __noinline__ bool check_range(const void *p, uint64_t bytes, uint32_t allowed)
+{
+    const CheckCtx &c = check_ctx();
+    const char *q     = reinterpret_cast<const char *>(p);
+    bool ok           = false;
+    if (c.base && q >= c.base && (uint64_t)(q - c.base) < c.stride * c.nranks) {
+        const uint64_t o = (uint64_t)(q - c.base) % c.stride;
+        for (uint32_t i = 0; i < c.nreg; ++i) ok = ok || ((c.kind[i] & allowed) && o >= c.lo[i] && o + bytes <= c.hi[i]);
+    }
+    for (uint32_t i = 0; i < c.nabs; ++i) ok = ok || ((c.akind[i] & allowed) && q >= c.alo[i] && q + bytes <= c.ahi[i]);
+    if (!ok) check_fail(c, allowed);
+    return ok;
+}
+template <typename T>
+__device__ __forceinline__ T *check_ptr(T *p, uint64_t bytes, uint32_t allowed)
+{
+    if (check_range(p, bytes, allowed)) return p;
+    return reinterpret_cast<T *>(g_check_sink + (threadIdx.x & 63u) * 32u);
+}
+// First statement of every kernel on a heap (all threads): the regions of this call.
+__device__ __forceinline__ void check_begin(const KArgs &a, int nranks, uint64_t in_bytes, uint64_t out_bytes)
+{
+    if (threadIdx.x == 0) {
+        CheckCtx &c = check_ctx();
+        c.base   = a.seg0;
+        c.stride = a.stride;
+        c.nranks = (uint32_t)nranks;
+        c.nabs   = 0;
+        c.ctl    = a.ctl;
+        c.status = nullptr;
+        const uint64_t lo[8]   = {a.in_off, a.out_off, a.ll_off, a.sn_off, a.at_off, a.ready_off, a.done_off, a.epoch_off};
+        const uint64_t hi[8]   = {a.in_off + (in_bytes + 15) / 16 * 16,   // whole vectors are read (the region is padded)
+                                  a.out_off + out_bytes, a.sn_off, a.at_off, a.ready_off, a.done_off, a.epoch_off,
+                                  a.epoch_off + (uint64_t)kMaxCtas * 16};
+        const uint32_t kind[8] = {kRegIn, kRegOut, kRegLL, kRegSn, kRegAt, kRegReady, kRegDone, kRegCtr};
+        c.nreg = 8;
+        for (int i = 0; i < 8; ++i) {
+            c.lo[i]   = lo[i];
+            c.hi[i]   = hi[i];
+            c.kind[i] = kind[i];
+        }
+    }
+    __syncthreads();
+}
+// message bytes of an AllReduce call
+__device__ __forceinline__ uint64_t check_message_bytes(const KArgs &a)
+{
+    return a.tail_bytes ? (a.nvec - 1) * 16 + a.tail_bytes : a.nvec * 16;
+}
+#define SYMAR_CHECK_BEGIN(a, nranks, in_bytes, out_bytes) symar::check_begin(a, nranks, in_bytes, out_bytes)
+#define SYMAR_CHECK_BEGIN_ALLREDUCE(a, nranks) \
+    symar::check_begin(a, nranks, symar::check_message_bytes(a), symar::check_message_bytes(a))
+#define SYMAR_PTR(p, bytes, regions) symar::check_ptr(p, bytes, regions)
+#define SYMAR_RANGE_OK(p, bytes, regions) symar::check_range(p, bytes, regions)
+#else
+#define SYMAR_CHECK_BEGIN(a, nranks, in_bytes, out_bytes) ((void)0)
+#define SYMAR_CHECK_BEGIN_ALLREDUCE(a, nranks) ((void)0)
+#define SYMAR_PTR(p, bytes, regions) (p)
+#define SYMAR_RANGE_OK(p, bytes, regions) true
+#endif
+
 // ---- memory operations -------------------------------------------------------
 // On one device `.gpu` scope is sufficient; a multi-GPU build of the same
 // protocol would use `.sys`.  Compiling with -DSYMAR_SCOPE_SYS gives that build
@@ -24,16 +123,19 @@ namespace symar {
 
 __device__ __forceinline__ uint32_t ld_acquire_u32(const uint32_t *p)
 {
+    p = SYMAR_PTR(p, 4, kRegReady | kRegDone);
     uint32_t v;
     asm volatile("ld.acquire." SYMAR_SCOPE ".global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
     return v;
 }
 __device__ __forceinline__ void st_release_u32(uint32_t *p, uint32_t v)
 {
+    p = SYMAR_PTR(p, 4, kRegReady | kRegDone);
     asm volatile("st.release." SYMAR_SCOPE ".global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
 __device__ __forceinline__ uint32_t ld_relaxed_u32(const uint32_t *p)
 {
+    p = SYMAR_PTR(p, 4, kRegCtr | kRegIn);
     uint32_t v;
     asm volatile("ld.relaxed." SYMAR_SCOPE ".global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
     return v;
@@ -42,10 +144,12 @@ __device__ __forceinline__ uint32_t ld_relaxed_u32(const uint32_t *p)
 // this thread (and, through the preceding CTA barrier, of its CTA) before it.
 __device__ __forceinline__ void red_release_inc_u32(uint32_t *p)
 {
+    p = SYMAR_PTR(p, 4, kRegReady | kRegDone);
     asm volatile("red.release." SYMAR_SCOPE ".global.add.u32 [%0], 1;" ::"l"(p) : "memory");
 }
 __device__ __forceinline__ void red_relaxed_inc_u32(uint32_t *p)
 {
+    p = SYMAR_PTR(p, 4, kRegReady | kRegDone);
     asm volatile("red.relaxed." SYMAR_SCOPE ".global.add.u32 [%0], 1;" ::"l"(p) : "memory");
 }
 __device__ __forceinline__ void fence_acq_rel()
@@ -54,6 +158,7 @@ __device__ __forceinline__ void fence_acq_rel()
 }
 __device__ __forceinline__ uint64_t ld_relaxed_u64(const uint64_t *p)
 {
+    p = SYMAR_PTR(p, 8, kRegCtr);
     uint64_t v;
     asm volatile("ld.relaxed." SYMAR_SCOPE ".global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
     return v;
@@ -66,11 +171,13 @@ struct __align__(16) U64x2 { uint64_t a, b; };
 
 __device__ __forceinline__ void st_relaxed_v2u64(void *p, uint64_t a, uint64_t b)
 {
+    p = SYMAR_PTR(p, 16, kRegLL);
     asm volatile("st.relaxed." SYMAR_SCOPE ".global.v2.u64 [%0], {%1, %2};" ::"l"(p), "l"(a), "l"(b)
                  : "memory");
 }
 __device__ __forceinline__ U64x2 ld_relaxed_v2u64(const void *p)
 {
+    p = SYMAR_PTR(p, 16, kRegLL);
     U64x2 v;
     asm volatile("ld.relaxed." SYMAR_SCOPE ".global.v2.u64 {%0, %1}, [%2];"
                  : "=l"(v.a), "=l"(v.b)
@@ -82,12 +189,14 @@ __device__ __forceinline__ U64x2 ld_relaxed_v2u64(const void *p)
 // 16-byte strong accesses of four 32-bit elements (each element a single access)
 __device__ __forceinline__ void st_relaxed_v4(void *p, const uint4 &v)
 {
+    p = SYMAR_PTR(p, 16, kRegSn | kRegAt);
     asm volatile("st.relaxed." SYMAR_SCOPE ".global.v4.u32 [%0], {%1, %2, %3, %4};" ::"l"(p), "r"(v.x), "r"(v.y),
                  "r"(v.z), "r"(v.w)
                  : "memory");
 }
 __device__ __forceinline__ uint4 ld_relaxed_v4(const void *p)
 {
+    p = SYMAR_PTR(p, 16, kRegSn | kRegAt);
     uint4 v;
     asm volatile("ld.relaxed." SYMAR_SCOPE ".global.v4.u32 {%0, %1, %2, %3}, [%4];"
                  : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
@@ -100,6 +209,7 @@ __device__ __forceinline__ uint4 ld_relaxed_v4(const void *p)
 // read-only path, no L1 allocation.
 __device__ __forceinline__ uint4 ld_own(const void *p)
 {
+    p = SYMAR_PTR(p, 16, kRegIn);
     uint4 v;
     asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];"
                  : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
@@ -111,6 +221,7 @@ __device__ __forceinline__ uint4 ld_own(const void *p)
 // cached before the signal.
 __device__ __forceinline__ uint4 ld_peer(const void *p)
 {
+    p = SYMAR_PTR(p, 16, kRegIn);
     uint4 v;
     asm volatile("ld.relaxed." SYMAR_SCOPE ".global.v4.u32 {%0, %1, %2, %3}, [%4];"
                  : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
@@ -121,6 +232,7 @@ __device__ __forceinline__ uint4 ld_peer(const void *p)
 // Outputs are written once and not re-read by this kernel.
 __device__ __forceinline__ void st_output(void *p, uint4 v)
 {
+    p = SYMAR_PTR(p, 16, kRegOut);
     asm volatile("st.global.cs.v4.u32 [%0], {%1, %2, %3, %4};" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z),
                  "r"(v.w)
                  : "memory");
@@ -132,6 +244,7 @@ __device__ __forceinline__ void st_output(void *p, uint4 v)
 struct U32B { uint4 lo, hi; };
 __device__ __forceinline__ U32B ld_peer_32B(const void *p)
 {
+    p = SYMAR_PTR(p, 32, kRegIn);
     U32B v;
     asm volatile("ld.global.L1::no_allocate.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
                  : "=r"(v.lo.x), "=r"(v.lo.y), "=r"(v.lo.z), "=r"(v.lo.w), "=r"(v.hi.x), "=r"(v.hi.y),
@@ -142,6 +255,7 @@ __device__ __forceinline__ U32B ld_peer_32B(const void *p)
 }
 __device__ __forceinline__ void st_output_32B(void *p, const U32B &v)
 {
+    p = SYMAR_PTR(p, 32, kRegOut);
     asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(p), "r"(v.lo.x), "r"(v.lo.y),
                  "r"(v.lo.z), "r"(v.lo.w), "r"(v.hi.x), "r"(v.hi.y), "r"(v.hi.z), "r"(v.hi.w)
                  : "memory");
@@ -170,7 +284,19 @@ __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepc
 
 // L2 prefetch hint.  Safe on memory that an earlier kernel may still be writing: no data
 // is returned, and L2 is the point of coherence, so a later write simply updates the line.
-__device__ __forceinline__ void prefetch_l2(const void *p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
+__device__ __forceinline__ void prefetch_l2(const void *p)
+{
+    p = SYMAR_PTR(p, 1, kRegIn);
+    asm volatile("prefetch.global.L2 [%0];" ::"l"(p));
+}
+
+// a short, bounded pause (holding back a poll that would only arrive before its data)
+__device__ __forceinline__ void idle_cycles(uint32_t cycles)
+{
+    if (cycles == 0) return;
+    const uint32_t c0 = (uint32_t)clock();
+    while ((uint32_t)clock() - c0 < cycles) { /* bounded by `cycles` */ }
+}
 
 // ---- bounded waiting ------------------------------------------------------------
 // Counts polls in a register; every 256th poll reads the nanosecond timer.  The
@@ -282,6 +408,7 @@ template <int W> struct Words { uint32_t w[W]; };
 template <int W>
 __device__ __forceinline__ Words<W> ld_peer_words(const void *p)
 {
+    p = SYMAR_PTR(p, 4 * W, kRegIn);
     Words<W> v;
     if (W == 1)
         asm volatile("ld.relaxed." SYMAR_SCOPE ".global.u32 %0, [%1];" : "=r"(v.w[0]) : "l"(p) : "memory");
@@ -331,6 +458,7 @@ __device__ __forceinline__ Words<W> reduce_words_in_rank_order(const Words<W> (&
 template <int W>
 __device__ __forceinline__ void store_words(char *dst, const Words<W> &v, uint32_t valid)
 {
+    dst = SYMAR_PTR(dst, valid, kRegOut);
     if (valid >= 4u * W) {
         if (W == 1) asm volatile("st.global.u32 [%0], %1;" ::"l"(dst), "r"(v.w[0]) : "memory");
         else if (W == 2)
@@ -354,7 +482,7 @@ __device__ __forceinline__ void store_result(char *out, uint64_t v, const uint4 
                                              uint32_t tail_bytes)
 {
     if (tail_bytes != 0 && v == nvec - 1) {
-        uint16_t *dst = reinterpret_cast<uint16_t *>(out + v * 16);
+        uint16_t *dst = SYMAR_PTR(reinterpret_cast<uint16_t *>(out + v * 16), tail_bytes, kRegOut);
         const uint32_t w[4] = {val.x, val.y, val.z, val.w};
 #pragma unroll
         for (int b = 0; b < 8; ++b)

@@ -493,9 +493,9 @@ static int time_calls(symheap *h, cudaStream_t s, size_t count, int dtype, int a
 //     the payload through scratch; above 1 MiB also one-shot: P times the reads) and that lost by
 //     more than 1.5 x one step down is not timed again -- its traffic grows as fast as the winner's
 //     or faster, so it cannot come back (Table I's volume column); its row reads "not timed";
-//   * above 256 KiB the launch shapes of an algorithm are searched around its winner one step down
-//     (CTA counts from half to four times, block sizes from half to twice), since a message twice
-//     as large wants the same shape or the next larger one;
+//   * above 4 MiB the launch shapes of an algorithm are searched around its winner one step down
+//     (CTA counts from half to four times, every block size), since a message twice as large
+//     wants about as many CTAs or the next larger count;
 //   * a shape whose first two replays are a quarter slower than the algorithm's best so far is
 //     not replayed further.
 static int tune_bucket(symheap *h, int dtype, int b, size_t bytes, cudaStream_t s, Tuned &tn, int prev = -1)
@@ -555,16 +555,16 @@ static int tune_bucket(symheap *h, int dtype, int b, size_t bytes, cudaStream_t 
         struct Cand { double us; LaunchCfg cfg; };
         std::vector<Cand> cands;                     // bandwidth regime: the first pass's shapes, for a second look
         // the neighbourhood of this algorithm's winner one step down
-        // (above 256 KiB only: below, few shapes are valid, calls are short, and the best shape still moves
-        // between the unit widths from one size to the next)
+        // (above 4 MiB only, where every call is long and one kernel form covers all sizes: below, calls
+        // are short, and the best shape still moves with the unit width and, at 1 MiB, with the change
+        // from contiguous chunks to blocks dealt round-robin -- measured 5 to 8 % lost at 1 to 4 MiB)
         const LaunchCfg near =
-            (prune && bytes > (256u << 10) && tn.cfg[algo][prev].ctas > 0) ? tn.cfg[algo][prev] : LaunchCfg{};
+            (prune && bytes > (4u << 20) && tn.cfg[algo][prev].ctas > 0) ? tn.cfg[algo][prev] : LaunchCfg{};
         for (int var : variants) {
             // threads a shape needs: one per unit of this variant
             const uint64_t units = bulk ? work : work << ((var >> 8) & 3);
             for (int T : kThreads) {
                 if (bulk && var != 4 && T != 128 && T != 256) continue;
-                if (near.ctas > 0 && (2 * T < near.threads || T > 2 * near.threads)) continue;
                 for (int C : kCtas) {
                     // skip shapes with far more threads than vectors, except the smallest
                     if ((uint64_t)C * T > 2 * units && !(C == 1 && T == 64)) continue;
@@ -714,17 +714,25 @@ static int create_common(symheap_t **heap, int P, size_t bytes_per_rank, void *m
     }
     // Load every kernel this heap can launch now, so that a first call made
     // during stream capture does not trigger lazy module loading there.
+    // The bulk kernel's dynamic shared memory is what the opt-in limit leaves beside its
+    // static shared memory (none in the regular build).
+    int bulk_static = 0;
+    for (int dt = SYMAR_F32; dt <= SYMAR_BF16 && e == cudaSuccess; ++dt) {
+        cudaFuncAttributes attr;
+        e = cudaFuncGetAttributes(&attr, bulk_kernel_for(dt, P));
+        if (e == cudaSuccess) bulk_static = std::max(bulk_static, (int)attr.sharedSizeBytes);
+    }
+    h->max_smem -= bulk_static;
     for (int algo = SYMAR_ONESHOT; algo <= kLastAlgo && e == cudaSuccess; ++algo)
         for (int dt = SYMAR_F32; dt <= SYMAR_BF16 && e == cudaSuccess; ++dt) {
             cudaFuncAttributes attr;
             e = cudaFuncGetAttributes(&attr, any_kernel_for(algo, dt, P, false));
-            if (e == cudaSuccess && algo == SYMAR_TWOSHOT) {
-                KernelFn bk = bulk_kernel_for(dt, P);
-                e = cudaFuncGetAttributes(&attr, bk);
+            if (e == cudaSuccess && algo == SYMAR_TWOSHOT)
                 // opt in to the large dynamic shared memory now (not during a capture)
-                if (e == cudaSuccess)
-                    e = cudaFuncSetAttribute(bk, cudaFuncAttributeMaxDynamicSharedMemorySize, h->max_smem);
-            }
+                e = cudaFuncSetAttribute(bulk_kernel_for(dt, P), cudaFuncAttributeMaxDynamicSharedMemorySize, h->max_smem);
+            if (e == cudaSuccess && algo == SYMAR_LL)
+                for (int words = 2; words <= 4 && e == cudaSuccess; words += 2)
+                    e = cudaFuncGetAttributes(&attr, ll_small_kernel_for(dt, P, words, false));
         }
     if (e == cudaSuccess) e = cudaDeviceSynchronize();
     if (e != cudaSuccess) {
@@ -1213,6 +1221,35 @@ int symar_debug_phases(symheap_t *heap, const void *in, void *out, size_t count,
         host_ns[3 * k + 2] = (double)(long long)(w[kPhases + k] - t0);
     }
     return SYMAR_OK;
+}
+
+int symar_check_selftest(symheap_t *heap, void *cuda_stream)
+{
+    if (!heap || heap->bytes_per_rank < 4096) return SYMAR_ERR_INVAL;
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    Plan p;
+    int rc = make_plan(heap, 0, 1024, 16, SYMAR_F32, SYMAR_ONESHOT, &p);      // a 64-byte call: in at 0, out at 1024
+    if (rc != SYMAR_OK) return rc;
+    const uint32_t before[4] = {0xAAAAAAAAu, 0xAAAAAAAAu, 0xAAAAAAAAu, 0xAAAAAAAAu};
+    CU(cudaMemcpyAsync(heap->seg0 + 1024 + 64, before, sizeof before, cudaMemcpyHostToDevice, s));
+    CU(cudaStreamSynchronize(s));                          // `before` is on this stack frame
+    cudaError_t e = launch_check_selftest(p.args, s);
+    if (e == cudaErrorNotSupported) {
+        cudaGetLastError();
+        return SYMAR_ERR_UNSUPPORTED;                      // the regular build checks nothing
+    }
+    if (e != cudaSuccess) return cuda_fail(e, "self-test launch");
+    uint32_t inside[4] = {0, 0, 0, 0}, beyond[4] = {0, 0, 0, 0}, status[4] = {0, 0, 0, 0};
+    CU(cudaMemcpyAsync(inside, heap->seg0 + 1024, sizeof inside, cudaMemcpyDeviceToHost, s));
+    CU(cudaMemcpyAsync(beyond, heap->seg0 + 1024 + 64, sizeof beyond, cudaMemcpyDeviceToHost, s));
+    CU(cudaMemcpyAsync(status, heap->ctl, sizeof status, cudaMemcpyDeviceToHost, s));
+    CU(cudaStreamSynchronize(s));
+    const bool landed  = inside[0] == 1u && inside[3] == 4u;
+    const bool kept    = std::memcmp(beyond, before, sizeof before) == 0;
+    const bool flagged = (int)status[kCtlCode] == SYMAR_ERR_INVAL && status[kCtlPeer] == (uint32_t)kRegOutMask;
+    CU(cudaMemsetAsync(heap->ctl, 0, 16, s));              // the recorded violation was the point: clear it
+    CU(cudaStreamSynchronize(s));
+    return (landed && kept && flagged) ? SYMAR_OK : SYMAR_ERR_CUDA;
 }
 
 size_t symar_llbuffer_bytes(int sync_mode, size_t elem_bytes, size_t slots_per_cta, int ctas, int round_robin)

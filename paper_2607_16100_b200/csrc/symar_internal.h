@@ -26,6 +26,9 @@ KernelFn atomic_kernel_for(int dtype, int P, bool dbg);
 cudaError_t launch_kernel(KernelFn fn, int P, int ctas_per_rank, int threads, size_t smem_bytes,
                           const KArgs &args, cudaStream_t stream);
 
+// Checking build only (cudaErrorNotSupported otherwise): the kernel behind symar_check_selftest().
+cudaError_t launch_check_selftest(const KArgs &args, cudaStream_t stream);
+
 // Sibling collectives (symar_coll.cu): op = 0 ReduceScatter, 1 AllGather, 2 Broadcast, 3 Reduce.
 cudaError_t launch_collective(int op, int dtype, int P, int ctas_per_rank, int threads, const KArgs &k,
                               uint64_t bytes, int root, int unit, cudaStream_t stream);

@@ -69,6 +69,7 @@ enum : int { kCtlCode = 0, kCtlRank = 1, kCtlPeer = 2, kCtlCta = 3,
              // phase stamps (test hook): kPhases u64 each -- earliest, latest, wrapping sum, number of stamps
              kCtlPhaseMin = 64, kCtlPhaseMax = 80, kCtlPhaseSum = 96, kCtlPhaseCnt = 112 };
 constexpr int kPhases = 8;
+constexpr uint32_t kRegOutMask = 2;    // region bit of "this call's output range" in a bounds-check report (kCtlPeer)
 
 __host__ __device__ constexpr size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 

@@ -80,10 +80,30 @@ struct StaticArgs {
 template <typename E, int P>
 __global__ void __launch_bounds__(kStaticThreads) ll_static_kernel(const StaticArgs a)
 {
+#ifdef SYMAR_CHECK
+    if (threadIdx.x == 0) {       // checking build: the caller's rows and the two parts of the static array
+        CheckCtx &cc = check_ctx();
+        const uint64_t bytes = a.tail_bytes ? (a.nvec - 1) * 16 + a.tail_bytes : a.nvec * 16;
+        cc.base = nullptr;
+        cc.nreg = 0;
+        cc.nranks = 0;
+        cc.stride = 1;
+        cc.ctl    = nullptr;
+        cc.status = a.status;
+        cc.nabs   = 4;
+        cc.alo[0] = a.in;   cc.ahi[0] = a.in + (uint64_t)(P - 1) * a.pitch + bytes;  cc.akind[0] = kRegIn;
+        cc.alo[1] = a.out;  cc.ahi[1] = a.out + (uint64_t)(P - 1) * a.pitch + bytes; cc.akind[1] = kRegOut;
+        cc.alo[2] = reinterpret_cast<const char *>(a.scratch);
+        cc.ahi[2] = cc.alo[2] + kStaticCtrBytes;                                     cc.akind[2] = kRegCtr;
+        cc.alo[3] = cc.ahi[2];  cc.ahi[3] = cc.alo[2] + kStaticBytes;                cc.akind[3] = kRegLL;
+    }
+    __syncthreads();
+#endif
     const int c = blockIdx.x, r = blockIdx.y;
     const uint32_t t = threadIdx.x;
     constexpr uint32_t lg = Log2<P>::v;
-    uint64_t *ep = reinterpret_cast<uint64_t *>(a.scratch) + ((size_t)lg * kMaxRanks + r) * kStaticSlots + c;
+    uint64_t *ep = SYMAR_PTR(reinterpret_cast<uint64_t *>(a.scratch) + ((size_t)lg * kMaxRanks + r) * kStaticSlots + c, 8,
+                             kRegCtr);
     const uint64_t n = ld_relaxed_u64(ep) + 1;
     const uint32_t e = static_flag(n, lg);
     const uint64_t v = (uint64_t)c * kStaticThreads + t;
@@ -98,7 +118,8 @@ __global__ void __launch_bounds__(kStaticThreads) ll_static_kernel(const StaticA
         if (a.tail_bytes != 0 && v == a.nvec - 1) {
             // The caller's buffer may end with the message: read only the valid
             // bytes of a partial last vector (the rest is sent as zeros and never stored).
-            const uint16_t *src = reinterpret_cast<const uint16_t *>(a.in + (size_t)r * a.pitch + v * 16);
+            const uint16_t *src =
+                SYMAR_PTR(reinterpret_cast<const uint16_t *>(a.in + (size_t)r * a.pitch + v * 16), a.tail_bytes, kRegIn);
             uint32_t w[4] = {0u, 0u, 0u, 0u};
 #pragma unroll
             for (int b = 0; b < 8; ++b)

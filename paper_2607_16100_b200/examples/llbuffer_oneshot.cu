@@ -120,9 +120,76 @@ __global__ void allgather_u64_kernel(const char *in0, char *out0, size_t io_stri
     }
 }
 
+// Stress of the 16-byte LL slot that an 8-byte element occupies ({payload64, flag64} in one vector
+// store): for `epochs` epochs in one launch every thread sends a payload that spells out its epoch,
+// sender and slot to all peers and receives the peers' payloads; a payload whose flag says "this
+// epoch" while its own epoch field says otherwise would be a 16-byte store observed in two halves.
+// Seeded idle times before every epoch vary which side is ahead.  counts[0]: a wait ran out;
+// counts[1]: payloads that did not match their flag; counts[2]: payloads checked.
+template <int P>
+__global__ void slot_stress_u64_kernel(char *scratch0, size_t scratch_stride, int slots, uint64_t first_epoch,
+                                       uint32_t epochs, uint32_t seed, uint32_t max_idle_ns, unsigned long long *counts)
+{
+    const int cta = blockIdx.x, ctas = gridDim.x, rank = blockIdx.y, t = threadIdx.x;
+    LLBuffer<LLSync::LL> buf(scratch0, scratch_stride, rank, P, cta, ctas,
+                             (size_t)P * slots * LLBuffer<LLSync::LL>::template slotBytes<uint64_t>(), 2, first_epoch,
+                             1u << 22);
+    unsigned long long bad = 0, seen = 0;
+    for (uint32_t it = 0; it < epochs; ++it) {
+        if (max_idle_ns != 0) {          // bounded pause, different per CTA, rank and epoch
+            uint32_t h = seed ^ (uint32_t)(rank * 0x9E3779B1u) ^ (uint32_t)(cta * 0x85EBCA77u) ^ (it * 0xC2B2AE3Du);
+            h ^= h >> 16; h *= 0x7feb352dU; h ^= h >> 15; h *= 0x846ca68bU; h ^= h >> 16;
+            const uint64_t wait = h % max_idle_ns;
+            uint64_t t0, now;
+            asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t0));
+            do { asm volatile("mov.u64 %0, %globaltimer;" : "=l"(now)); } while (now - t0 < wait);
+        }
+        const uint64_t e = buf.epoch();
+        if (t < slots) {
+            const uint64_t mine = (e << 32) | ((uint64_t)rank << 16) | (uint64_t)t;
+            for (int q = 0; q < P; ++q)
+                if (q != rank) buf.template send<uint64_t>(q, (size_t)rank * slots + t, mine);
+            for (int q = 0; q < P; ++q) {
+                if (q == rank) continue;
+                uint64_t v;
+                if (!buf.template recv<uint64_t>((size_t)q * slots + t, v)) {
+                    atomicAdd(&counts[0], 1ull);
+                    return;
+                }
+                ++seen;
+                if (v != ((e << 32) | ((uint64_t)q << 16) | (uint64_t)t)) ++bad;
+            }
+        }
+        buf.advanceEpoch();
+    }
+    if (bad) atomicAdd(&counts[1], bad);
+    atomicAdd(&counts[2], seen);
+}
+
 }  // namespace
 
 extern "C" {
+
+// Runs the slot stress above: P ranks x ctas CTAs x `slots` threads, `epochs` epochs from `first_epoch`
+// (epochs below 2^32 so that the payload's epoch field is the flag).  Scratch per rank:
+// symar_llbuffer_bytes(0, 8, P * slots, ctas, 2), zeroed before the first launch.  device_counts: three
+// zeroed 64-bit counters (waits that ran out, mismatching payloads, payloads checked).
+int llbuffer_slot_stress_u64(int P, void *scratch0, size_t scratch_stride, int ctas, int slots, unsigned long long first_epoch,
+                             unsigned epochs, unsigned seed, unsigned max_idle_ns, unsigned long long *device_counts,
+                             void *cuda_stream)
+{
+    if (!scratch0 || !device_counts || ctas < 1 || slots < 1 || slots > 1024 || first_epoch == 0 || max_idle_ns > 100000u ||
+        first_epoch + epochs >= (1ull << 32))
+        return -1;
+    const dim3 grid(ctas, P), block((slots + 31) / 32 * 32);
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    char *s0 = (char *)scratch0;
+    if (P == 2) slot_stress_u64_kernel<2><<<grid, block, 0, s>>>(s0, scratch_stride, slots, first_epoch, epochs, seed, max_idle_ns, device_counts);
+    else if (P == 4) slot_stress_u64_kernel<4><<<grid, block, 0, s>>>(s0, scratch_stride, slots, first_epoch, epochs, seed, max_idle_ns, device_counts);
+    else if (P == 8) slot_stress_u64_kernel<8><<<grid, block, 0, s>>>(s0, scratch_stride, slots, first_epoch, epochs, seed, max_idle_ns, device_counts);
+    else return -1;
+    return cudaGetLastError() == cudaSuccess ? 0 : -3;
+}
 
 // All-gather of nwords 64-bit words per rank: out[r] = in[0] | in[1] | ... | in[P-1] for every rank r.
 // Scratch per rank: symar_llbuffer_bytes(mode, 8, P * ceil(nwords / ctas), ctas, 0).  mode / epoch /

@@ -73,6 +73,7 @@ SIGNATURES = [
     ("symar_debug_span", c_int, [c_void_p, c_void_p, c_void_p, c_size_t, c_int, c_int, c_void_p, POINTER(c_double)]),
     ("symar_debug_phases", c_int, [c_void_p, c_void_p, c_void_p, c_size_t, c_int, c_int, c_void_p, POINTER(c_double),
                                    POINTER(c_int)]),
+    ("symar_check_selftest", c_int, [c_void_p, c_void_p]),
     ("symar_probe_barrier", c_int, [c_int, c_int, c_int, POINTER(c_double)]),
     ("symar_llbuffer_bytes", c_size_t, [c_int, c_size_t, c_size_t, c_int, c_int]),
     ("symar_llbuffer_init_sentinel", c_int, [c_void_p, c_size_t, c_void_p]),
@@ -326,6 +327,10 @@ class SymHeap:
                                          algo, stream, ns, n), "symar_debug_phases")
         return {k: {"first": ns[3 * k], "mean": ns[3 * k + 1], "last": ns[3 * k + 2], "ctas": n[k]}
                 for k in range(8) if n[k] > 0}
+
+    def check_selftest(self, stream: int = 0) -> int:
+        """Raw status of the bounds-checking build's self-test (ERR_UNSUPPORTED in the regular build)."""
+        return int(self._lib.symar_check_selftest(self._h, stream))
 
     def debug_inject(self, mute_rank: int = -1, delay_seed: int = 0, delay_max_ns: int = 0) -> None:
         _ck(self._lib.symar_debug_inject(self._h, mute_rank, delay_seed, delay_max_ns), "symar_debug_inject")

@@ -172,3 +172,35 @@ def test_allgather_of_64_bit_words_on_the_primitives(allgather, mode, P):
     finally:
         torch.cuda.synchronize()
         h.destroy()
+
+
+@pytest.mark.parametrize("P,ctas,slots,epochs", [(2, 8, 128, 4000), (8, 4, 64, 1500), (4, 16, 32, 2500)])
+def test_16_byte_slots_of_64_bit_elements_are_observed_whole(P, ctas, slots, epochs):
+    # An 8-byte element travels as {payload64, flag64} in ONE 16-byte store; the buffer is correct only if a
+    # reader never sees the new flag beside the old payload.  Thousands of epochs in one launch, every payload
+    # spelling out its epoch, sender and slot, seeded idle times shifting which rank is ahead: no payload may
+    # disagree with its flag, and no wait may run out.
+    lib = ctypes.CDLL(str(build.build_example()))
+    fn = lib.llbuffer_slot_stress_u64
+    fn.restype = ctypes.c_int
+    fn.argtypes = [ctypes.c_int, ctypes.c_void_p, ctypes.c_size_t, ctypes.c_int, ctypes.c_int, ctypes.c_ulonglong,
+                   ctypes.c_uint, ctypes.c_uint, ctypes.c_uint, ctypes.c_void_p, ctypes.c_void_p]
+    nbytes = symar.llbuffer_bytes(LL, 8, P * slots, ctas, 2)
+    assert nbytes == 2 * 8 * P * slots * ctas * 2
+    h = symar.SymHeap.on_torch(P, nbytes)
+    try:
+        for q in range(P):
+            h.write_rank(q, 0, np.zeros(nbytes, dtype=np.uint8))
+        epoch = 1
+        for seed, idle_ns in ((1, 0), (2, 2000), (3, 300), (4, 20000)):
+            counts = torch.zeros(3, dtype=torch.int64, device="cuda")
+            n = epochs if idle_ns <= 2000 else epochs // 10
+            assert fn(P, h.rank_ptr(0, 0), h.info().stride, ctas, slots, epoch, n, seed, idle_ns, counts.data_ptr(), 0) == 0
+            torch.cuda.synchronize()
+            timeouts, mismatches, checked = (int(v) for v in counts.cpu())
+            assert timeouts == 0 and mismatches == 0, (seed, timeouts, mismatches)
+            assert checked == P * ctas * slots * (P - 1) * n
+            epoch += n
+    finally:
+        torch.cuda.synchronize()
+        h.destroy()
