@@ -631,6 +631,12 @@ def latency_suite(torch, symar, synth, hbm_gbs, quick=False, autotune=True):
                 ra = bench_size(8192 * B, (symar.TWOSHOT_ATOMIC,))["twoshot_atomic"]
                 fl = empty_floor(row["auto"]["ctas_per_rank"], P, row["auto"]["threads"], n=100)
                 s_ol = fl["p50"] + rt_ns / 1000.0 + bytes_us(16384 * B, P)
+                try:       # where two-shot's time goes: exchange, data, CTA barrier, release fence, "done" hop
+                    ph = [h.debug_phases(0, out_off, 8192 * B, symar.BF16, symar.TWOSHOT) for _ in range(15)]
+                    ts_phases = {str(k): {f: float(np.median([p_[k][f] for p_ in ph])) / 1e3
+                                          for f in ("first", "mean", "last")} for k in sorted(ph[0])}
+                except symar.SymarError as exc:
+                    ts_phases = {"error": str(exc)}
                 sweep.append({"bytes_per_rank": 16384 * B, "p50_us": {k: v["p50"] for k, v in row.items()},
                               "twoshot_atomic_p50_us": ra["p50"], "twoshot_atomic_within_tolerance":
                                   ra["within_tolerance"],
@@ -643,6 +649,7 @@ def latency_suite(torch, symar, synth, hbm_gbs, quick=False, autotune=True):
                                                "bytes_at_measured_hbm_copy_rate": bytes_us(16384 * B, P)},
                               "oracle_cpu": oracle_us(O, synth.make_inputs("normal", "bf16", P, 8192 * B,
                                                                            synth.seed_for_config(2))),
+                              "twoshot_phase_stamps_us": ts_phases,
                               "bit_exact": all(v["bit_exact"] for v in row.values())})
             out["sweep"] = sweep
             out["sweep_note"] = "sol_us = empty launch of the selector's shape + median flag round trip + 2*P*M bytes at " \
