@@ -453,6 +453,10 @@ def latency_suite(torch, symar, synth, hbm_gbs, quick=False, autotune=True):
                 rep_rows.append({"p50_us": p_i, "empty_launch_us": fl_i, "flag_round_trip_median_us": rt_i["median_us"],
                                  "flag_round_trip_min_us": rt_i["min_us"], "sol_us": sol_i, "ratio_to_sol": p_i / sol_i,
                                  "ratio_to_sol_fastest_pair": p_i / (fl_i + rt_i["min_us"] + t_bytes_us)})
+            # the same call with every reader on copy 0 of the flags and counters (no placement on the L2 halves)
+            h.set_placement(False)
+            unplaced = bench_size(8192, (symar.AUTO,))["auto"]
+            h.set_placement(True)
             o_a, o_c, o_t = h.query_choice(8192, symar.BF16, symar.ONESHOT)
             o_var = row["oneshot"]["variant"]
             release = with_variant(symar.ONESHOT, o_var | 0x8000, o_c, o_t)
@@ -490,6 +494,9 @@ def latency_suite(torch, symar, synth, hbm_gbs, quick=False, autotune=True):
                     "note": "the selector's one-shot with red.release on the ready signal and nothing else changed: "
                             "the form a system needs whose ranks do not share a kernel boundary"},
                 "system_scope_build": sys_scope,
+                "placement": dict(zip(("measured", "sms_on_second_half", "home_bits"), h.placement())),
+                "without_placement_on_l2_halves": {"p50_us": unplaced["p50"], "bit_exact": unplaced["bit_exact"],
+                                                   "note": "every reader takes copy 0 of its flags and counters"},
                 "in_kernel_span_us_p50": {
                     names[a_]: float(np.median([h.debug_span(0, out_off, 8192, symar.BF16, a_) for _ in range(31)])) / 1e3
                     for a_ in (symar.ONESHOT, symar.TWOSHOT, symar.LL, symar.SENTINEL)},
@@ -801,6 +808,7 @@ def compact_line(bw, lat, details):
             "bit_exact": all(v.get("bit_exact") for v in c2.get("per_algo", {}).values()),
             "ll_p50_us": _r((c2.get("per_algo", {}).get("ll") or {}).get("p50"), 3),
             "oneshot_release_p50_us": _r((c2.get("oneshot_release_signal") or {}).get("p50_us"), 3),
+            "unplaced_p50_us": _r((c2.get("without_placement_on_l2_halves") or {}).get("p50_us"), 3),
             "sys_scope_p50_us": {k: _r((sysb.get(k) or {}).get("p50_us"), 3) for k in ("oneshot", "ll")}
             if "error" not in sysb else None,
             "oracle_cpu_us": _r((c2.get("oracle_cpu") or {}).get("all_cores_us"), 1),

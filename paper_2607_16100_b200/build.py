@@ -12,7 +12,7 @@ ROOT = PKG.parent
 CSRC = PKG / "csrc"
 LIB = PKG / "libsymar.so"
 SOURCES = ["symar_kernels.cu", "symar_bulk.cu", "symar_host.cu", "symar_probe.cu", "symar_static.cu", "symar_coll.cu",
-           "symar_atomic.cu"]
+           "symar_atomic.cu", "symar_place.cu"]
 
 LIB_SYS = PKG / "libsymar_sys.so"
 LIB_CHECK = PKG / "libsymar_check.so"

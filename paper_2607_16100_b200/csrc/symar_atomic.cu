@@ -87,7 +87,7 @@ __global__ void __launch_bounds__(kMaxThreads) twoshot_atomic_kernel(const KArgs
     const uint32_t j = t & 7u;                       // position in the 8-thread group of a line
     const uint32_t g = t >> 3, G = T >> 3;           // group index, groups per CTA
     char *seg_r      = a.seg0 + (size_t)r * a.stride;
-    uint32_t *dcount = SYMAR_PTR(reinterpret_cast<uint32_t *>(seg_r + a.epoch_off + done_count_off(c)), 4, kRegCtr);
+    const uint32_t *dcount = reinterpret_cast<const uint32_t *>(counters_near(a, r, c) + kCtrDone);
     if (a.pdl) {
         pdl_wait();                                  // the previous call has left the heap
         pdl_launch_dependents();
@@ -184,8 +184,8 @@ __global__ void __launch_bounds__(kMaxThreads) twoshot_atomic_kernel(const KArgs
     // until every peer's CTA c has delivered its part here.
     uint32_t dwant;
     const bool all_ok = __syncthreads_and(ok);
-    flag_exchange<P, true>(a, a.done_off, dcount, r, c, !all_ok, false, dwant);
-    if (t == 0) *dcount = dwant;
+    flag_exchange<P, true>(a, a.done_off, kPairDone, dcount, r, c, !all_ok, false, dwant);
+    publish_u32(a, r, c, kCtrDone, dwant);
     if (DBG) debug_stamp_out(a);
 }
 

@@ -87,9 +87,8 @@ __global__ void __launch_bounds__(kMaxThreads) twoshot_bulk_kernel(const KArgs a
     unsigned char *in_tiles  = smem + kBulkBarBytes;                        // [S][P][TB]
     unsigned char *out_tiles = in_tiles + (size_t)S * P * TB;               // [kBulkOutBufs][TB]
 
-    char *seg_r = a.seg0 + (size_t)r * a.stride;
-    uint32_t *rcount = SYMAR_PTR(reinterpret_cast<uint32_t *>(seg_r + a.epoch_off + ready_count_off(c)), 4, kRegCtr);
-    uint32_t *dcount = SYMAR_PTR(reinterpret_cast<uint32_t *>(seg_r + a.epoch_off + done_count_off(c)), 4, kRegCtr);
+    const uint32_t *rcount = reinterpret_cast<const uint32_t *>(counters_near(a, r, c) + kCtrReady);
+    const uint32_t *dcount = reinterpret_cast<const uint32_t *>(counters_near(a, r, c) + kCtrDone);
 
     if (t == 0) {
         for (uint32_t s = 0; s < S; ++s) mbar_init(&full[s], 1);
@@ -99,7 +98,7 @@ __global__ void __launch_bounds__(kMaxThreads) twoshot_bulk_kernel(const KArgs a
 
     if (a.pdl) pdl_wait();                  // the previous call has left the heap
     uint32_t rwant, dwant;
-    bool ok = flag_exchange<P, false>(a, a.ready_off, rcount, r, c, false, true, rwant);
+    bool ok = flag_exchange<P, false>(a, a.ready_off, kPairReady, rcount, r, c, false, true, rwant);
     ok = __syncthreads_and(ok);            // the whole CTA enters the pipeline, or none of it
 
     // The bulk path moves whole vectors; a partial last vector is done by hand below.
@@ -193,11 +192,9 @@ __global__ void __launch_bounds__(kMaxThreads) twoshot_bulk_kernel(const KArgs a
         twoshot_vector<E, P>(a, a.nvec - 1);
 
     __syncthreads();
-    flag_exchange<P, true>(a, a.done_off, dcount, r, c, !ok, false, dwant);
-    if (t == 0) {
-        *rcount = rwant;
-        *dcount = dwant;
-    }
+    flag_exchange<P, true>(a, a.done_off, kPairDone, dcount, r, c, !ok, false, dwant);
+    publish_u32(a, r, c, kCtrReady, rwant);
+    publish_u32(a, r, c, kCtrDone, dwant);
 }
 
 template <typename E>

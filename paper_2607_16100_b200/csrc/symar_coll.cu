@@ -124,14 +124,13 @@ __global__ void __launch_bounds__(kMaxThreads) coll_kernel(const CollArgs a)
     const int c = blockIdx.x, r = blockIdx.y, C = gridDim.x;
     const uint32_t t = threadIdx.x, T = blockDim.x;
     const KArgs &k = a.k;
-    char *seg_r = k.seg0 + (size_t)r * k.stride;
-    uint32_t *count = SYMAR_PTR(reinterpret_cast<uint32_t *>(seg_r + k.epoch_off + ready_count_off(c)), 4, kRegCtr);
+    const uint32_t *count = reinterpret_cast<const uint32_t *>(counters_near(k, r, c) + kCtrReady);
     if (k.pdl) pdl_wait();
 
     uint32_t want;
-    const bool ok = flag_exchange<P, false>(k, k.ready_off, count, r, c, false, true, want);
+    const bool ok = flag_exchange<P, false>(k, k.ready_off, kPairReady, count, r, c, false, true, want);
     __syncthreads();
-    if (t == 0) *count = want;
+    publish_u32(k, r, c, kCtrReady, want);
     if (k.pdl) pdl_launch_dependents();
     if (!ok) return;
     if (OP == kOpReduce && r != a.root) return;          // only the root receives the sum

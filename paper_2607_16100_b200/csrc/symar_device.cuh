@@ -82,7 +82,7 @@ __device__ __forceinline__ void check_begin(const KArgs &a, int nranks, uint64_t
         const uint64_t lo[8]   = {a.in_off, a.out_off, a.ll_off, a.sn_off, a.at_off, a.ready_off, a.done_off, a.epoch_off};
         const uint64_t hi[8]   = {a.in_off + (in_bytes + 15) / 16 * 16,   // whole vectors are read (the region is padded)
                                   a.out_off + out_bytes, a.sn_off, a.at_off, a.ready_off, a.done_off, a.epoch_off,
-                                  a.epoch_off + (uint64_t)kMaxCtas * 16};
+                                  a.epoch_off + (uint64_t)kPairBytes};
         const uint32_t kind[8] = {kRegIn, kRegOut, kRegLL, kRegSn, kRegAt, kRegReady, kRegDone, kRegCtr};
         c.nreg = 8;
         for (int i = 0; i < 8; ++i) {
@@ -539,6 +539,38 @@ __device__ __forceinline__ void debug_delay(const KArgs &a, int rank, int cta)
     while (globaltimer_ns() - t0 < wait) { /* bounded by dbg_delay_ns */ }
 }
 
+// ---- the copy of a flag or counter that is homed on this SM's half of the chip ------------------
+__device__ __forceinline__ uint32_t my_half(const KArgs &a)
+{
+    uint32_t smid;
+    asm("mov.u32 %0, %%smid;" : "=r"(smid));
+    const uint64_t w = smid < 64u ? a.sm_half[0] : (smid < 128u ? a.sm_half[1] : (smid < 192u ? a.sm_half[2] : a.sm_half[3]));
+    return (uint32_t)(w >> (smid & 63u)) & 1u;
+}
+__device__ __forceinline__ uint32_t near_copy(const KArgs &a, uint32_t half, int rank, int pair)
+{
+    return half ^ ((uint32_t)(a.home >> (rank * kPairsPerRank + pair)) & 1u);
+}
+// the counters of (rank r, slot c), copy k
+__device__ __forceinline__ char *counters_at(const KArgs &a, int r, int c, uint32_t k)
+{
+    return a.seg0 + (size_t)r * a.stride + a.epoch_off + counters_off(c, k);
+}
+// the copy to READ (this SM's half)
+__device__ __forceinline__ const char *counters_near(const KArgs &a, int r, int c)
+{
+    return counters_at(a, r, c, near_copy(a, my_half(a), r, kPairCounters));
+}
+// WRITE a counter: threads 0 and 1 of the CTA store the two copies
+__device__ __forceinline__ void publish_u32(const KArgs &a, int r, int c, size_t which, uint32_t v)
+{
+    if (threadIdx.x < 2) *SYMAR_PTR(reinterpret_cast<uint32_t *>(counters_at(a, r, c, threadIdx.x) + which), 4, kRegCtr) = v;
+}
+__device__ __forceinline__ void publish_u64(const KArgs &a, int r, int c, size_t which, uint64_t v)
+{
+    if (threadIdx.x < 2) *SYMAR_PTR(reinterpret_cast<uint64_t *>(counters_at(a, r, c, threadIdx.x) + which), 8, kRegCtr) = v;
+}
+
 // ---- one synchronisation of Table I ---------------------------------------------------
 // Slot c of rank r signals slot c of every peer and waits for every peer's
 // signal.
@@ -558,18 +590,20 @@ __device__ __forceinline__ void debug_delay(const KArgs &a, int rank, int cta)
 // `want` receives the count to publish.  Returns false if the wait ran out.
 // The addresses one exchange touches, computable before the kernel may touch memory.
 struct ExchangePtrs {
-    uint32_t       *signal;   // thread t < P: this rank's word in peer t's flag group
-    const uint32_t *mine;     // lane q: peer q's word in this rank's flag group
+    uint32_t       *signal;   // thread t < 2P: this rank's word in copy t / P of peer (t mod P)'s flag group
+    const uint32_t *mine;     // lane q: peer q's word in this rank's flag group, the copy homed on this SM's half
 };
+// `pair` = kPairReady or kPairDone, matching flags_off
 template <int P>
-__device__ __forceinline__ ExchangePtrs exchange_ptrs(const KArgs &a, uint64_t flags_off, int r, int c)
+__device__ __forceinline__ ExchangePtrs exchange_ptrs(const KArgs &a, uint64_t flags_off, int pair, int r, int c)
 {
     const uint32_t t    = threadIdx.x;
     const uint32_t lane = t & 31u;
+    const uint32_t peer = t & (uint32_t)(P - 1), copy = (t / P) & 1u;
     ExchangePtrs p;
-    p.signal = reinterpret_cast<uint32_t *>(a.seg0 + (size_t)(t < P ? t : 0) * a.stride + flags_off +
-                                            (size_t)c * kFlagGroup) + r;
-    p.mine   = reinterpret_cast<const uint32_t *>(a.seg0 + (size_t)r * a.stride + flags_off + (size_t)c * kFlagGroup) +
+    p.signal = reinterpret_cast<uint32_t *>(a.seg0 + (size_t)peer * a.stride + flags_off + flag_group_off(c, copy)) + r;
+    const uint32_t nc = near_copy(a, my_half(a), r, pair + c / kFlagSlotsPerPair);
+    p.mine   = reinterpret_cast<const uint32_t *>(a.seg0 + (size_t)r * a.stride + flags_off + flag_group_off(c, nc)) +
              (lane < P ? lane : 0);
     return p;
 }
@@ -582,7 +616,7 @@ __device__ __forceinline__ bool flag_exchange_at(const KArgs &a, const ExchangeP
 {
     const uint32_t t    = threadIdx.x;
     const uint32_t lane = t & 31u;
-    if (t < P && !silent) {
+    if (t < 2 * P && !silent) {              // both copies of every peer's flag word
         if (RELEASE) red_release_inc_u32(p.signal);
         else red_relaxed_inc_u32(p.signal);
     }
@@ -607,11 +641,11 @@ __device__ __forceinline__ bool flag_exchange_at(const KArgs &a, const ExchangeP
 }
 
 template <int P, bool RELEASE, int STAMP = -1>
-__device__ __forceinline__ bool flag_exchange(const KArgs &a, uint64_t flags_off, const uint32_t *count,
+__device__ __forceinline__ bool flag_exchange(const KArgs &a, uint64_t flags_off, int pair, const uint32_t *count,
                                               int r, int c, bool silent, bool all_warps, uint32_t &want)
 {
-    return flag_exchange_at<P, RELEASE, STAMP>(a, exchange_ptrs<P>(a, flags_off, r, c), count, r, c, silent, all_warps,
-                                               want);
+    return flag_exchange_at<P, RELEASE, STAMP>(a, exchange_ptrs<P>(a, flags_off, pair, r, c), count, r, c, silent,
+                                               all_warps, want);
 }
 
 // Reduce-scatter + all-gather of one 16-byte vector: P loads, the rank-ordered

@@ -8,6 +8,7 @@
 #include <cstdlib>
 #include <cstring>
 #include <map>
+#include <mutex>
 #include <new>
 #include <string>
 #include <tuple>
@@ -45,6 +46,12 @@ struct Tuned {
 
 static thread_local std::string g_last_cuda_error;
 
+// which half of the chip every SM of a device sits on: measured once per device and process
+constexpr int kMaxDevices = 64;
+struct DevicePlace { bool tried = false, ok = false; uint64_t sm_half[4] = {0, 0, 0, 0}; };
+static DevicePlace g_place[kMaxDevices];
+static std::mutex  g_place_mutex;
+
 static int cuda_fail(cudaError_t e, const char *what)
 {
     g_last_cuda_error = std::string(what) + ": " + cudaGetErrorString(e);
@@ -76,6 +83,10 @@ struct symheap {
     int       env_algo     = 0;       // SYMAR_ALGO override of SYMAR_AUTO, 0 = none
     bool      debug_log    = false;   // SYMAR_DEBUG=1: one stderr line per call
     bool      tune_exhaustive = false;   // SYMAR_TUNE=exhaustive: the tuner prunes nothing
+    bool      placed   = false;       // sm_half / home were measured cleanly
+    bool      place_on = true;        // readers take the copy of their own L2 half (SYMAR_PLACE=0 / symar_set_placement)
+    uint64_t  sm_half[4] = {0, 0, 0, 0};
+    uint64_t  home = 0;
     size_t    scratch_limit = 0;      // push algorithms: payload bytes per rank and iteration, 0 = all there is
     int       dbg_mute     = -1;
     unsigned  dbg_seed     = 0;
@@ -197,9 +208,10 @@ static LaunchCfg default_cfg(const symheap *h, int algo, uint64_t nvec)
 // thread, which is a gain only while those are few.
 static int default_algo(int P, size_t bytes)
 {
-    // the data+flag protocol leads at the smallest sizes (Sec. VII Obs. 1); measured here: up to
-    // 16 KiB between two ranks, up to a few hundred bytes among eight, nowhere among four
-    if ((P == 2 && bytes <= (16u << 10)) || (P == 8 && bytes <= 512)) return SYMAR_LL;
+    // the data+flag protocol leads at the smallest sizes (Sec. VII Obs. 1); measured here, with flag
+    // and counter reads placed on the reader's L2 half: up to 1 KiB between two ranks (1.24 against
+    // 1.43 us at 128 B), nowhere among four or eight (one-shot 1.37 / 1.53 us against 1.49 / 1.69 us)
+    if (P == 2 && bytes <= 1024) return SYMAR_LL;
     if (bytes <= (256u << 10)) return SYMAR_ONESHOT;
     return SYMAR_TWOSHOT;
 }
@@ -307,6 +319,10 @@ static int make_plan(symheap *h, size_t in_off, size_t out_off, size_t count, in
     a.dbg_seed   = h->dbg_seed;
     a.dbg_delay_ns = h->dbg_delay_ns;
     a.dbg_span   = h->dbg_span ? 1u : 0u;
+    if (h->placed && h->place_on) {
+        std::memcpy(a.sm_half, h->sm_half, sizeof a.sm_half);
+        a.home = h->home;
+    }
     if (algo == SYMAR_TWOSHOT) {
         const bool cyclic = nvec >= kCyclicMinVec && !(var & 1u);
         a.blk_log2 = cyclic ? kCyclicLog2 : kOneChunk;
@@ -420,6 +436,10 @@ static int run_collective(symheap *h, int op, const void *in, void *out, size_t 
     a.spin_ns   = h->spin_ns;
     a.pdl       = h->pdl ? 1u : 0u;
     a.dbg_mute  = -1;
+    if (h->placed && h->place_on) {
+        std::memcpy(a.sm_half, h->sm_half, sizeof a.sm_half);
+        a.home = h->home;
+    }
     cudaError_t e = launch_collective(op, dtype, h->P, ctas, threads, a, bytes, root, unit, s);
     if (e != cudaSuccess) return cuda_fail(e, "collective launch");
     h->last_algo    = SYMAR_ONESHOT;
@@ -433,8 +453,8 @@ static int run_collective(symheap *h, int op, const void *in, void *out, size_t 
 // ---- autotuner ---------------------------------------------------------------------
 
 // Median per-call time (us) of K back-to-back calls captured in one graph.
-// `give_up_us` > 0: a candidate whose first two replays both take longer than that is not worth
-// the remaining replays (its faster replay is returned).
+// `give_up_us` > 0: a candidate whose first three replays all take longer than that is not worth
+// the remaining replays (its fastest replay is returned).
 static int time_calls(symheap *h, cudaStream_t s, size_t count, int dtype, int algo, int K, int reps,
                       double *us_out, double give_up_us = 0.0)
 {
@@ -468,8 +488,8 @@ static int time_calls(symheap *h, cudaStream_t s, size_t count, int dtype, int a
         cudaEventRecord(e1, s);
         cudaEventSynchronize(e1);
         cudaEventElapsedTime(&ms[i], e0, e1);
-        if (i == 1 && give_up_us > 0.0 && (double)std::min(ms[0], ms[1]) * 1000.0 / K > give_up_us) {
-            ms.assign(reps, std::min(ms[0], ms[1]));
+        if (i == 2 && give_up_us > 0.0 && (double)std::min({ms[0], ms[1], ms[2]}) * 1000.0 / K > give_up_us) {
+            ms.assign(reps, std::min({ms[0], ms[1], ms[2]}));
             break;
         }
     }
@@ -496,8 +516,8 @@ static int time_calls(symheap *h, cudaStream_t s, size_t count, int dtype, int a
 //   * above 4 MiB the launch shapes of an algorithm are searched around its winner one step down
 //     (CTA counts from half to four times, every block size), since a message twice as large
 //     wants about as many CTAs or the next larger count;
-//   * a shape whose first two replays are a quarter slower than the algorithm's best so far is
-//     not replayed further.
+//   * a shape whose first three replays are all a quarter slower than the algorithm's best so far
+//     is not replayed further.
 static int tune_bucket(symheap *h, int dtype, int b, size_t bytes, cudaStream_t s, Tuned &tn, int prev = -1)
 {
     static const int kThreads[] = {64, 128, 256, 512};
@@ -579,7 +599,7 @@ static int tune_bucket(symheap *h, int dtype, int b, size_t bytes, cudaStream_t 
                     if (make_plan(h, 0, round_up(bytes, kAlign), count, dtype, algo, &p) != SYMAR_OK) continue;
                     if (p.cfg.ctas != C || p.cfg.threads != T) continue;   // clamped: a duplicate of another shape
                     double us = 0;
-                    // a shape a quarter slower than this algorithm's best so far is dropped after two replays
+                    // a shape a quarter slower than this algorithm's best so far is dropped after three replays
                     rc = time_calls(h, s, count, dtype, algo, K, reps, &us,
                                     h->tune_exhaustive || tn.us[algo][b] > 1e29 ? 0.0 : 1.25 * tn.us[algo][b]);
                     if (rc != SYMAR_OK) break;
@@ -707,6 +727,24 @@ static int create_common(symheap_t **heap, int P, size_t bytes_per_rank, void *m
     cudaError_t e = cudaGetDevice(&h->device);
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&h->num_sms, cudaDevAttrMultiProcessorCount, h->device);
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&h->max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, h->device);
+    // Where the SMs and this heap's flag and counter lines sit on the chip's two L2 halves (measured once
+    // per device and once per heap, in the heap's own scratch, before everything is zeroed).
+    if (const char *v = std::getenv("SYMAR_PLACE")) h->place_on = std::atoi(v) != 0;
+    if (e == cudaSuccess && h->place_on && h->device >= 0 && h->device < kMaxDevices) {
+        unsigned char *scratch = reinterpret_cast<unsigned char *>(h->seg0 + L.ll_off);
+        bool ok = false;
+        {
+            std::lock_guard<std::mutex> lock(g_place_mutex);
+            DevicePlace &dp = g_place[h->device];
+            if (!dp.tried) {
+                e = place_measure_sms(scratch, h->num_sms, h->max_smem, dp.sm_half, &dp.ok);
+                dp.tried = e == cudaSuccess;
+            }
+            ok = dp.ok;
+            std::memcpy(h->sm_half, dp.sm_half, sizeof h->sm_half);
+        }
+        if (e == cudaSuccess && ok) e = place_measure_heap(h->seg0, L.stride, P, L, h->sm_half, scratch, &h->home, &h->placed);
+    }
     if (e == cudaSuccess) e = cudaMemset(h->mem, 0, kCtlBytes);
     for (int q = 0; q < P && e == cudaSuccess; ++q) {
         e = cudaMemset(h->seg0 + (size_t)q * L.stride + L.ll_off, 0, L.seg_bytes - L.ll_off);
@@ -744,7 +782,8 @@ static int create_common(symheap_t **heap, int P, size_t bytes_per_rank, void *m
     // SYMAR_PDL = 0 turns programmatic dependent launch off; SYMAR_CTAS_PER_RANK and
     // SYMAR_THREADS fix the launch shape of every algorithm; SYMAR_DEBUG = 1 logs every
     // call's resolved algorithm and shape to stderr; SYMAR_TUNE = exhaustive makes
-    // allreduce_autotune time every algorithm and shape at every size (no pruning).
+    // allreduce_autotune time every algorithm and shape at every size (no pruning);
+    // SYMAR_PLACE = 0 (read above) skips the placement measurement: every reader takes copy 0.
     if (const char *v = std::getenv("SYMAR_SPIN_LIMIT_US")) {
         const long us = std::atol(v);
         if (us > 0) h->spin_ns = (uint64_t)us * 1000ull;
@@ -1138,6 +1177,26 @@ int symar_set_pdl(symheap_t *heap, int enabled)
 {
     if (!heap) return SYMAR_ERR_INVAL;
     heap->pdl = enabled != 0;
+    return SYMAR_OK;
+}
+
+int symar_set_placement(symheap_t *heap, int enabled)
+{
+    if (!heap) return SYMAR_ERR_INVAL;
+    heap->place_on = enabled != 0;
+    return SYMAR_OK;
+}
+
+int symar_placement(const symheap_t *heap, int *measured, int *sms_on_half1, unsigned long long *home_bits)
+{
+    if (!heap) return SYMAR_ERR_INVAL;
+    if (measured) *measured = heap->placed ? 1 : 0;
+    if (sms_on_half1) {
+        int n = 0;
+        for (int i = 0; i < 4; ++i) n += __builtin_popcountll(heap->sm_half[i]);
+        *sms_on_half1 = n;
+    }
+    if (home_bits) *home_bits = heap->home;
     return SYMAR_OK;
 }
 

@@ -26,6 +26,13 @@ KernelFn atomic_kernel_for(int dtype, int P, bool dbg);
 cudaError_t launch_kernel(KernelFn fn, int P, int ctas_per_rank, int threads, size_t smem_bytes,
                           const KArgs &args, cudaStream_t stream);
 
+// Placement on the chip's two L2 halves (symar_place.cu): which half every SM sits on, and which half
+// homes copy 0 of every flag / counter pair of a heap.  `scratch`: 3 * kPairBytes of device memory,
+// 8 KiB-aligned, left zeroed.  *ok = false (and all-zero results) when the measurement is not clean.
+cudaError_t place_measure_sms(unsigned char *scratch, int num_sms, int max_smem_optin, uint64_t sm_half[4], bool *ok);
+cudaError_t place_measure_heap(char *seg0, size_t stride, int P, const Layout &L, const uint64_t sm_half[4],
+                               unsigned char *scratch, uint64_t *home, bool *ok);
+
 // Checking build only (cudaErrorNotSupported otherwise): the kernel behind symar_check_selftest().
 cudaError_t launch_check_selftest(const KArgs &args, cudaStream_t stream);
 

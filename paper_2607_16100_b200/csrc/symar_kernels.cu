@@ -33,14 +33,14 @@
 namespace symar {
 
 // One-shot data phase with W words per thread: unit u covers bytes [4W u, 4W u + 4W).
-// For small messages the loads are issued BEFORE the CTA barrier that lets thread 0 publish
-// the exchange count, so that the barrier, the publication and the trigger of the dependent
-// launch cost nothing while the data travels (measured -0.03 us of 1.72 us at 16 KiB).
+// For small messages the loads are issued BEFORE the CTA barrier that lets threads 0 and 1 publish
+// the exchange count, so that the barrier and the publication cost nothing while the data
+// travels (measured -0.03 us of 1.72 us at 16 KiB).
 // (Measured and dropped: two units per thread in half as many CTAs, +0.1 to +0.3 us at 16 KiB;
 // leaving the trigger of the dependent launch to the kernel's end, +0.1 us at every size.)
 template <typename E, int P, int W, bool DBG>
 __device__ __forceinline__ void oneshot_data(const KArgs &a, char *out, uint64_t first, uint64_t step, bool ok,
-                                             uint32_t *count, uint32_t want)
+                                             int r, int c, uint32_t want)
 {
     const uint64_t bytes  = a.tail_bytes ? (a.nvec - 1) * 16 + a.tail_bytes : a.nvec * 16;
     const uint64_t nunits = (bytes + 4 * W - 1) / (4 * W);
@@ -57,8 +57,7 @@ __device__ __forceinline__ void oneshot_data(const KArgs &a, char *out, uint64_t
     // Every warp has consumed the count: publish the next one now, so that its store drains
     // while the data is in flight.
     __syncthreads();
-    if (threadIdx.x == 0) *count = want;
-    if (a.pdl) pdl_launch_dependents();       // the next call may take its seats now
+    publish_u32(a, r, c, kCtrReady, want);
     if (have && late) {
 #pragma unroll
         for (int q = 0; q < P; ++q)
@@ -88,8 +87,8 @@ __global__ void __launch_bounds__(kMaxThreads) oneshot_kernel(const KArgs a)
     const int c = blockIdx.x, r = blockIdx.y, C = gridDim.x;
     const uint32_t t = threadIdx.x, T = blockDim.x;
     char *seg_r = a.seg0 + (size_t)r * a.stride;
-    uint32_t *count = SYMAR_PTR(reinterpret_cast<uint32_t *>(seg_r + a.epoch_off + ready_count_off(c)), 4, kRegCtr);
-    const ExchangePtrs xp = exchange_ptrs<P>(a, a.ready_off, r, c);
+    const uint32_t *count = reinterpret_cast<const uint32_t *>(counters_near(a, r, c) + kCtrReady);
+    const ExchangePtrs xp = exchange_ptrs<P>(a, a.ready_off, kPairReady, r, c);
     if (a.pdl) {
         // Made resident early, this CTA has time while its predecessor still runs: pull the peers'
         // input lines of its first passes towards L2 (a hint only -- if a line is still being written,
@@ -102,6 +101,13 @@ __global__ void __launch_bounds__(kMaxThreads) oneshot_kernel(const KArgs a)
             for (int q = 0; q < P; ++q) prefetch_l2(a.seg0 + (size_t)q * a.stride + a.in_off + off);
         }
         pdl_wait_holding(xp.signal, xp.mine, count);   // the previous call has left the heap
+        // The successor may take its seats at once: it then has this whole call for its own address
+        // arithmetic and prefetch hints before its wait ends.  (Measured against a trigger after the
+        // exchange, with flag reads placed on the near L2 half: 1.53 -> 1.43 us at 128 B, 1.72 -> 1.62 us
+        // at 16 KiB, 2.04 -> 1.90 us at 64 KiB, 2.34 -> 2.01 us per call of the decode-step graph; the
+        // same early trigger gains nothing in the two-shot kernel and costs 0.1-0.2 us in the LL kernel,
+        // which have no such prologue.)
+        pdl_launch_dependents();
     }
     if (DBG) debug_delay(a, r, c);
     if (DBG && a.dbg_mute == r) return;       // test hook: this rank never joins
@@ -127,15 +133,15 @@ __global__ void __launch_bounds__(kMaxThreads) oneshot_kernel(const KArgs a)
     char *out = seg_r + a.out_off;
     const uint64_t first = (uint64_t)c * T + t, step = (uint64_t)C * T;
     const uint32_t narrow = (a.variant >> 8) & 3u;     // bytes per thread: 16, 8 or 4
-    if (narrow == 2) oneshot_data<E, P, 1, DBG>(a, out, first, step, ok, count, want);
-    else if (narrow == 1) oneshot_data<E, P, 2, DBG>(a, out, first, step, ok, count, want);
-    else oneshot_data<E, P, 4, DBG>(a, out, first, step, ok, count, want);
+    if (narrow == 2) oneshot_data<E, P, 1, DBG>(a, out, first, step, ok, r, c, want);
+    else if (narrow == 1) oneshot_data<E, P, 2, DBG>(a, out, first, step, ok, r, c, want);
+    else oneshot_data<E, P, 4, DBG>(a, out, first, step, ok, r, c, want);
     if (prior_art) {
-        uint32_t *dcount = SYMAR_PTR(reinterpret_cast<uint32_t *>(seg_r + a.epoch_off + done_count_off(c)), 4, kRegCtr);
+        const uint32_t *dcount = reinterpret_cast<const uint32_t *>(counters_near(a, r, c) + kCtrDone);
         uint32_t dwant;
         __syncthreads();
-        flag_exchange<P, true>(a, a.done_off, dcount, r, c, !ok, false, dwant);
-        if (t == 0) *dcount = dwant;
+        flag_exchange<P, true>(a, a.done_off, kPairDone, dcount, r, c, !ok, false, dwant);
+        publish_u32(a, r, c, kCtrDone, dwant);
     }
     if (DBG) {
         debug_stamp_out(a);
@@ -169,9 +175,8 @@ __global__ void __launch_bounds__(kMaxThreads) twoshot_kernel(const KArgs a)
     SYMAR_CHECK_BEGIN_ALLREDUCE(a, P);
     const int c = blockIdx.x, r = blockIdx.y, C = gridDim.x;
     const uint32_t t = threadIdx.x, T = blockDim.x;
-    char *seg_r = a.seg0 + (size_t)r * a.stride;
-    uint32_t *rcount = SYMAR_PTR(reinterpret_cast<uint32_t *>(seg_r + a.epoch_off + ready_count_off(c)), 4, kRegCtr);
-    uint32_t *dcount = SYMAR_PTR(reinterpret_cast<uint32_t *>(seg_r + a.epoch_off + done_count_off(c)), 4, kRegCtr);
+    const uint32_t *rcount = reinterpret_cast<const uint32_t *>(counters_near(a, r, c) + kCtrReady);
+    const uint32_t *dcount = reinterpret_cast<const uint32_t *>(counters_near(a, r, c) + kCtrDone);
     if (a.pdl) pdl_wait();                    // the previous call has left the heap
     if (DBG) debug_delay(a, r, c);
     if (DBG && a.dbg_mute == r) return;       // test hook: this rank never joins
@@ -179,7 +184,7 @@ __global__ void __launch_bounds__(kMaxThreads) twoshot_kernel(const KArgs a)
     // reduce-scatter: which vectors rank r owns
     uint32_t rwant, dwant;
     if (DBG) debug_phase(a, 0);
-    bool ok = flag_exchange<P, false>(a, a.ready_off, rcount, r, c, false, true, rwant);
+    bool ok = flag_exchange<P, false>(a, a.ready_off, kPairReady, rcount, r, c, false, true, rwant);
     if (a.pdl) pdl_launch_dependents();
     if (DBG) debug_phase(a, 1);               // every peer's input is ready
     if (ok) {
@@ -224,13 +229,11 @@ __global__ void __launch_bounds__(kMaxThreads) twoshot_kernel(const KArgs a)
     if (DBG) debug_phase(a, 2);               // thread 0's share reduced, its stores issued
     __syncthreads();
     if (DBG) debug_phase(a, 3);               // the whole CTA's stores issued
-    if (DBG) flag_exchange<P, true, 5>(a, a.done_off, dcount, r, c, !ok, false, dwant);   // 5: release fence done, signal sent
-    else flag_exchange<P, true>(a, a.done_off, dcount, r, c, !ok, false, dwant);
+    if (DBG) flag_exchange<P, true, 5>(a, a.done_off, kPairDone, dcount, r, c, !ok, false, dwant);   // 5: release fence done, signal sent
+    else flag_exchange<P, true>(a, a.done_off, kPairDone, dcount, r, c, !ok, false, dwant);
     if (DBG) debug_phase(a, 4);               // every peer's part has landed here
-    if (t == 0) {
-        *rcount = rwant;
-        *dcount = dwant;
-    }
+    publish_u32(a, r, c, kCtrReady, rwant);
+    publish_u32(a, r, c, kCtrDone, dwant);
     if (DBG) {
         debug_stamp_out(a);
         debug_phase(a, 7);
@@ -321,7 +324,7 @@ __global__ void __launch_bounds__(kLLMaxThreads) ll_kernel(const KArgs a)
     const int c = blockIdx.x, r = blockIdx.y, C = gridDim.x;
     const uint32_t t = threadIdx.x, T = blockDim.x;
     char *seg_r  = a.seg0 + (size_t)r * a.stride;
-    uint64_t *ep = SYMAR_PTR(reinterpret_cast<uint64_t *>(seg_r + a.epoch_off) + c, 8, kRegCtr);
+    const uint64_t *ep = reinterpret_cast<const uint64_t *>(counters_near(a, r, c) + kCtrLL);
     if (a.pdl) {
         pdl_wait();                           // the previous call has left the heap
         pdl_launch_dependents();
@@ -414,7 +417,7 @@ __global__ void __launch_bounds__(kLLMaxThreads) ll_kernel(const KArgs a)
         // iteration i-1 -- so the sub-buffer of parity (i+1)&1 is free.
     }
     __syncthreads();          // every thread has read the counter before it moves
-    if (t == 0) *ep = n0 + a.iters;
+    publish_u64(a, r, c, kCtrLL, n0 + a.iters);
     if (DBG) {
         debug_stamp_out(a);
         debug_phase(a, 7);
@@ -474,7 +477,7 @@ __global__ void __launch_bounds__(kLLMaxThreads) ll_small_kernel(const KArgs a)
     const int c = blockIdx.x, r = blockIdx.y;
     const uint32_t t = threadIdx.x, T = blockDim.x;
     char *seg_r  = a.seg0 + (size_t)r * a.stride;
-    uint64_t *ep = SYMAR_PTR(reinterpret_cast<uint64_t *>(seg_r + a.epoch_off) + c, 8, kRegCtr);
+    const uint64_t *ep = reinterpret_cast<const uint64_t *>(counters_near(a, r, c) + kCtrLL);
     const uint64_t bytes = a.tail_bytes ? (a.nvec - 1) * 16 + a.tail_bytes : a.nvec * 16;
     const uint64_t lo    = ((uint64_t)c * T + t) * (4 * W);
     const uint32_t valid = lo < bytes ? (bytes - lo < 4u * W ? (uint32_t)(bytes - lo) : 4u * W) : 0u;
@@ -545,7 +548,7 @@ __global__ void __launch_bounds__(kLLMaxThreads) ll_small_kernel(const KArgs a)
         if (DBG) debug_phase(a, 4);
     }
     __syncthreads();          // every thread has read the counter before it moves
-    if (t == 0) *ep = n;
+    publish_u64(a, r, c, kCtrLL, n);
     if (DBG) {
         debug_stamp_out(a);
         debug_phase(a, 7);
@@ -570,7 +573,7 @@ __global__ void __launch_bounds__(kMaxThreads) sentinel_kernel(const KArgs a)
     const int c = blockIdx.x, r = blockIdx.y, C = gridDim.x;
     const uint32_t t = threadIdx.x, T = blockDim.x;
     char *seg_r  = a.seg0 + (size_t)r * a.stride;
-    uint64_t *ep = SYMAR_PTR(reinterpret_cast<uint64_t *>(seg_r + a.epoch_off) + c, 8, kRegCtr);
+    const uint64_t *ep = reinterpret_cast<const uint64_t *>(counters_near(a, r, c) + kCtrLL);
     if (a.pdl) {
         pdl_wait();
         pdl_launch_dependents();
@@ -642,7 +645,7 @@ __global__ void __launch_bounds__(kMaxThreads) sentinel_kernel(const KArgs a)
         if (a.iters > 1) fence_acq_rel();
     }
     __syncthreads();
-    if (t == 0) *ep = n0 + a.iters;
+    publish_u64(a, r, c, kCtrLL, n0 + a.iters);
     if (DBG) {
         debug_stamp_out(a);
         debug_phase(a, 7);
@@ -724,7 +727,7 @@ __global__ void __launch_bounds__(kPushTwoshotMaxThreads) twoshot_push_kernel(co
     const int c = blockIdx.x, r = blockIdx.y, C = gridDim.x;
     const uint32_t t = threadIdx.x, T = blockDim.x;
     char *seg_r  = a.seg0 + (size_t)r * a.stride;
-    uint64_t *ep = SYMAR_PTR(reinterpret_cast<uint64_t *>(seg_r + a.epoch_off) + c, 8, kRegCtr);
+    const uint64_t *ep = reinterpret_cast<const uint64_t *>(counters_near(a, r, c) + kCtrLL);
     if (a.pdl) {
         pdl_wait();
         pdl_launch_dependents();
@@ -818,7 +821,7 @@ __global__ void __launch_bounds__(kPushTwoshotMaxThreads) twoshot_push_kernel(co
         if (SENT && a.iters > 1) fence_acq_rel();      // restored sentinels before the sub-buffer's next use
     }
     __syncthreads();
-    if (t == 0) *ep = n0 + a.iters;
+    publish_u64(a, r, c, kCtrLL, n0 + a.iters);
     if (DBG) {
         debug_stamp_out(a);
         debug_phase(a, 7);

@@ -29,7 +29,7 @@ _ERR_NAMES = {
     ERR_TIMEOUT: "SYMAR_ERR_TIMEOUT", ERR_UNSUPPORTED: "SYMAR_ERR_UNSUPPORTED",
 }
 
-MAX_RANKS, MAX_CTAS, LL_SLOTS, LL_SLOT_VECS, ALIGN = 8, 160, 64, 1024, 4096
+MAX_RANKS, MAX_CTAS, LL_SLOTS, LL_SLOT_VECS, ALIGN = 8, 160, 64, 1024, 8192
 
 # every symbol include/symar.h declares: (name, restype, argtypes)
 SIGNATURES = [
@@ -60,6 +60,8 @@ SIGNATURES = [
     ("symar_set_launch", c_int, [c_void_p, c_int, c_int, c_int]),
     ("symar_set_variant", c_int, [c_void_p, c_int, c_uint]),
     ("symar_set_pdl", c_int, [c_void_p, c_int]),
+    ("symar_set_placement", c_int, [c_void_p, c_int]),
+    ("symar_placement", c_int, [c_void_p, POINTER(c_int), POINTER(c_int), POINTER(ctypes.c_ulonglong)]),
     ("symar_set_scratch_limit", c_int, [c_void_p, c_size_t]),
     ("symar_set_spin_limit_us", c_int, [c_void_p, c_uint]),
     ("symar_debug_inject", c_int, [c_void_p, c_int, c_uint, c_uint]),
@@ -304,6 +306,15 @@ class SymHeap:
 
     def set_pdl(self, enabled: bool) -> None:
         _ck(self._lib.symar_set_pdl(self._h, 1 if enabled else 0), "symar_set_pdl")
+
+    def set_placement(self, enabled: bool) -> None:
+        _ck(self._lib.symar_set_placement(self._h, 1 if enabled else 0), "symar_set_placement")
+
+    def placement(self):
+        """(measured cleanly?, SMs on the second L2 half, home bits)"""
+        m, n, hb = c_int(), c_int(), ctypes.c_ulonglong()
+        _ck(self._lib.symar_placement(self._h, byref(m), byref(n), byref(hb)), "symar_placement")
+        return bool(m.value), n.value, hb.value
 
     def set_scratch_limit(self, payload_bytes_per_iteration: int) -> None:
         _ck(self._lib.symar_set_scratch_limit(self._h, payload_bytes_per_iteration), "symar_set_scratch_limit")

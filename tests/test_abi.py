@@ -71,7 +71,9 @@ def test_required_bytes_layout(lib, P):
     # Table I, two-shot LL128 atomic: about D / N per iteration; this build gives every
     # rank two parity halves of 512 KiB x P of 128-byte accumulator lines
     atomic = 2 * (512 << 10) * P
-    flags = 2 * symar.MAX_CTAS * 32 + symar.MAX_CTAS * 8
+    # flags and counters: two copies of everything, one per half of the chip's L2, in 8 KiB pairs
+    # (ready flags 2 pairs, done flags 2 pairs, counters 1 pair)
+    flags = 5 * 8192
     assert total >= P * (user + ll + sentinel + atomic + flags)
     assert total <= P * (user + ll + sentinel + atomic + flags + 16 * symar.ALIGN) + 4096
     assert total % symar.ALIGN == 0

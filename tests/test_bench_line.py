@@ -59,6 +59,7 @@ def canned_latency_record():
             "p50_us": 1.8461234567, "best": dict(algo_row), "per_algo": per_algo, "repeats": [dict(rep)] * 5,
             "ratio_to_sol_over_repeats": dict(spread), "p50_us_over_repeats": dict(spread),
             "oneshot_release_signal": {"p50_us": 2.3123456789, "bit_exact": True},
+            "without_placement_on_l2_halves": {"p50_us": 1.9876543219, "bit_exact": True},
             "system_scope_build": {"oneshot": {"p50_us": 2.5123456789, "bit_exact": True},
                                    "ll": {"p50_us": 3.0123456789, "bit_exact": True}},
             "oracle_cpu": {"single_thread_us": 123.456789, "all_cores_us": 45.6789123, "cores": 16},

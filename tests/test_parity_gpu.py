@@ -572,6 +572,51 @@ def test_default_wait_bound_is_a_fraction_of_a_second(algo):
         h.destroy()
 
 
+@pytest.mark.parametrize("P", [2, 4, 8])
+def test_placement_on_the_two_l2_halves_changes_no_bits(P):
+    # Flags and counters are kept twice, one copy per half of the chip's L2; a reader takes the copy of its own
+    # half when the heap could measure where things sit, copy 0 otherwise or when told so.  Calls with
+    # placement on and off alternate on one heap (every call updates both copies): same bits as the oracle.
+    h = symar.SymHeap.on_torch(P, 2 << 20)
+    try:
+        measured, sms_on_second_half, home = h.placement()
+        if measured:                        # a B200: two halves, each with a good part of the SMs
+            n = torch.cuda.get_device_properties(0).multi_processor_count
+            assert n // 4 <= sms_on_second_half <= 3 * n // 4
+        for i, (algo, count) in enumerate([(symar.ONESHOT, 8192), (symar.TWOSHOT, 8192), (symar.LL, 8192),
+                                           (symar.ONESHOT, 77), (symar.TWOSHOT, 70001), (symar.LL, 1023),
+                                           (symar.SENTINEL, 4099), (symar.TWOSHOT_LL, 4099), (symar.ONESHOT, 70001),
+                                           (symar.TWOSHOT, 300000), (symar.ONESHOT, 8192), (symar.LL, 8192)]):
+            h.set_placement(i % 2 == 0)
+            x = synth.make_inputs("normal", "bf16", P, count, seed=500 + i)
+            assert_bits(run(h, x, symar.BF16, algo), O.allreduce(x), f"placement {'on' if i % 2 == 0 else 'off'} {algo} {count}")
+        # the sibling collectives share the flags and counters
+        h.set_placement(True)
+        x = synth.make_inputs("normal", "bf16", P, 4096 * P, seed=9)
+        for q in range(P):
+            h.write_rank(q, 0, x[q])
+        assert h.reduce_scatter(0, 1 << 20, 4096, symar.BF16) == 0
+        torch.cuda.synchronize()
+        got = np.stack([h.read_rank(q, 1 << 20, 4096, np.uint16) for q in range(P)])
+        assert np.array_equal(got, O.reduce_scatter(x)) and h.status()[0] == symar.OK
+    finally:
+        h.set_placement(True)
+        torch.cuda.synchronize()
+        h.destroy()
+
+
+def test_placement_can_be_switched_off_in_the_environment(monkeypatch):
+    monkeypatch.setenv("SYMAR_PLACE", "0")
+    h = symar.SymHeap.on_torch(4, 1 << 18)
+    try:
+        assert h.placement() == (False, 0, 0)
+        x = synth.make_inputs("normal", "bf16", 4, 8192, seed=3)
+        assert_bits(run(h, x, symar.BF16, symar.ONESHOT, out_off=1 << 17), O.allreduce(x))
+    finally:
+        torch.cuda.synchronize()
+        h.destroy()
+
+
 def test_host_buffer_entry_point(heaps):
     h = heaps[8]
     count = 50000
