@@ -443,16 +443,25 @@ def latency_suite(torch, symar, synth, hbm_gbs, quick=False, autotune=True):
             floor11 = empty_floor(1, 1, 1)
             t_bytes_us = bytes_us(16384, P)
             sol = floor["p50"] + rt_ns / 1000.0 + t_bytes_us
-            # the whole comparison again, bound and kernel interleaved in this process, REPEATS times
-            rep_rows = []
+            # the whole comparison again, bound and kernel interleaved in this process, REPEATS times; the
+            # bound then uses the SMALLEST empty launch seen (it is a floor; its p50 wanders between 0.50
+            # and 0.73 us from one measurement to the next) and the median of the pair medians
+            rep_rows = [{"p50_us": best["p50"], "empty_launch_us": floor["p50"],
+                         "flag_round_trip_median_us": rt0["median_us"], "flag_round_trip_min_us": rt0["min_us"]}]
             for _ in range(REPEATS):
                 rt_i = sample_flag_round_trips(torch, symar)
                 fl_i = empty_floor(best["ctas_per_rank"], P, best["threads"])["p50"]
                 p_i = bench_size(8192, (symar.AUTO,))["auto"]["p50"]
-                sol_i = fl_i + rt_i["median_us"] + t_bytes_us
                 rep_rows.append({"p50_us": p_i, "empty_launch_us": fl_i, "flag_round_trip_median_us": rt_i["median_us"],
-                                 "flag_round_trip_min_us": rt_i["min_us"], "sol_us": sol_i, "ratio_to_sol": p_i / sol_i,
-                                 "ratio_to_sol_fastest_pair": p_i / (fl_i + rt_i["min_us"] + t_bytes_us)})
+                                 "flag_round_trip_min_us": rt_i["min_us"]})
+            floor_us = min(r_["empty_launch_us"] for r_ in rep_rows)
+            rt_us = float(np.median([r_["flag_round_trip_median_us"] for r_ in rep_rows]))
+            rt_min_us = min(r_["flag_round_trip_min_us"] for r_ in rep_rows)
+            sol = floor_us + rt_us + t_bytes_us
+            sol_fast = floor_us + rt_min_us + t_bytes_us
+            for r_ in rep_rows:
+                r_["ratio_to_sol"] = r_["p50_us"] / sol
+            p50_all = spread([r_["p50_us"] for r_ in rep_rows])
             # the same call with every reader on copy 0 of the flags and counters (no placement on the L2 halves)
             h.set_placement(False)
             unplaced = bench_size(8192, (symar.AUTO,))["auto"]
@@ -479,10 +488,10 @@ def latency_suite(torch, symar, synth, hbm_gbs, quick=False, autotune=True):
                 "workload": "c2: P=8, bf16, 8192 elements (16 KiB) per rank, N(0,1); buffers L2-resident (warm)",
                 "harness": f"{K} back-to-back calls in one CUDA graph, one replay = one sample, {reps} samples; "
                            "numerator and denominator use the same harness",
-                "p50_us": best["p50"], "best": best, "per_algo": row,
+                "p50_us": p50_all["median"], "best": best, "per_algo": row,
                 "repeats": rep_rows,
                 "ratio_to_sol_over_repeats": spread([r_["ratio_to_sol"] for r_ in rep_rows]),
-                "p50_us_over_repeats": spread([r_["p50_us"] for r_ in rep_rows]),
+                "p50_us_over_repeats": p50_all,
                 "twoshot_atomic_not_bit_reproducible": bench_size(8192, (symar.TWOSHOT_ATOMIC,))["twoshot_atomic"],
                 "prior_art_two_barrier_oneshot": {
                     "p50_us": prior["p50"], "bit_exact": prior["bit_exact"], "ctas_per_rank": prior["ctas_per_rank"],
@@ -508,15 +517,19 @@ def latency_suite(torch, symar, synth, hbm_gbs, quick=False, autotune=True):
                                      "CTA's start; median of 31 instrumented calls; phases as in symar_debug_phases",
                 "oracle_cpu": oracle_us(O, load_inputs(8192)),
                 "sol_us": sol,
-                "sol_parts_us": {"empty_launch_same_shape": floor["p50"], "empty_launch_1x1": floor11["p50"],
-                                 "flag_round_trip": rt_ns / 1000.0, "bytes_at_peak": t_bytes_us},
-                "ratio_to_sol": best["p50"] / sol,
-                "sol_note": "flag round trip = the MEDIAN over SM pairs spread over the chip (the exchange needs every "
-                            "pair of ranks, wherever their CTAs sit); the same bound with the FASTEST pair follows",
-                "sol_fastest_pair_us": floor["p50"] + rt_min_ns / 1000.0 + t_bytes_us,
-                "ratio_to_sol_fastest_pair": best["p50"] / (floor["p50"] + rt_min_ns / 1000.0 + t_bytes_us),
-                "sol_strictest_us": floor11["p50"] + rt_min_ns / 1000.0 + t_bytes_us,
-                "ratio_to_sol_strictest": best["p50"] / (floor11["p50"] + rt_min_ns / 1000.0 + t_bytes_us),
+                "sol_parts_us": {"empty_launch_same_shape": floor_us, "empty_launch_1x1": floor11["p50"],
+                                 "flag_round_trip": rt_us, "bytes_at_peak": t_bytes_us},
+                "ratio_to_sol": p50_all["median"] / sol,
+                "sol_note": "empty launch = the smallest p50 over the repeats; flag round trip = the MEDIAN over SM pairs "
+                            "spread over the chip (the exchange needs every pair of ranks, wherever their CTAs sit; two hops "
+                            "through L2 of a flag that is not placed), median over the repeats; the same bound with the "
+                            "FASTEST pair follows.  The kernel's own exchange is one hop and a poll of a flag placed on the "
+                            "reader's L2 half, and its launch overlaps the previous call, so this form is a yardstick, not a "
+                            "strict floor; the fastest-pair form is the strict one",
+                "sol_fastest_pair_us": sol_fast,
+                "ratio_to_sol_fastest_pair": p50_all["median"] / sol_fast,
+                "sol_strictest_us": min(floor11["p50"], floor_us) + rt_min_us + t_bytes_us,
+                "ratio_to_sol_strictest": p50_all["median"] / (min(floor11["p50"], floor_us) + rt_min_us + t_bytes_us),
                 "sol_strictest_note": "empty 1x1 launch + fastest SM pair + bytes at peak",
                 "paper_style_sol_us": (2 * fence_ns + rt_ns / 2) / 1000.0,
                 "fence_us": fence_ns / 1000.0,
@@ -665,6 +678,12 @@ def latency_suite(torch, symar, synth, hbm_gbs, quick=False, autotune=True):
         # C5: 160 calls in one graph
         calls, count = 160, 8192 * 4
         nb = count * 2
+        if autotune:
+            # the launch shape for this message size as it occurs in the trace -- every call on its own buffers --
+            # measured on this GPU (untimed set-up, as a deployment does once for its decode step)
+            t0 = time.time()
+            h.autotune_stream(symar.BF16, count, calls)
+            res["autotune_stream_seconds"] = time.time() - t0
         xs = [synth.make_inputs("normal", "bf16", P, count, synth.seed_for_config(5), call=k) for k in range(calls)]
         for k in range(calls):
             for q in range(P):
@@ -686,17 +705,29 @@ def latency_suite(torch, symar, synth, hbm_gbs, quick=False, autotune=True):
         floor = empty_floor(c, P, t)
         t_bytes_us = bytes_us(nb, P)
         sol = floor["p50"] + rt_ns / 1000.0 + t_bytes_us
-        dec_rows = []
+        dec_rows = [{"per_call_us": r["p50"], "empty_launch_us": floor["p50"], "flag_round_trip_median_us": rt_ns / 1000.0,
+                     "flag_round_trip_min_us": rt_min_ns / 1000.0}]
         for _ in range(REPEATS):
             rt_i = sample_flag_round_trips(torch, symar)
             fl_i = empty_floor(c, P, t)["p50"]
             p_i = time_graph(torch, g, stream, calls, n_dec)["p50"]
-            sol_i = fl_i + rt_i["median_us"] + t_bytes_us
-            dec_rows.append({"per_call_us": p_i, "empty_launch_us": fl_i,
-                             "flag_round_trip_median_us": rt_i["median_us"], "sol_us": sol_i,
-                             "ratio_to_sol": p_i / sol_i})
-        res.update({"step_total_us_p50": r["p50"] * calls, "per_call_us": r, "sol_per_call_us": sol,
-                    "ratio_to_sol": r["p50"] / sol, "algo": names[a], "ctas_per_rank": c, "threads": t,
+            dec_rows.append({"per_call_us": p_i, "empty_launch_us": fl_i, "flag_round_trip_median_us": rt_i["median_us"],
+                             "flag_round_trip_min_us": rt_i["min_us"]})
+        floor_us = min(d_["empty_launch_us"] for d_ in dec_rows)
+        sol = floor_us + float(np.median([d_["flag_round_trip_median_us"] for d_ in dec_rows])) + t_bytes_us
+        sol_fast = floor_us + min(d_["flag_round_trip_min_us"] for d_ in dec_rows) + t_bytes_us
+        for d_ in dec_rows:
+            d_["ratio_to_sol"] = d_["per_call_us"] / sol
+        per_call = float(np.median([d_["per_call_us"] for d_ in dec_rows]))
+        res.update({"step_total_us_p50": per_call * calls, "per_call_us": dict(r, p50=per_call), "sol_per_call_us": sol,
+                    "ratio_to_sol": per_call / sol, "algo": names[a], "ctas_per_rank": c, "threads": t,
+                    "sol_fastest_pair_us": sol_fast,
+                    "ratio_to_sol_fastest_pair": per_call / sol_fast,
+                    "sol_note": "smallest empty launch of the same shape over the repeats + the MEDIAN SM pair's flag round "
+                                "trip (two hops through L2, flag not placed; median over the repeats) + bytes at peak; the "
+                                "exchange itself needs one hop and a poll of a flag placed on the reader's L2 half, and the "
+                                "successor's launch overlaps this call, so this form is a yardstick, not a strict floor; "
+                                "the fastest-pair form is the strict one",
                     "repeats": dec_rows, "ratio_to_sol_over_repeats": spread([d_["ratio_to_sol"] for d_ in dec_rows]),
                     "oracle_cpu_one_call": oracle_us(O, xs[0]),
                     "bit_exact": exact, "calls": calls, "bytes_per_rank": nb,
@@ -803,7 +834,6 @@ def compact_line(bw, lat, details):
             "sol_us": _r(c2.get("sol_us"), 3), "ratio_to_sol": _r(c2.get("ratio_to_sol"), 3),
             "repeats": rs.get("n"), "ratio_median": _r(rs.get("median"), 3), "ratio_min": _r(rs.get("min"), 3),
             "ratio_max": _r(rs.get("max"), 3),
-            "sol_fastest_pair_us": _r(c2.get("sol_fastest_pair_us"), 3),
             "ratio_to_sol_fastest_pair": _r(c2.get("ratio_to_sol_fastest_pair"), 3),
             "bit_exact": all(v.get("bit_exact") for v in c2.get("per_algo", {}).values()),
             "ll_p50_us": _r((c2.get("per_algo", {}).get("ll") or {}).get("p50"), 3),
@@ -811,7 +841,6 @@ def compact_line(bw, lat, details):
             "unplaced_p50_us": _r((c2.get("without_placement_on_l2_halves") or {}).get("p50_us"), 3),
             "sys_scope_p50_us": {k: _r((sysb.get(k) or {}).get("p50_us"), 3) for k in ("oneshot", "ll")}
             if "error" not in sysb else None,
-            "oracle_cpu_us": _r((c2.get("oracle_cpu") or {}).get("all_cores_us"), 1),
         }
     if lat and "decode_trace" in lat:
         line["decode_trace"] = {}
@@ -819,13 +848,14 @@ def compact_line(bw, lat, details):
             rs = d.get("ratio_to_sol_over_repeats", {})
             line["decode_trace"][key] = {
                 "us_per_call": _r((d.get("per_call_us") or {}).get("p50"), 3), "ratio_to_sol": _r(d.get("ratio_to_sol"), 3),
-                "ratio_min": _r(rs.get("min"), 3), "ratio_max": _r(rs.get("max"), 3), "algo": d.get("algo"),
+                "ratio_min": _r(rs.get("min"), 3), "ratio_max": _r(rs.get("max"), 3),
+                "ratio_fastest_pair": _r(d.get("ratio_to_sol_fastest_pair"), 3), "algo": d.get("algo"),
                 "bit_exact": d.get("bit_exact")}
     if lat and "sweep" in lat:
         line["sweep_ok"] = {"selector_within_5pct": all(r_.get("selector_within_5pct") for r_ in lat["sweep"]),
                             "bit_exact": all(r_.get("bit_exact") for r_ in lat["sweep"])}
-    names = sorted(Path(d_).name for d_ in details)
-    line["details"] = (str(Path(details[0]).parent) + "/{" + ",".join(names) + "}") if details else None
+    which = ",".join(sorted(Path(d_).stem.replace("results_", "") for d_ in details))
+    line["details"] = (str(Path(details[0]).parent) + "/results_{" + which + "}.json") if details else None
     return finite(line)
 
 

@@ -236,6 +236,15 @@ int allreduce_autotune(symheap_t *heap, symar_dtype_t dtype);
  * their message sizes, and for sizes beyond the 64 MiB grid.  OVERWRITES the user region. */
 int allreduce_autotune_size(symheap_t *heap, symar_dtype_t dtype, size_t count);
 
+/* The same for one message size as it occurs in a STREAM of calls that each have their own buffers
+ * (the AllReduces of a decode step: 2 per layer, every one on activations that were just produced):
+ * every candidate is timed in a graph of `calls` (2..1024) back-to-back calls, call k on the k-th of
+ * `calls` input / output pairs laid side by side in the user region (2 * calls * count elements,
+ * rounded up to SYMAR_ALIGN per buffer, must fit).  With enough pairs the inputs are not in L2 when
+ * a call starts, and the shape that is best then is not always the one that is best on warm buffers.
+ * Records the winners for that size's bucket only.  OVERWRITES the user region.                 */
+int allreduce_autotune_stream(symheap_t *heap, symar_dtype_t dtype, size_t count, int calls);
+
 /* What the last allreduce() on this heap launched (for reporting). */
 int symar_last_choice(const symheap_t *heap, symar_algo_t *algo,
                       int *ctas_per_rank, int *threads);
@@ -278,7 +287,8 @@ int symar_set_launch(symheap_t *heap, symar_algo_t algo, int ctas_per_rank, int 
  * single-iteration kernel holds back its first poll;
  * two-shot: bit 0 = contiguous chunks also for large messages (no block-cyclic
  * ownership), bit 1 = 16-byte instead of 32-byte accesses for large messages,
- * bit 2 = never use the bulk-copy kernel, bits 8-10 = its pipeline depth (0:
+ * bit 2 = never use the bulk-copy kernel, bit 6 = 8 instead of 16 bytes per thread and
+ * trip for messages below 1 MiB, bits 8-10 = the bulk kernel's pipeline depth (0:
  * default), bits 12-13 = log2 of its tile size over 4 KiB.                        */
 int symar_set_variant(symheap_t *heap, symar_algo_t algo, unsigned int variant);
 

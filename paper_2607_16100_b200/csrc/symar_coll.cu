@@ -125,13 +125,15 @@ __global__ void __launch_bounds__(kMaxThreads) coll_kernel(const CollArgs a)
     const uint32_t t = threadIdx.x, T = blockDim.x;
     const KArgs &k = a.k;
     const uint32_t *count = reinterpret_cast<const uint32_t *>(counters_near(k, r, c) + kCtrReady);
-    if (k.pdl) pdl_wait();
+    if (k.pdl) {
+        pdl_wait();
+        pdl_launch_dependents();      // as in the one-shot AllReduce kernel: the successor may take its seats at once
+    }
 
     uint32_t want;
     const bool ok = flag_exchange<P, false>(k, k.ready_off, kPairReady, count, r, c, false, true, want);
     __syncthreads();
     publish_u32(k, r, c, kCtrReady, want);
-    if (k.pdl) pdl_launch_dependents();
     if (!ok) return;
     if (OP == kOpReduce && r != a.root) return;          // only the root receives the sum
 

@@ -83,6 +83,7 @@ struct symheap {
     int       env_algo     = 0;       // SYMAR_ALGO override of SYMAR_AUTO, 0 = none
     bool      debug_log    = false;   // SYMAR_DEBUG=1: one stderr line per call
     bool      tune_exhaustive = false;   // SYMAR_TUNE=exhaustive: the tuner prunes nothing
+    int       tune_rotate = 0;        // tuner: > 0 = every call of a timing graph has its own buffers (that many pairs)
     bool      placed   = false;       // sm_half / home were measured cleanly
     bool      place_on = true;        // readers take the copy of their own L2 half (SYMAR_PLACE=0 / symar_set_placement)
     uint64_t  sm_half[4] = {0, 0, 0, 0};
@@ -181,7 +182,12 @@ static LaunchCfg default_cfg(const symheap *h, int algo, uint64_t nvec)
     // messages are bound by the per-thread instruction chain, so a thread takes
     // 4 or 8 bytes instead of 16 (measured -0.3 us at 16 KiB, P = 8).
     uint64_t units = work;
-    if (algo == SYMAR_ONESHOT) {
+    if (algo == SYMAR_TWOSHOT && h->P == 8 && nvec * 16 <= (256u << 10)) {
+        // 8 bytes per thread and trip: measured 0.35-0.45 us ahead of 16 bytes from 16 KiB to 256 KiB among
+        // eight ranks (no gain among four, none from 512 KiB)
+        c.variant = 0x40;
+        units     = work * 2;
+    } else if (algo == SYMAR_ONESHOT) {
         const uint64_t bytes = nvec * 16;
         const int narrow = bytes <= (8u << 10) ? 2 : (bytes <= (128u << 10) ? 1 : 0);
         c.variant = narrow << 8;
@@ -459,13 +465,17 @@ static int time_calls(symheap *h, cudaStream_t s, size_t count, int dtype, int a
                       double *us_out, double give_up_us = 0.0)
 {
     const size_t bytes = count * elem_size(dtype);
-    const void *in = h->seg0;
-    void *out      = h->seg0 + round_up(bytes, kAlign);
+    // Warm: every call on the same input and output.  Streaming (tune_rotate pairs): call k reads and writes its
+    // own pair of buffers, as the calls of a decode step do; the graph then holds one call per pair.
+    const size_t slice = round_up(bytes, kAlign);
+    const int pairs    = h->tune_rotate > 0 ? h->tune_rotate : 1;
+    if (h->tune_rotate > 0) K = pairs;
     cudaGraph_t graph;
     cudaGraphExec_t exec;
     CU(cudaStreamBeginCapture(s, cudaStreamCaptureModeThreadLocal));
     int rc = SYMAR_OK;
-    for (int k = 0; k < K && rc == SYMAR_OK; ++k) rc = run(h, in, out, count, dtype, algo, s);
+    for (int k = 0; k < K && rc == SYMAR_OK; ++k)
+        rc = run(h, h->seg0 + (size_t)(k % pairs) * slice, h->seg0 + (size_t)(pairs + k % pairs) * slice, count, dtype, algo, s);
     cudaError_t ce = cudaStreamEndCapture(s, &graph);
     if (rc != SYMAR_OK) {
         if (ce == cudaSuccess) cudaGraphDestroy(graph);
@@ -560,6 +570,8 @@ static int tune_bucket(symheap *h, int dtype, int b, size_t bytes, cudaStream_t 
                         bulk_variant(4, 0), 4};
         else if (algo == SYMAR_ONESHOT && bytes <= (1u << 20))
             variants = {0, 0x100, 0x200};            // 16, 8 or 4 bytes per thread
+        else if (algo == SYMAR_TWOSHOT && nvec < kCyclicMinVec)
+            variants = {0, 0x40};                    // 16 or 8 bytes per thread and trip
         else if (algo == SYMAR_LL && bytes <= kLLSmallMaxBytes) {
             // 8 bytes of payload per thread with the first poll held back by the default for this
             // traffic, by a quarter of a hop less and more, and not at all; 16 bytes per thread
@@ -573,7 +585,7 @@ static int tune_bucket(symheap *h, int dtype, int b, size_t bytes, cudaStream_t 
         } else if (algo == SYMAR_LL && bytes <= (256u << 10))
             variants = {0, 0x100};                   // general kernel: 16 or 8 bytes of payload per thread
         struct Cand { double us; LaunchCfg cfg; };
-        std::vector<Cand> cands;                     // bandwidth regime: the first pass's shapes, for a second look
+        std::vector<Cand> cands;                     // the first pass's shapes, for a second look
         // the neighbourhood of this algorithm's winner one step down
         // (above 4 MiB only, where every call is long and one kernel form covers all sizes: below, calls
         // are short, and the best shape still moves with the unit width and, at 1 MiB, with the change
@@ -582,7 +594,7 @@ static int tune_bucket(symheap *h, int dtype, int b, size_t bytes, cudaStream_t 
             (prune && bytes > (4u << 20) && tn.cfg[algo][prev].ctas > 0) ? tn.cfg[algo][prev] : LaunchCfg{};
         for (int var : variants) {
             // threads a shape needs: one per unit of this variant
-            const uint64_t units = bulk ? work : work << ((var >> 8) & 3);
+            const uint64_t units = bulk ? work : (work << ((var >> 8) & 3)) << ((algo == SYMAR_TWOSHOT && (var & 0x40)) ? 1 : 0);
             for (int T : kThreads) {
                 if (bulk && var != 4 && T != 128 && T != 256) continue;
                 for (int C : kCtas) {
@@ -603,7 +615,7 @@ static int tune_bucket(symheap *h, int dtype, int b, size_t bytes, cudaStream_t 
                     rc = time_calls(h, s, count, dtype, algo, K, reps, &us,
                                     h->tune_exhaustive || tn.us[algo][b] > 1e29 ? 0.0 : 1.25 * tn.us[algo][b]);
                     if (rc != SYMAR_OK) break;
-                    if (bulk) cands.push_back(Cand{us, LaunchCfg{C, T, var}});
+                    cands.push_back(Cand{us, LaunchCfg{C, T, var}});
                     // a larger launch must win by more than the timing noise (1.5 %) to displace a smaller one
                     const LaunchCfg &cur = tn.cfg[algo][b];
                     const bool larger    = cur.ctas > 0 && (long)C * T > (long)cur.ctas * cur.threads;
@@ -636,6 +648,27 @@ static int tune_bucket(symheap *h, int dtype, int b, size_t bytes, cudaStream_t 
                 }
             }
         }
+        // Latency regime: shapes of an algorithm that could win this size differ by a timer step or two
+        // (0.03 us per call in a 24-call graph).  Time its three fastest again in a graph twice as long
+        // and keep the winner, so that the choice does not hang on one noisy replay.
+        if (!bulk && rc == SYMAR_OK && cands.size() > 1 && tn.us[algo][b] <= 1.2 * best_us) {
+            std::sort(cands.begin(), cands.end(), [](const Cand &x, const Cand &y) { return x.us < y.us; });
+            cands.resize(std::min<size_t>(cands.size(), 3));
+            double best = 1e30;
+            for (const Cand &cd : cands) {
+                h->forced[algo]         = cd.cfg;
+                h->variant[algo]        = (unsigned)cd.cfg.variant;
+                h->variant_forced[algo] = true;
+                double us = 0;
+                rc = time_calls(h, s, count, dtype, algo, 2 * K, 9, &us);
+                if (rc != SYMAR_OK) break;
+                if (us < best) {
+                    best            = us;
+                    tn.us[algo][b]  = us;
+                    tn.cfg[algo][b] = cd.cfg;
+                }
+            }
+        }
         h->forced[algo]         = saved[algo];
         h->variant[algo]        = saved_variant[algo];
         h->variant_forced[algo] = saved_forced[algo];
@@ -653,10 +686,11 @@ static int tune_bucket(symheap *h, int dtype, int b, size_t bytes, cudaStream_t 
 }
 
 // only_bytes == 0: the whole power-of-two grid; else just the bucket of that size, at that size
-static int autotune(symheap *h, int dtype, size_t only_bytes)
+static int autotune(symheap *h, int dtype, size_t only_bytes, int rotate = 0)
 {
     const size_t es = elem_size(dtype);
-    const size_t fit = h->bytes_per_rank / 2 / kAlign * kAlign;      // input and output side by side
+    // input and output side by side; with `rotate` pairs of buffers, that many of each
+    const size_t fit = h->bytes_per_rank / 2 / (size_t)(rotate > 0 ? rotate : 1) / kAlign * kAlign;
     if (fit < 16) return SYMAR_ERR_INVAL;
     cudaStream_t s;
     CU(cudaStreamCreateWithFlags(&s, cudaStreamNonBlocking));
@@ -673,7 +707,9 @@ static int autotune(symheap *h, int dtype, size_t only_bytes)
         tn.have[b]    = false;
         h->tuned[dtype].valid = false;                 // time with defaults, not with a stale table
         std::memset(h->tuned[dtype].have, 0, sizeof h->tuned[dtype].have);
+        h->tune_rotate = rotate;
         rc = tune_bucket(h, dtype, b, bytes, s, tn);
+        h->tune_rotate = 0;
         tn.have[b] = rc == SYMAR_OK;
         cudaStreamSynchronize(s);
         cudaStreamDestroy(s);
@@ -1020,6 +1056,15 @@ int allreduce_autotune_size(symheap_t *heap, symar_dtype_t dtype, size_t count)
     if (!heap || (dtype != SYMAR_F32 && dtype != SYMAR_BF16) || count == 0) return SYMAR_ERR_INVAL;
     if (count > heap->bytes_per_rank / elem_size((int)dtype)) return SYMAR_ERR_INVAL;
     return autotune(heap, (int)dtype, count * elem_size((int)dtype));
+}
+
+int allreduce_autotune_stream(symheap_t *heap, symar_dtype_t dtype, size_t count, int calls)
+{
+    if (!heap || (dtype != SYMAR_F32 && dtype != SYMAR_BF16) || count == 0 || calls < 2 || calls > 1024) return SYMAR_ERR_INVAL;
+    const size_t es = elem_size((int)dtype);
+    if (count > heap->bytes_per_rank / es) return SYMAR_ERR_INVAL;
+    if (round_up(count * es, kAlign) * 2 * (size_t)calls > heap->bytes_per_rank) return SYMAR_ERR_INVAL;   // the pairs must fit
+    return autotune(heap, (int)dtype, count * es, calls);
 }
 
 int symar_last_choice(const symheap_t *heap, symar_algo_t *algo, int *ctas_per_rank, int *threads)

@@ -194,7 +194,24 @@ __global__ void __launch_bounds__(kMaxThreads) twoshot_kernel(const KArgs a)
             const uint64_t chv = (a.nvec + P - 1) / P;
             const uint64_t lo  = (uint64_t)r * chv;
             const uint64_t hi  = (lo + chv < a.nvec) ? lo + chv : a.nvec;
-            for (uint64_t v = lo + (uint64_t)c * T + t; v < hi; v += step) twoshot_vector<E, P>(a, v);
+            if (a.variant & 0x40u) {
+                // 8 bytes per thread and trip instead of 16: twice the threads share a chunk, each with half
+                // the unpack-add-store chain (what made the one-shot kernel faster below 128 KiB)
+                const uint64_t bytes = a.tail_bytes ? (a.nvec - 1) * 16 + a.tail_bytes : a.nvec * 16;
+                for (uint64_t u = 2 * lo + (uint64_t)c * T + t; u < 2 * hi; u += step) {
+                    if (u * 8 >= bytes) break;
+                    Words<2> x[P];
+#pragma unroll
+                    for (int q = 0; q < P; ++q) x[q] = ld_peer_words<2>(a.seg0 + (size_t)q * a.stride + a.in_off + u * 8);
+                    const Words<2> res  = reduce_words_in_rank_order<E, P, 2>(x);
+                    const uint64_t left = bytes - u * 8;
+#pragma unroll
+                    for (int q = 0; q < P; ++q)
+                        store_words<2>(a.seg0 + (size_t)q * a.stride + a.out_off + u * 8, res, left < 8u ? (uint32_t)left : 8u);
+                }
+            } else {
+                for (uint64_t v = lo + (uint64_t)c * T + t; v < hi; v += step) twoshot_vector<E, P>(a, v);
+            }
         } else {
             // large messages: blocks of 2^blk_log2 vectors are dealt to the ranks
             // round-robin, so that at any moment all P * C CTAs stream through the

@@ -71,7 +71,7 @@ __host__ __device__ constexpr size_t counters_off(int c, uint32_t k) { return (s
 //   LL       : bit 8    = 8 instead of 16 payload bytes per thread; bit 9 = never the single-iteration
 //              kernel; bits 12-15 = cycles / 64 the single-iteration kernel holds back its first poll
 //   two-shot : bit 0 = contiguous chunks for large messages, bit 1 = 16-byte accesses,
-//              bit 2 = never the bulk-copy kernel, bits 8-10 = bulk pipeline depth,
+//              bit 2 = never the bulk-copy kernel, bit 6 = 8-byte units below 1 MiB, bits 8-10 = bulk pipeline depth,
 //              bits 12-13 = log2(bulk tile size / 4 KiB)
 //   atomic two-shot: bit 0 = skip the confirming re-read of a completed line
 //   sibling collectives: the unit size in bytes (16, 4 or 2)

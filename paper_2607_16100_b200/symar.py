@@ -50,6 +50,7 @@ SIGNATURES = [
     ("symar_reduce", c_int, [c_void_p, c_void_p, c_void_p, c_size_t, c_int, c_int, c_void_p]),
     ("allreduce_autotune", c_int, [c_void_p, c_int]),
     ("allreduce_autotune_size", c_int, [c_void_p, c_int, c_size_t]),
+    ("allreduce_autotune_stream", c_int, [c_void_p, c_int, c_size_t, c_int]),
     ("symar_last_choice", c_int, [c_void_p, POINTER(c_int), POINTER(c_int), POINTER(c_int)]),
     ("symar_last_kernel", c_int, [c_void_p, POINTER(c_uint), POINTER(c_size_t)]),
     ("symar_query_choice", c_int, [c_void_p, c_size_t, c_int, POINTER(c_int), POINTER(c_int), POINTER(c_int)]),
@@ -268,6 +269,9 @@ class SymHeap:
 
     def autotune_size(self, dtype: int, count: int) -> None:
         _ck(self._lib.allreduce_autotune_size(self._h, dtype, count), "allreduce_autotune_size")
+
+    def autotune_stream(self, dtype: int, count: int, calls: int) -> None:
+        _ck(self._lib.allreduce_autotune_stream(self._h, dtype, count, calls), "allreduce_autotune_stream")
 
     def last_choice(self):
         a, c, t = c_int(), c_int(), c_int()

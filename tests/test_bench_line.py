@@ -47,7 +47,7 @@ def canned_latency_record():
            "sol_us": 1.42, "ratio_to_sol": 1.23456789, "ratio_to_sol_fastest_pair": 1.7}
     dec = {"autotune_seconds": 4.5, "step_total_us_p50": 346.64, "per_call_us": {"p10": 2.1, "p50": 2.16650003567338,
                                                                                  "p90": 2.2},
-           "sol_per_call_us": 1.9573064848973445, "ratio_to_sol": 1.1068782801212693, "algo": "twoshot_sentinel",
+           "sol_per_call_us": 1.9573064848973445, "ratio_to_sol": 1.1068782801212693, "ratio_to_sol_fastest_pair": 1.6123456789, "algo": "twoshot_sentinel",
            "ctas_per_rank": 64, "threads": 128, "repeats": [dict(rep)] * 5, "ratio_to_sol_over_repeats": dict(spread),
            "bit_exact": True, "calls": 160, "bytes_per_rank": 65536, "cache_state": "c" * 200}
     return {

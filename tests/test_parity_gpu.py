@@ -211,7 +211,9 @@ FORCE_PLAIN = 1 << 31
                                           (symar.LL, FORCE_PLAIN), (symar.LL, 0x100), (symar.LL, 0x3100),
                                           (symar.LL, 0xC000), (symar.LL, 0x200), (symar.LL, 0x300),
                                           (symar.SENTINEL, FORCE_PLAIN), (symar.TWOSHOT_LL, FORCE_PLAIN),
-                                          (symar.TWOSHOT_SENTINEL, FORCE_PLAIN)])
+                                          (symar.TWOSHOT_SENTINEL, FORCE_PLAIN),
+                                          # two-shot: 16 or 8 bytes per thread and trip
+                                          (symar.TWOSHOT, FORCE_PLAIN), (symar.TWOSHOT, 0x40)])
 def test_unit_width_variants(heaps, algo, variant, P, dtype, dist, count):
     # every implementation variant of a kernel gives the same bits, whatever the ragged tail
     h = heaps[P]
@@ -471,6 +473,30 @@ def test_autotune_of_one_size_fills_only_its_bucket(tmp_path):
         torch.cuda.synchronize()
         h.destroy()
         g.destroy()
+
+
+def test_autotune_for_a_stream_of_calls_with_their_own_buffers():
+    # the tuner's streaming mode: every timed call on its own input / output pair, as in a decode step
+    h = symar.SymHeap.on_torch(4, 4 << 20)
+    try:
+        count = 8192                                             # 16 KiB of bf16: bucket 14
+        before = h.query_choice(300, symar.BF16)
+        h.autotune_stream(symar.BF16, count, 24)                 # 24 pairs of 16 KiB = 768 KiB of the 4 MiB region
+        assert h.tuned_entry(symar.BF16, 14, symar.ONESHOT) is not None
+        assert h.tuned_entry(symar.BF16, 13, symar.ONESHOT) is None
+        assert h.query_choice(300, symar.BF16) == before
+        a, c, t = h.query_choice(count, symar.BF16)
+        assert a in ALGOS and (c, t) == h.tuned_entry(symar.BF16, 14, a)[:2]
+        x = synth.make_inputs("normal", "bf16", 4, count, seed=21)
+        assert_bits(run(h, x, symar.BF16, symar.AUTO), O.allreduce(x))
+        assert h.last_choice() == (a, c, t)
+        with pytest.raises(symar.SymarError):
+            h.autotune_stream(symar.BF16, count, 200)            # 200 pairs do not fit
+        with pytest.raises(symar.SymarError):
+            h.autotune_stream(symar.BF16, count, 1)
+    finally:
+        torch.cuda.synchronize()
+        h.destroy()
 
 
 def test_tuned_table_round_trips_through_a_file(tmp_path):
