@@ -457,6 +457,10 @@ __global__ void __launch_bounds__(kLLMaxThreads) ll_kernel(const KArgs a)
 // row in flight instead (a second one issued half a round trip after the first) was measured
 // slower at every size (+0.4 us).
 //
+// (Measured and dropped: writing every row twice, 4 KiB apart, so that the receiver can poll a copy on its
+// own half of the L2 -- what pays for flags and counters.  The second set of stores costs more than the
+// nearer poll gains: +0.06 to +0.5 us from 16 B to 2 KiB at P = 2, 4 and 8.)
+//
 // Dependent launch.  The kernel never triggers its dependent early: the next call then starts when
 // this grid has drained, overlapping only its launch with this grid's completion.  Measured against
 // a trigger before the stores, after them or after the polls: 1.56 instead of 1.81 us at 128 B,
