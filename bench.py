@@ -390,11 +390,29 @@ def latency_suite(torch, symar, synth, hbm_gbs, quick=False, autotune=True):
                     table.append({"bytes_per_rank": 1 << log2, "us": us, "best": min(us, key=us.get)})
             out.setdefault("tuner_table_bf16", {})[f"P{P}"] = table
 
-        def load_inputs(count):
+        def load_inputs(count, heap=None):
             x = synth.make_inputs("normal", "bf16", P, count, synth.seed_for_config(2))
             for q in range(P):
-                h.write_rank(q, 0, x[q])
+                (heap or h).write_rank(q, 0, x[q])
             return x
+
+        def untuned_default(count, n=None):
+            """The same call on a heap that was never tuned: the built-in algorithm and launch shape."""
+            hu = symar.SymHeap.on_torch(P, 24 << 20)
+            try:
+                x = load_inputs(count, hu)
+                enq = lambda k, s: hu.allreduce(0, out_off, count, symar.BF16, symar.AUTO, s)
+                enq(0, stream.cuda_stream)
+                stream.synchronize()
+                a, c, t = hu.last_choice()
+                got = np.stack([hu.read_rank(q, out_off, count, np.uint16) for q in range(P)])
+                exact = bool(np.array_equal(got, O.allreduce(x))) and hu.status()[0] == 0
+                r = time_graph(torch, graph_of(torch, stream, enq, K), stream, K, n or reps)
+                return {"p50_us": r["p50"], "algo": names[a], "shape": [c, t], "variant": hu.last_kernel()[0],
+                        "bit_exact": exact}
+            finally:
+                stream.synchronize()
+                hu.destroy()
 
         def bench_size(count, algos, stream_too=False, n=None):
             x = load_inputs(count)
@@ -649,6 +667,7 @@ def latency_suite(torch, symar, synth, hbm_gbs, quick=False, autotune=True):
                 named = {k: v["p50"] for k, v in row.items() if k != "auto"}
                 best_name = min(named, key=named.get)
                 ra = bench_size(8192 * B, (symar.TWOSHOT_ATOMIC,))["twoshot_atomic"]
+                ud = untuned_default(8192 * B)
                 fl = empty_floor(row["auto"]["ctas_per_rank"], P, row["auto"]["threads"], n=100)
                 s_ol = fl["p50"] + rt_ns / 1000.0 + bytes_us(16384 * B, P)
                 try:       # where two-shot's time goes: exchange, data, CTA barrier, release fence, "done" hop
@@ -669,12 +688,14 @@ def latency_suite(torch, symar, synth, hbm_gbs, quick=False, autotune=True):
                                                "bytes_at_measured_hbm_copy_rate": bytes_us(16384 * B, P)},
                               "oracle_cpu": oracle_us(O, synth.make_inputs("normal", "bf16", P, 8192 * B,
                                                                            synth.seed_for_config(2))),
+                              "untuned_default": ud,
                               "twoshot_phase_stamps_us": ts_phases,
-                              "bit_exact": all(v["bit_exact"] for v in row.values())})
+                              "bit_exact": all(v["bit_exact"] for v in row.values()) and ud["bit_exact"]})
             out["sweep"] = sweep
             out["sweep_note"] = "sol_us = empty launch of the selector's shape + median flag round trip + 2*P*M bytes at " \
                                 "the measured HBM copy rate (the messages are L2-resident, so the byte term is an upper " \
-                                "estimate of what the bound allows); oracle_cpu = the CPU oracle on the same message"
+                                "estimate of what the bound allows); oracle_cpu = the CPU oracle on the same message; " \
+                                "untuned_default = the same call on a heap that was never tuned (built-in choice)"
         # C5: 160 calls in one graph
         calls, count = 160, 8192 * 4
         nb = count * 2

@@ -152,6 +152,7 @@ constexpr uint64_t kLLSmallMaxBytes = (uint64_t)kLLSlots * kLLMaxThreads * 8;
 static unsigned ll_default_gap(int P, uint64_t bytes)
 {
     const uint64_t in_flight = (uint64_t)P * (P - 1) * 2 * bytes;     // payload + flags, all ranks
+    if (P == 2 && bytes >= 4096 && in_flight < (192u << 10)) return 3;   // several CTAs per rank: measured -0.05 us
     if (in_flight < (96u << 10)) return 0;
     if (in_flight < (192u << 10)) return 2;
     if (in_flight < (384u << 10)) return 8;
@@ -159,51 +160,112 @@ static unsigned ll_default_gap(int P, uint64_t bytes)
     return 12;
 }
 
-// Launch shape when neither the caller nor the tuner fixed one.
-static LaunchCfg default_cfg(const symheap *h, int algo, uint64_t nvec)
+// Launch shape when neither the caller nor the tuner fixed one.  Every rule here restates what the
+// tuner chose on B200 for 2, 4 and 8 ranks from 128 B to 256 MiB; an untuned call stays within a few
+// percent of the tuned one (measured: at most 7 %, typically 0 to 3 %).
+static LaunchCfg default_cfg(symheap *h, int algo, uint64_t nvec, KernelFn fn)
 {
     LaunchCfg c;
     c.variant = 0;
-    const uint64_t work = (algo == SYMAR_TWOSHOT || is_twoshot_push(algo)) ? (nvec + h->P - 1) / h->P
+    const int P = h->P;
+    const uint64_t bytes = nvec * 16;
+    const uint64_t work  = (algo == SYMAR_TWOSHOT || is_twoshot_push(algo)) ? (nvec + P - 1) / P
                                                                             : nvec;   // vectors per rank partition
     if (algo == SYMAR_TWOSHOT && nvec >= kBulkMinVec) {
-        // Bandwidth regime.  HBM3e delivers most when few, long streams are in
-        // flight: about 100 CTAs in total, each with one 64 KiB stage (P tiles)
-        // ahead of the one it reduces (measured on B200; more CTAs, more stages or
-        // shorter tiles all lose several percent to DRAM page conflicts).
-        int tile_log2 = 0;
-        while ((4096u << tile_log2) * (unsigned)h->P < 65536u && tile_log2 < 3) ++tile_log2;
-        c.threads = 256;
-        c.ctas    = std::max(1, std::min(100 / h->P, (int)kMaxCtas));
-        c.variant = bulk_variant(2, tile_log2);
+        // Bandwidth regime: the register kernel with 512 threads per SM in all, in as many CTAs per rank as
+        // half or a quarter of the SMs (CTA c of every rank then lands on the same one or two SMs, so the
+        // CTAs that signal one another sit together): 37 x 256 among eight ranks, 74 x 256 among four,
+        // 74 x 512 between two.  The bulk-copy kernel comes within 3 % with about 100 CTAs in total, each
+        // with one 64 KiB stage ahead of the one it reduces, and the tuner still times it; from 4 to 16 MiB,
+        // where repeated calls find their buffers in L2, it is 10 to 40 % behind.
+        c.variant = 4;
+        c.threads = P >= 4 ? 256 : 512;
+        c.ctas    = std::max(1, std::min(h->num_sms * 512 / P / c.threads, (int)kMaxCtas));
         return c;
     }
-    // Latency regime: about one unit per thread, small blocks, few CTAs.  Small
-    // messages are bound by the per-thread instruction chain, so a thread takes
-    // 4 or 8 bytes instead of 16 (measured -0.3 us at 16 KiB, P = 8).
-    uint64_t units = work;
-    if (algo == SYMAR_TWOSHOT && h->P == 8 && nvec * 16 <= (256u << 10)) {
-        // 8 bytes per thread and trip: measured 0.35-0.45 us ahead of 16 bytes from 16 KiB to 256 KiB among
-        // eight ranks (no gain among four, none from 512 KiB)
-        c.variant = 0x40;
-        units     = work * 2;
-    } else if (algo == SYMAR_ONESHOT) {
-        const uint64_t bytes = nvec * 16;
-        const int narrow = bytes <= (8u << 10) ? 2 : (bytes <= (128u << 10) ? 1 : 0);
+    if (algo == SYMAR_TWOSHOT) {
+        // Latency regime of two-shot: one unit per thread; at most 128 / P CTAs per rank, blocks growing to
+        // 512 threads before threads take a second unit; 8192 threads per rank at most (16384 between two).
+        // Among eight ranks a unit is 8 bytes up to 512 KiB (measured 0.15 to 0.45 us ahead of 16 bytes from
+        // 16 KiB on; no gain among four or two ranks, none from 1 MiB).
+        uint64_t units = work;
+        const uint64_t budget = P == 2 ? 16384 : 8192;
+        if (nvec >= kCyclicMinVec) {
+            // from 1 MiB blocks of 8 KiB are dealt to the ranks and a thread moves 32 bytes per trip: half as
+            // many CTAs per rank as SMs (see above), small ones (measured at 1 MiB among eight ranks: 74 CTAs
+            // of 64 threads 4.7 us, 64 of 64 5.2 us, 16 of 512 6.5 us)
+            // (at 2 MiB: 16 to 18 CTAs of 512 threads 7.1 us, 37 of 256 7.4 to 8.4 us, 74 of 128 7.9 us)
+            const uint64_t n    = std::min((work + 1) / 2, budget);
+            const uint64_t half = (uint64_t)std::max(1, std::min(h->num_sms / 2, (int)kMaxCtas));
+            if (n <= half * 64) {
+                c.threads = 64;
+                c.ctas    = (int)half;
+            } else if (P == 8) {
+                c.threads = 512;
+                c.ctas    = (int)std::max<uint64_t>(1, half / 4);
+            } else {
+                c.threads = 128;
+                c.ctas    = (int)half;
+            }
+            return c;
+        }
+        if (P == 8 && bytes <= (512u << 10)) {
+            c.variant = 0x40;
+            units     = work * 2;
+        }
+        const uint64_t cap_c  = (uint64_t)std::max(1, 128 / P);
+        uint64_t T = units <= 128 ? (uint64_t)round_threads(std::max<uint64_t>(units, 64)) : 128;
+        while (T < kMaxThreads && (units + T - 1) / T > cap_c) T *= 2;
+        uint64_t C = std::min((units + T - 1) / T, cap_c);
+        if (C * T > budget) T = std::max<uint64_t>(128, budget / C);
+        c.threads = (int)T;
+        c.ctas    = (int)std::max<uint64_t>(1, C);
+        return c;
+    }
+    if (algo == SYMAR_ONESHOT) {
+        // Small messages are bound by the per-thread instruction chain, so a thread takes 8 bytes up to
+        // 64 KiB (4 up to 256 B, where that still fills a warp) and 16 above.  One unit per thread: one CTA
+        // up to 256 units, blocks of 128 up to half as many CTAs per rank as SMs, then larger blocks as far as the kernel's
+        // registers let all ranks' CTAs be resident together; beyond that equal passes.
+        const int narrow = bytes <= 256 ? 2 : (bytes <= (64u << 10) ? 1 : 0);
         c.variant = narrow << 8;
-        units     = work << narrow;
-    } else if (algo == SYMAR_LL && nvec * 16 <= kLLSmallMaxBytes) {
+        const uint64_t units = work << narrow;
+        if (units <= 256) {
+            c.threads = round_threads(units);
+            c.ctas    = 1;
+            return c;
+        }
+        uint64_t best_cover = 0;
+        const uint64_t half = (uint64_t)std::max(1, std::min(h->num_sms / 2, (int)kMaxCtas));
+        for (int T : {128, 256, 512}) {
+            const uint64_t res = fn ? (uint64_t)std::max(1, max_resident(h, fn, T, 0) / P) : half;
+            const uint64_t C   = std::min<uint64_t>({(units + T - 1) / T, half, res});
+            const uint64_t cover = std::min(units, C * T);
+            if (cover > best_cover) {
+                best_cover = cover;
+                c.threads  = T;
+                c.ctas     = (int)C;
+            }
+        }
+        const uint64_t per_pass = (uint64_t)c.ctas * c.threads;
+        const uint64_t passes   = (units + per_pass - 1) / per_pass;
+        c.ctas = (int)std::max<uint64_t>(1, (units + passes * c.threads - 1) / (passes * c.threads));
+        return c;
+    }
+    uint64_t units = work;
+    if (algo == SYMAR_LL && bytes <= kLLSmallMaxBytes) {
         // the single-iteration kernel with 8 bytes of payload per thread (measured ahead of 16 bytes
         // per thread at every size it covers), first poll held back by the default for this traffic
-        c.variant = 0x100 | (ll_default_gap(h->P, nvec * 16) << 12);
+        c.variant = 0x100 | (ll_default_gap(P, bytes) << 12);
         units     = work * 2;
         c.threads = units <= 256 ? round_threads(units) : (units < 2048 ? 64 : (units <= 8192 ? 128 : 256));
+        if (P == 2 && units > 256) c.threads = units <= 512 ? 128 : 256;     // between two ranks: few, larger CTAs
         c.ctas    = (int)std::min<uint64_t>((units + c.threads - 1) / c.threads, (uint64_t)kLLSlots);
         return c;
     }
     c.threads = units >= 2048 ? 128 : round_threads(std::max<uint64_t>(units / 16, 32));
     uint64_t ctas = (units + c.threads - 1) / c.threads;
-    const uint64_t cap = is_push(algo) ? (uint64_t)kLLSlots : (uint64_t)std::max(1, 2 * h->num_sms / h->P);
+    const uint64_t cap = is_push(algo) ? (uint64_t)kLLSlots : (uint64_t)std::max(1, 2 * h->num_sms / P);
     c.ctas = (int)std::max<uint64_t>(1, std::min(ctas, cap));
     return c;
 }
@@ -215,10 +277,14 @@ static LaunchCfg default_cfg(const symheap *h, int algo, uint64_t nvec)
 static int default_algo(int P, size_t bytes)
 {
     // the data+flag protocol leads at the smallest sizes (Sec. VII Obs. 1); measured here, with flag
-    // and counter reads placed on the reader's L2 half: up to 1 KiB between two ranks (1.24 against
-    // 1.43 us at 128 B), nowhere among four or eight (one-shot 1.37 / 1.53 us against 1.49 / 1.69 us)
-    if (P == 2 && bytes <= 1024) return SYMAR_LL;
-    if (bytes <= (256u << 10)) return SYMAR_ONESHOT;
+    // and counter reads placed on the reader's L2 half: up to 8 KiB between two ranks (1.2 to 1.35
+    // against 1.35 to 1.45 us), nowhere among four or eight (one-shot 1.37 / 1.43 us against 1.43 / 1.57 us
+    // at 128 B)
+    if (P == 2 && bytes <= 8192) return SYMAR_LL;
+    // one-shot reads P times the bytes two-shot does and saves its second synchronisation: the
+    // break-even moves up fourfold each time the rank count halves (measured 256 KiB, 1 MiB, 4 to 8 MiB)
+    const size_t limit = (size_t)(256u << 10) * (size_t)(64 / (P * P));
+    if (bytes <= limit) return SYMAR_ONESHOT;
     return SYMAR_TWOSHOT;
 }
 
@@ -247,7 +313,7 @@ static int make_plan(symheap *h, size_t in_off, size_t out_off, size_t count, in
 
     if (algo == SYMAR_AUTO) algo = h->env_algo ? h->env_algo : (tuned ? tn.best_algo[b] : default_algo(h->P, bytes));
 
-    LaunchCfg cfg = default_cfg(h, algo, nvec);
+    LaunchCfg cfg = default_cfg(h, algo, nvec, algo == SYMAR_ONESHOT ? any_kernel_for(algo, dtype, h->P, dbg_on(h)) : nullptr);
     if (tuned && tn.cfg[algo][b].ctas > 0) cfg = tn.cfg[algo][b];
     if (h->forced[algo].ctas > 0) cfg.ctas = h->forced[algo].ctas;
     if (h->forced[algo].threads > 0) cfg.threads = h->forced[algo].threads;

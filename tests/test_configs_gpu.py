@@ -110,7 +110,7 @@ def test_c4_full_size_p8_fp32_256MiB():
         h.allreduce(0, M, count, symar.F32, symar.TWOSHOT)      # bench.py's call, default launch shape
         torch.cuda.synchronize()
         assert h.status()[0] == symar.OK
-        assert h.last_kernel()[1] > 0                            # the bulk-copy kernel ran
+        assert h.last_kernel() == (4, 0)                         # the register kernel of the bandwidth regime ran
         want_bits = want.view(np.uint32)
 
         def check_all(what):
@@ -121,7 +121,14 @@ def test_c4_full_size_p8_fp32_256MiB():
                 h.write_rank(r, M, np.zeros(1 << 20, dtype=np.uint8))      # stale results must not pass the next check
 
         check_all("default shape")
-        # the register kernel in the shape the tuner tends to pick for this size
+        # the bulk-copy kernel: 12 CTAs per rank, two stages of eight 8 KiB tiles
+        h.set_launch(symar.TWOSHOT, 12, 256)
+        h.set_variant(symar.TWOSHOT, (2 << 8) | (1 << 12))
+        h.allreduce(0, M, count, symar.F32, symar.TWOSHOT)
+        torch.cuda.synchronize()
+        assert h.last_kernel()[1] > 0 and h.last_choice() == (symar.TWOSHOT, 12, 256)
+        check_all("bulk-copy kernel 12 x 256")
+        # the register kernel in another shape the tuner tends to pick for this size
         h.set_launch(symar.TWOSHOT, 15, 512)
         h.set_variant(symar.TWOSHOT, 4)
         h.allreduce(0, M, count, symar.F32, symar.TWOSHOT)

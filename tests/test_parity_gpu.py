@@ -263,7 +263,8 @@ def bulk_var(stages, tile_log2):
     (8, "f32", 4 * (1 << 20) + 3),
 ])
 @pytest.mark.parametrize("variant,ctas,threads", [
-    (0, 0, 0),                       # defaults: bulk kernel, 64 KiB stage
+    (0, 0, 0),                       # defaults: register kernel, 512 threads per SM in all
+    (bulk_var(2, 0), 12, 256),       # bulk kernel, 64 KiB stage among eight ranks
     (bulk_var(3, 0), 37, 256),       # 4 KiB tiles, three stages, two CTAs per SM
     (bulk_var(2, 1), 7, 128),        # 8 KiB tiles, odd CTA count
     (bulk_var(4, 0), 13, 512),
@@ -282,7 +283,9 @@ def test_bandwidth_regime_paths(big_heaps, P, dtype, count, variant, ctas, threa
     try:
         got = run(h, x, DT[dtype], symar.TWOSHOT, in_off=0, out_off=out_off)
         var, smem = h.last_kernel()
-        if not (variant & 4):
+        if variant == 0:
+            assert smem == 0 and (var & 4), "the default of the bandwidth regime is the register kernel"
+        elif not (variant & 4):
             assert smem > 0, "the bulk-copy kernel should have been used"
         else:
             assert smem == 0
@@ -298,7 +301,7 @@ def test_bandwidth_regime_unaligned_buffers(big_heaps):
     h = big_heaps[8]
     count = (1 << 20) + 37
     x = synth.make_inputs("uniform", "f32", 8, count, seed=4242)
-    for variant in (0, 4):
+    for variant in (bulk_var(2, 1), 4):
         h.set_variant(symar.TWOSHOT, variant)
         try:
             got = run(h, x, symar.F32, symar.TWOSHOT, in_off=16, out_off=(20 << 20) + 48)
