@@ -13,7 +13,7 @@ process) and the 160-call decode-step graph ride in the same line as a handful o
 
 Everything else -- per-algorithm rows, the 16 KiB..1 MiB sweep with the selector's choice, the
 sampled flag round trips, phase stamps, the tuner's table, the context measurements -- goes to one
-file per workload in DIR (default gpurun_out/): results_c2.json, results_c3.json, results_c4.json,
+file per workload in the directory given by --out-dir: results_c2.json, results_c3.json, results_c4.json,
 results_c5.json.  The line names them under `details`.
 
 N > 1 runs N independent replicas (one process and one heap per GPU; the path itself is a

@@ -226,7 +226,10 @@ int symar_reduce(symheap_t *heap, const void *in, void *out, size_t count,
  * winner and lost by more than 1.5 x one size down is not timed again, and shapes
  * are searched around the previous size's winner (SYMAR_TUNE = exhaustive in the
  * environment searches everything).  Synchronous; takes seconds.  OVERWRITES the
- * user region of every rank.  Before it is called, built-in defaults apply.     */
+ * user region of every rank.  Before it is called, built-in defaults apply: the
+ * data+flag protocol up to 8 KiB between two ranks, else one-shot up to
+ * 256 KiB x (8 / P)^2 per rank, else two-shot, each in a launch shape that restates
+ * what this tuner chose on B200 (within a few percent of a tuned call).          */
 int allreduce_autotune(symheap_t *heap, symar_dtype_t dtype);
 
 /* The same for ONE message size: times every algorithm, shape and variant on messages
@@ -287,7 +290,8 @@ int symar_set_launch(symheap_t *heap, symar_algo_t algo, int ctas_per_rank, int 
  * single-iteration kernel holds back its first poll;
  * two-shot: bit 0 = contiguous chunks also for large messages (no block-cyclic
  * ownership), bit 1 = 16-byte instead of 32-byte accesses for large messages,
- * bit 2 = never use the bulk-copy kernel, bit 6 = 8 instead of 16 bytes per thread and
+ * bit 2 = the register kernel instead of the bulk-copy kernel from 4 MiB (the built-in
+ * choice there), bit 6 = 8 instead of 16 bytes per thread and
  * trip for messages below 1 MiB, bits 8-10 = the bulk kernel's pipeline depth (0:
  * default), bits 12-13 = log2 of its tile size over 4 KiB.                        */
 int symar_set_variant(symheap_t *heap, symar_algo_t algo, unsigned int variant);
