@@ -812,7 +812,7 @@ def compact_line(bw, lat, details):
                   "vs_baseline", "dtype", "data", "impl"):
             line[k] = _r(bw.get(k))
         cfg = bw.get("config", {})
-        line["config"] = {"workload": "c4: P=8 emulated ranks, fp32, %s el/rank, U(-1,1), two-shot; value=2PM bytes/time; "
+        line["config"] = {"workload": "c4: P=8 emulated ranks, fp32, %s el/rank, U(-1,1), two-shot; value=2PM B/time; "
                                       "4 GiB per step >> L2" % cfg.get("elements_per_rank"),
                           "kernel": cfg.get("kernel"),
                           "ctas_per_rank": cfg.get("ctas_per_rank"), "threads": cfg.get("threads"),
@@ -827,6 +827,7 @@ def compact_line(bw, lat, details):
                             "unit": rf.get("unit"), "frac": _r(rf.get("frac")), "peak_source": "measured"
                             if str(rf.get("peak_source", "")).startswith("measured") else "fallback",
                             "frac_nominal_8TBs": _r(rf.get("frac_of_nominal_8TBps")),
+                            "live_copy": _r(rf.get("live_copy_gbs"), 0),
                             "algorithmic_bytes": rf.get("algorithmic_bytes_per_launch"),
                             "launch_ms": _r((rf.get("launch_ms") or {}).get("mean")), "traffic": rf.get("traffic")}
         if bw.get("cpu_baseline"):
@@ -1092,6 +1093,26 @@ def main():
             "traffic": None,
         },
     }
+    # context for the fraction: a plain device-to-device copy of as many bytes, timed in this process on this
+    # GPU (the denominator above is the pool-wide measured copy rate; this says what this box's copy does now)
+    try:
+        src = torch.empty(algbytes // 2, dtype=torch.uint8, device="cuda")
+        dst = torch.empty_like(src)
+        src.fill_(1)
+        with torch.cuda.stream(stream):
+            for _ in range(2):
+                dst.copy_(src)
+            ca, cb_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            ca.record(stream)
+            for _ in range(5):
+                dst.copy_(src)
+            cb_.record(stream)
+        stream.synchronize()
+        line["roofline"]["live_copy_gbs"] = 5 * algbytes / (ca.elapsed_time(cb_) * 1e-3) / 1e9
+        del src, dst
+    except RuntimeError as exc:
+        line["roofline"]["live_copy_gbs"] = None
+        line["roofline"]["live_copy_error"] = str(exc)[:200]
     traffic_note = ROOT / "profiles" / ("twoshot_bulk_f32_p8_traffic.txt" if smem else "twoshot_f32_p8_traffic.txt")
     if traffic_note.exists() and count == synth.WORKLOADS["c4"]["count"]:
         kv = dict(l.split("=", 1) for l in traffic_note.read_text().splitlines() if "=" in l and not l.startswith("#"))

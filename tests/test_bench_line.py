@@ -30,7 +30,7 @@ def canned_bandwidth_record():
                      "peak_source": "measured (MEASURED_PEAKS.json hbm_gbs)", "kernel": "twoshot_bulk_kernel<F32, 8>",
                      "algorithmic_bytes_per_launch": 4294967296,
                      "launch_ms": {"mean": 0.65365123456, "min": 0.6501234567, "max": 0.6601234567},
-                     "frac_of_nominal_8TBps": 0.82134567891, "traffic": 3893700198, "traffic_source": "z" * 200},
+                     "frac_of_nominal_8TBps": 0.82134567891, "live_copy_gbs": 6543.21987654321, "traffic": 3893700198, "traffic_source": "z" * 200},
         "cpu_baseline": {"value": 59.512345678, "unit": "GB/s", "cores": 16, "kind": "oracle", "sample": "s" * 300},
         "e2e": {"value": 90.912345678, "unit": "GB/s", "h2d_bytes_per_step": 2147483648, "d2h_bytes_per_step": 2147483648,
                 "steps": 5, "ms_per_step": 47.2123456789, "bit_exact_sampled": True, "note": "n" * 300},
