@@ -310,6 +310,26 @@ def test_bandwidth_regime_unaligned_buffers(big_heaps):
         assert_bits(got, O.allreduce(x), f"variant {variant}")
 
 
+# sizes at which the built-in algorithm, the unit width or the rule for the launch shape changes
+BOUNDARY_BYTES = [256, 272, 2048, 2064, 8192, 8208, 65536, 65552, 262144, 262160, 524288, 524304, (1 << 20) - 16,
+                  1 << 20, (1 << 20) + 48, (2 << 20) + 4112, (4 << 20) - 16, 4 << 20, (4 << 20) + 16]
+
+
+@pytest.mark.parametrize("nbytes", BOUNDARY_BYTES)
+@pytest.mark.parametrize("P", [2, 4, 8])
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_builtin_choices_at_their_boundaries(big_heaps, P, dtype, nbytes):
+    """No tuning, no forced shape: what a first call gets, on both sides of every threshold."""
+    h = big_heaps[P]
+    es = 4 if dtype == "f32" else 2
+    for count in (nbytes // es, nbytes // es - 1):
+        x = synth.make_inputs("uniform" if dtype == "f32" else "normal", dtype, P, count, seed=nbytes + P)
+        want = O.allreduce(x)
+        for algo in (symar.AUTO, symar.ONESHOT, symar.TWOSHOT):
+            got = run(h, x, DT[dtype], algo, in_off=0, out_off=20 << 20)
+            assert_bits(got, want, f"P={P} {dtype} count={count} algo={algo} launched {h.last_choice()}")
+
+
 # ---- determinism, algorithm equality, interleaving stress ---------------------------
 
 def test_algorithms_agree_and_repeat(heaps):
