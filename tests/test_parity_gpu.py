@@ -677,26 +677,33 @@ def test_host_buffer_entry_point(heaps):
     assert_bits(hout.numpy(), O.allreduce(x))
 
 
-def test_host_buffer_entry_point_pipelines_large_messages():
-    # 80 MiB per rank: cut into 16 MiB chunks (the last one ragged) that overlap transfers and kernels
-    P, count = 2, 20 * (1 << 20) + 12345
-    M = count * 4
+@pytest.mark.parametrize("dtype,count", [
+    ("f32", 20 * (1 << 20) + 12345),      # 80 MiB per rank: 16 MiB chunks, the last one ragged
+    ("f32", 25 * (1 << 20) + 12345),      # 100 MiB: seven chunks, 4 bytes past a 16-byte boundary
+    ("bf16", 52 * (1 << 20) + 7),         # 104 MiB: an odd count of 2-byte elements
+])
+def test_host_buffer_entry_point_pipelines_large_messages(dtype, count):
+    # cut into chunks that overlap transfers and kernels
+    P = 2
+    es = 4 if dtype == "f32" else 2
+    M = count * es
     out_off = (M + 4095) // 4096 * 4096
     h = symar.SymHeap.on_torch(P, out_off + M)
     try:
-        x = synth.make_inputs("uniform", "f32", P, count, seed=17)
+        x = synth.make_inputs("uniform" if dtype == "f32" else "normal", dtype, P, count, seed=17)
+        want = O.allreduce(x)
         hin = torch.from_numpy(x).pin_memory()
         hout = torch.empty_like(hin).pin_memory()
         s = torch.cuda.Stream()
         for rep in range(2):                                     # twice: the second call reuses the pipeline's events
             hout.zero_()
-            h.allreduce_host(hin.data_ptr(), hout.data_ptr(), 0, out_off, count, symar.F32, symar.AUTO, s.cuda_stream)
+            h.allreduce_host(hin.data_ptr(), hout.data_ptr(), 0, out_off, count, DT[dtype], symar.AUTO, s.cuda_stream)
             s.synchronize()
             assert h.status()[0] == symar.OK
-            assert_bits(hout.numpy(), O.allreduce(x), f"rep {rep}")
+            assert_bits(hout.numpy(), want, f"rep {rep}")
         # the device copy of the result is complete as well
-        got = np.stack([h.read_rank(q, out_off, count, np.float32) for q in range(P)])
-        assert_bits(got, O.allreduce(x))
+        got = np.stack([h.read_rank(q, out_off, count, NP_DT[DT[dtype]]) for q in range(P)])
+        assert_bits(got, want)
     finally:
         torch.cuda.synchronize()
         h.destroy()
