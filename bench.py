@@ -293,22 +293,28 @@ def scope_probe(shapes_json, quick):
 
 
 def run_case(spec, steps, warmup):
-    """`--case ALGO:BYTES[:P[:VARIANT[:CTAS:THREADS]]]`: a few stream-launched calls of ONE algorithm on a
-    bf16 message of BYTES per rank, checked against the oracle -- a small, self-ending command for
+    """`--case ALGO:BYTES[:P[:VARIANT[:CTAS:THREADS]]]` (or `--case c1`): a few stream-launched calls of ONE
+    algorithm on a bf16 message of BYTES per rank, checked against the oracle -- a small, self-ending command for
     profilers (a few MiB on the device, `warmup` + `steps` launches)."""
     import torch
     from oracle import allreduce_oracle as O
     from paper_2607_16100_b200 import symar, synth
-    f = spec.split(":")
-    algo = {v: k for k, v in symar.ALGO_NAMES.items()}[f[0]]
-    nbytes = int(f[1])
-    P = int(f[2]) if len(f) > 2 else 8
-    variant = int(f[3], 0) if len(f) > 3 else 0
-    ctas, threads = (int(f[4]), int(f[5])) if len(f) > 5 else (0, 0)
-    count = nbytes // 2
+    if spec == "c1":          # the smallest workload as it is defined: P = 4, fp32, 1024 integer-valued elements, one-shot
+        w = synth.WORKLOADS["c1"]
+        algo, P, variant, ctas, threads = symar.ONESHOT, w["P"], 0, 0, 0
+        count, nbytes, dt, npdt = w["count"], w["count"] * 4, symar.F32, np.uint32
+        x = synth.make_inputs(w["dist"], "f32", P, count, w["seed"])
+    else:
+        f = spec.split(":")
+        algo = {v: k for k, v in symar.ALGO_NAMES.items()}[f[0]]
+        nbytes = int(f[1])
+        P = int(f[2]) if len(f) > 2 else 8
+        variant = int(f[3], 0) if len(f) > 3 else 0
+        ctas, threads = (int(f[4]), int(f[5])) if len(f) > 5 else (0, 0)
+        count, dt, npdt = nbytes // 2, symar.BF16, np.uint16
+        x = synth.make_inputs("normal", "bf16", P, count, synth.seed_for_config(2))
     out_off = (nbytes + 4095) // 4096 * 4096
     h = symar.SymHeap.on_torch(P, max(2 * out_off, 1 << 16))
-    x = synth.make_inputs("normal", "bf16", P, count, synth.seed_for_config(2))
     for q in range(P):
         h.write_rank(q, 0, x[q])
     if variant:
@@ -316,7 +322,7 @@ def run_case(spec, steps, warmup):
     if ctas or threads:
         h.set_launch(algo, ctas, threads)
     stream = torch.cuda.Stream()
-    call = lambda: h.allreduce(0, out_off, count, symar.BF16, algo, stream.cuda_stream)
+    call = lambda: h.allreduce(0, out_off, count, dt, algo, stream.cuda_stream)
     for _ in range(max(1, warmup)):
         call()
     stream.synchronize()
@@ -327,12 +333,12 @@ def run_case(spec, steps, warmup):
             call()
         b.record(stream)
     stream.synchronize()
-    got = np.stack([h.read_rank(q, out_off, count, np.uint16) for q in range(P)])
+    got = np.stack([h.read_rank(q, out_off, count, npdt) for q in range(P)])
     al, c, t = h.last_choice()
     print(json.dumps({"case": spec, "algo": symar.ALGO_NAMES[al], "ctas_per_rank": c, "threads": t,
                       "variant": h.last_kernel()[0], "launches": max(1, warmup) + steps,
                       "stream_launched_us_per_call": a.elapsed_time(b) * 1000.0 / steps,
-                      "bit_exact": bool(np.array_equal(got, O.allreduce(x))) and h.status()[0] == 0}))
+                      "bit_exact": bool(np.array_equal(got, O.allreduce(x).view(npdt))) and h.status()[0] == 0}))
     h.destroy()
 
 
