@@ -19,6 +19,8 @@ LIB_CHECK = PKG / "libsymar_check.so"
 
 EXAMPLE_SRC = PKG / "examples" / "llbuffer_oneshot.cu"
 EXAMPLE_LIB = PKG / "libsymar_example.so"
+C_EXAMPLE_SRC = PKG / "examples" / "allreduce_from_c.c"
+C_EXAMPLE_BIN = PKG / "allreduce_from_c.bin"
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a",
@@ -95,9 +97,26 @@ def build_example(force: bool = False) -> Path:
     return EXAMPLE_LIB
 
 
+def build_c_example(force: bool = False) -> Path:
+    """examples/allreduce_from_c.c: a plain C99 program on include/symar.h and libsymar.so alone (gcc, no
+    CUDA header); also the check that the header is valid C."""
+    build_lib()
+    deps = [C_EXAMPLE_SRC, ROOT / "include" / "symar.h", LIB, Path(__file__)]
+    if not force and C_EXAMPLE_BIN.exists() and all(d.stat().st_mtime <= C_EXAMPLE_BIN.stat().st_mtime for d in deps):
+        return C_EXAMPLE_BIN
+    tmp = C_EXAMPLE_BIN.with_suffix(f".bin.tmp{os.getpid()}")
+    cmd = [os.environ.get("CC", "gcc"), "-std=c99", "-pedantic", "-Wall", "-Wextra", "-Werror", "-O2",
+           "-I", str(ROOT / "include"), str(C_EXAMPLE_SRC), "-L", str(PKG), "-lsymar", "-Wl,-rpath,$ORIGIN",
+           "-o", str(tmp)]
+    subprocess.run(cmd, check=True)
+    os.replace(tmp, C_EXAMPLE_BIN)
+    return C_EXAMPLE_BIN
+
+
 if __name__ == "__main__":
     print(build_lib(force="--force" in sys.argv, verbose="-v" in sys.argv))
     print(build_example(force="--force" in sys.argv))
+    print(build_c_example(force="--force" in sys.argv))
     if "--sys" in sys.argv:
         print(build_lib_sys(force="--force" in sys.argv))
     if "--check" in sys.argv:
