@@ -173,8 +173,9 @@ static LaunchCfg default_cfg(symheap *h, int algo, uint64_t nvec, KernelFn fn)
                                                                             : nvec;   // vectors per rank partition
     if (algo == SYMAR_TWOSHOT && nvec >= kBulkMinVec) {
         // Bandwidth regime: the register kernel with 512 threads per SM in all, in as many CTAs per rank as
-        // half or a quarter of the SMs (CTA c of every rank then lands on the same one or two SMs, so the
-        // CTAs that signal one another sit together): 37 x 256 among eight ranks, 74 x 256 among four,
+        // half or a quarter of the SMs (all ranks' CTAs together are then a whole number per SM, an even
+        // load; 64 CTAs per rank among eight leave some SMs with three and some with four): 37 x 256 among
+        // eight ranks, 74 x 256 among four,
         // 74 x 512 between two.  The bulk-copy kernel comes within 3 % with about 100 CTAs in total, each
         // with one 64 KiB stage ahead of the one it reduces, and the tuner still times it; from 4 to 16 MiB,
         // where repeated calls find their buffers in L2, it is 10 to 40 % behind.
@@ -192,7 +193,7 @@ static LaunchCfg default_cfg(symheap *h, int algo, uint64_t nvec, KernelFn fn)
         const uint64_t budget = P == 2 ? 16384 : 8192;
         if (nvec >= kCyclicMinVec) {
             // from 1 MiB blocks of 8 KiB are dealt to the ranks and a thread moves 32 bytes per trip: half as
-            // many CTAs per rank as SMs (see above), small ones (measured at 1 MiB among eight ranks: 74 CTAs
+            // many CTAs per rank as SMs (an even load, see above), small ones (measured at 1 MiB among eight ranks: 74 CTAs
             // of 64 threads 4.7 us, 64 of 64 5.2 us, 16 of 512 6.5 us)
             // (at 2 MiB: 16 to 18 CTAs of 512 threads 7.1 us, 37 of 256 7.4 to 8.4 us, 74 of 128 7.9 us)
             const uint64_t n    = std::min((work + 1) / 2, budget);
