@@ -193,9 +193,9 @@ static LaunchCfg default_cfg(symheap *h, int algo, uint64_t nvec, KernelFn fn)
         const uint64_t budget = P == 2 ? 16384 : 8192;
         if (nvec >= kCyclicMinVec) {
             // from 1 MiB blocks of 8 KiB are dealt to the ranks and a thread moves 32 bytes per trip: half as
-            // many CTAs per rank as SMs (an even load, see above), small ones (measured at 1 MiB among eight ranks: 74 CTAs
-            // of 64 threads 4.7 us, 64 of 64 5.2 us, 16 of 512 6.5 us)
-            // (at 2 MiB: 16 to 18 CTAs of 512 threads 7.1 us, 37 of 256 7.4 to 8.4 us, 74 of 128 7.9 us)
+            // many CTAs per rank as SMs (an even load, see above), small ones.  Measured among eight ranks at
+            // 1 MiB: 74 CTAs of 64 threads 4.7 us, 64 of 64 5.2 us, 16 of 512 6.5 us; at 2 MiB: 16 to 18 CTAs of
+            // 512 threads 7.1 us, 37 of 256 7.4 to 8.4 us, 74 of 128 7.9 us.
             const uint64_t n    = std::min((work + 1) / 2, budget);
             const uint64_t half = (uint64_t)std::max(1, std::min(h->num_sms / 2, (int)kMaxCtas));
             if (n <= half * 64) {
@@ -226,8 +226,8 @@ static LaunchCfg default_cfg(symheap *h, int algo, uint64_t nvec, KernelFn fn)
     if (algo == SYMAR_ONESHOT) {
         // Small messages are bound by the per-thread instruction chain, so a thread takes 8 bytes up to
         // 64 KiB (4 up to 256 B, where that still fills a warp) and 16 above.  One unit per thread: one CTA
-        // up to 256 units, blocks of 128 up to half as many CTAs per rank as SMs, then larger blocks as far as the kernel's
-        // registers let all ranks' CTAs be resident together; beyond that equal passes.
+        // up to 256 units, blocks of 128 up to half as many CTAs per rank as SMs, then larger blocks as far as
+        // the kernel's registers let all ranks' CTAs be resident together; beyond that equal passes.
         const int narrow = bytes <= 256 ? 2 : (bytes <= (64u << 10) ? 1 : 0);
         c.variant = narrow << 8;
         const uint64_t units = work << narrow;
