@@ -293,7 +293,15 @@ int symar_set_launch(symheap_t *heap, symar_algo_t algo, int ctas_per_rank, int 
  * bit 2 = the register kernel instead of the bulk-copy kernel from 4 MiB (the built-in
  * choice there), bit 6 = 8 instead of 16 bytes per thread and
  * trip for messages below 1 MiB, bits 8-10 = the bulk kernel's pipeline depth (0:
- * default), bits 12-13 = log2 of its tile size over 4 KiB.                        */
+ * default), bits 12-13 = log2 of its tile size over 4 KiB.
+ * Every algorithm: SYMAR_VARIANT_CLUSTER (bit 30) = the P CTAs of a slot, one per rank, are launched
+ * as one thread-block cluster, i.e. on SMs of one GPC and so on one half of the chip.  Only their
+ * placement changes: the kernels use nothing of a cluster (no distributed shared memory, no cluster
+ * barrier), the ranks meet through flags in global memory as before.  Ignored for one rank and for the
+ * bulk-copy kernel; where the clusters of a shape cannot all be resident, that shape is launched
+ * plainly (symar_last_kernel tells).  The built-in choice and the tuner set it where it was measured
+ * faster: the data+flag protocol at every size, the others while their CTAs are few.              */
+#define SYMAR_VARIANT_CLUSTER 0x40000000u
 int symar_set_variant(symheap_t *heap, symar_algo_t algo, unsigned int variant);
 
 /* Programmatic dependent launch (ON by default; SYMAR_PDL=0 in the environment or

@@ -134,6 +134,20 @@ static int max_resident(symheap *h, KernelFn fn, int threads, size_t smem = 0)
     return n;
 }
 
+// Clusters of one slot's P CTAs that fit on the device at once (0: such a cluster cannot be launched).
+static int max_clusters(symheap *h, KernelFn fn, int threads, size_t smem)
+{
+    auto key = std::make_tuple((const void *)fn, -(threads + (int)(smem << 4)) - 1);
+    auto it  = h->resident.find(key);
+    if (it != h->resident.end()) return it->second;
+    const int n = max_resident_clusters(fn, h->P, threads, smem);
+    if (h->debug_log)
+        std::fprintf(stderr, "symar: clusters of %d CTAs x %d threads resident at once: %d%s\n", h->P, threads, n,
+                     n < 0 ? " (minus the CUDA error of the occupancy query)" : "");
+    h->resident[key] = n;
+    return n;
+}
+
 static int round_threads(uint64_t want)
 {
     int t = 32;
@@ -160,10 +174,26 @@ static unsigned ll_default_gap(int P, uint64_t bytes)
     return 12;
 }
 
+// Whether the P CTAs of a slot are launched as one thread-block cluster (on SMs of one GPC, hence on one
+// half of the chip) when nobody said otherwise.  Measured on B200, A/B on one heap (64-call graphs): the
+// data+flag protocol gains 0.2 to 0.5 us at nearly every size and rank count (its rows are written and
+// polled across the chip otherwise); one-shot and two-shot gain 0.03 to 0.13 us while the CTAs are few
+// and lose as much or far more once they fill the chip (a cluster must find P free SMs in one GPC).
+static bool cluster_default(int algo, int P, uint64_t bytes)
+{
+    if (P < 2 || bytes >= kBulkMinVec * 16) return false;
+    if (is_push(algo)) return true;                      // sentinel and the push two-shots gain 0.2 to 1 us
+    if (algo == SYMAR_ONESHOT)
+        return P == 8 ? bytes <= (128u << 10) : (P == 4 ? bytes > (16u << 10) && bytes <= (2u << 20) : bytes >= (128u << 10));
+    if (algo == SYMAR_TWOSHOT)
+        return P == 8 ? bytes <= (128u << 10) : (P == 4 ? bytes <= (256u << 10) : bytes >= (16u << 10));
+    return false;
+}
+
 // Launch shape when neither the caller nor the tuner fixed one.  Every rule here restates what the
 // tuner chose on B200 for 2, 4 and 8 ranks from 128 B to 256 MiB; an untuned call stays within a few
 // percent of the tuned one (measured: at most 7 %, typically 0 to 3 %).
-static LaunchCfg default_cfg(symheap *h, int algo, uint64_t nvec, KernelFn fn)
+static LaunchCfg default_shape(symheap *h, int algo, uint64_t nvec, KernelFn fn)
 {
     LaunchCfg c;
     c.variant = 0;
@@ -260,7 +290,7 @@ static LaunchCfg default_cfg(symheap *h, int algo, uint64_t nvec, KernelFn fn)
         c.variant = 0x100 | (ll_default_gap(P, bytes) << 12);
         units     = work * 2;
         c.threads = units <= 256 ? round_threads(units) : (units < 2048 ? 64 : (units <= 8192 ? 128 : 256));
-        if (P == 2 && units > 256) c.threads = units <= 512 ? 128 : 256;     // between two ranks: few, larger CTAs
+        if (P == 2 && units > 256) c.threads = (units <= 512 || units > 1024) ? 128 : 256;   // between two ranks: as the tuner chose
         c.ctas    = (int)std::min<uint64_t>((units + c.threads - 1) / c.threads, (uint64_t)kLLSlots);
         return c;
     }
@@ -271,6 +301,13 @@ static LaunchCfg default_cfg(symheap *h, int algo, uint64_t nvec, KernelFn fn)
     return c;
 }
 
+static LaunchCfg default_cfg(symheap *h, int algo, uint64_t nvec, KernelFn fn)
+{
+    LaunchCfg c = default_shape(h, algo, nvec, fn);
+    if (cluster_default(algo, h->P, nvec * 16)) c.variant |= (int)kVarCluster;
+    return c;
+}
+
 // Before autotuning.  Measured on B200: with ranks that share one L2 the pull
 // one-shot wins from about 1 KiB up to 256 KiB per rank, two-shot above; LL saves
 // one dependent round trip and pays for it with P - 1 flagged stores and polls per
@@ -278,10 +315,11 @@ static LaunchCfg default_cfg(symheap *h, int algo, uint64_t nvec, KernelFn fn)
 static int default_algo(int P, size_t bytes)
 {
     // the data+flag protocol leads at the smallest sizes (Sec. VII Obs. 1); measured here, with flag
-    // and counter reads placed on the reader's L2 half: up to 8 KiB between two ranks (1.2 to 1.35
-    // against 1.35 to 1.45 us), nowhere among four or eight (one-shot 1.37 / 1.43 us against 1.43 / 1.57 us
-    // at 128 B)
-    if (P == 2 && bytes <= 8192) return SYMAR_LL;
+    // and counter reads placed on the reader's L2 half and each slot's ranks launched as a cluster: between
+    // two ranks within 0.1 us of one-shot either way up to 2 KiB (which of the two leads differs from GPU
+    // to GPU) and 0.03 to 0.1 us ahead from 4 to 32 KiB; among four within 0.1 us up to 4 KiB, among eight
+    // 0.15 us and more behind everywhere
+    if (P == 2 && bytes <= (32u << 10)) return SYMAR_LL;
     // one-shot reads P times the bytes two-shot does and saves its second synchronisation: the
     // break-even moves up fourfold each time the rank count halves (measured 256 KiB, 1 MiB, 4 to 8 MiB)
     const size_t limit = (size_t)(256u << 10) * (size_t)(64 / (P * P));
@@ -294,6 +332,7 @@ struct Plan {
     LaunchCfg cfg;
     KernelFn  fn;
     size_t    smem = 0;     // dynamic shared memory of the launch
+    bool      cluster = false;   // the ranks of a slot as one thread-block cluster
     KArgs     args;
 };
 
@@ -320,7 +359,8 @@ static int make_plan(symheap *h, size_t in_off, size_t out_off, size_t count, in
     if (h->forced[algo].threads > 0) cfg.threads = h->forced[algo].threads;
     if (h->variant_forced[algo]) cfg.variant = (int)h->variant[algo];
     if (cfg.variant < 0) cfg.variant = 0;
-    const unsigned var = (unsigned)cfg.variant;
+    bool cluster       = ((unsigned)cfg.variant & kVarCluster) != 0 && h->P > 1;
+    const unsigned var = (unsigned)cfg.variant & ~kVarCluster;      // what the kernel sees
 
     cfg.threads = std::min<int>(std::max(32, (cfg.threads + 31) / 32 * 32),
                                 is_twoshot_push(algo) ? (int)kPushTwoshotMaxThreads
@@ -368,8 +408,13 @@ static int make_plan(symheap *h, size_t in_off, size_t out_off, size_t count, in
             cfg.ctas = (int)need;
         }
     }
-    const int cap_res   = std::max(1, max_resident(h, fn, cfg.threads, p->smem) / h->P);
+    const int cap_res = std::max(1, max_resident(h, fn, cfg.threads, p->smem) / h->P);
     cfg.ctas = std::max(1, std::min({cfg.ctas, cap_slots, cap_res}));
+    // all clusters must be resident together, like all CTAs; where they are not, the plain launch of the
+    // same shape (the bulk-copy kernel is never launched in clusters)
+    if (cluster && (p->smem != 0 || max_clusters(h, fn, cfg.threads, p->smem) < cfg.ctas)) cluster = false;
+    cfg.variant = (int)(var | (cluster ? kVarCluster : 0u));
+    p->cluster  = cluster;
 
     a.seg0       = h->seg0;
     a.stride     = h->L.stride;
@@ -449,16 +494,16 @@ static int run(symheap *h, const void *in, void *out, size_t count, int dtype, i
     Plan p;
     rc = make_plan(h, io, oo, count, dtype, algo, &p);
     if (rc != SYMAR_OK) return rc;
-    cudaError_t e = launch_kernel(p.fn, h->P, p.cfg.ctas, p.cfg.threads, p.smem, p.args, s);
+    cudaError_t e = launch_kernel(p.fn, h->P, p.cfg.ctas, p.cfg.threads, p.smem, p.args, s, p.cluster);
     if (e != cudaSuccess) return cuda_fail(e, "kernel launch");
     h->last_algo    = p.algo;
     h->last_ctas    = p.cfg.ctas;
     h->last_threads = p.cfg.threads;
-    h->last_variant = p.args.variant;
+    h->last_variant = (unsigned)p.cfg.variant;      // with the cluster bit, which no kernel sees
     h->last_smem    = p.smem;
     if (h->debug_log)
         std::fprintf(stderr, "symar: allreduce count=%zu dtype=%d algo=%d grid=(%d,%d) block=%d variant=%#x smem=%zu pdl=%d\n",
-                     count, dtype, p.algo, p.cfg.ctas, h->P, p.cfg.threads, p.args.variant, p.smem, (int)h->pdl);
+                     count, dtype, p.algo, p.cfg.ctas, h->P, p.cfg.threads, (unsigned)p.cfg.variant, p.smem, (int)h->pdl);
     return SYMAR_OK;
 }
 
@@ -659,6 +704,8 @@ static int tune_bucket(symheap *h, int dtype, int b, size_t bytes, cudaStream_t 
         // from contiguous chunks to blocks dealt round-robin -- measured 5 to 8 % lost at 1 to 4 MiB)
         const LaunchCfg near =
             (prune && bytes > (4u << 20) && tn.cfg[algo][prev].ctas > 0) ? tn.cfg[algo][prev] : LaunchCfg{};
+        if (!bulk && cluster_default(algo, h->P, bytes))
+            for (int &v : variants) v |= (int)kVarCluster;     // launched as the built-in rule would; the second look tries the other way
         for (int var : variants) {
             // threads a shape needs: one per unit of this variant
             const uint64_t units = bulk ? work : (work << ((var >> 8) & 3)) << ((algo == SYMAR_TWOSHOT && (var & 0x40)) ? 1 : 0);
@@ -721,6 +768,13 @@ static int tune_bucket(symheap *h, int dtype, int b, size_t bytes, cudaStream_t 
         if (!bulk && rc == SYMAR_OK && cands.size() > 1 && tn.us[algo][b] <= 1.2 * best_us) {
             std::sort(cands.begin(), cands.end(), [](const Cand &x, const Cand &y) { return x.us < y.us; });
             cands.resize(std::min<size_t>(cands.size(), 3));
+            // ... each also with the slot's ranks launched the other way (as one cluster, or not)
+            if (h->P > 1)
+                for (size_t i = 0, n = cands.size(); i < n; ++i) {
+                    Cand other = cands[i];
+                    other.cfg.variant ^= (int)kVarCluster;
+                    cands.push_back(other);
+                }
             double best = 1e30;
             for (const Cand &cd : cands) {
                 h->forced[algo]         = cd.cfg;

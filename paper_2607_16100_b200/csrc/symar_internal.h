@@ -24,7 +24,12 @@ KernelFn atomic_kernel_for(int dtype, int P, bool dbg);
 
 // grid = (ctas_per_rank, P), block = threads; returns the launch status.
 cudaError_t launch_kernel(KernelFn fn, int P, int ctas_per_rank, int threads, size_t smem_bytes,
-                          const KArgs &args, cudaStream_t stream);
+                          const KArgs &args, cudaStream_t stream, bool cluster = false);
+int max_resident_clusters(KernelFn fn, int P, int threads, size_t smem_bytes);
+
+// Variant bit common to all algorithms (host side only, never passed to a kernel): launch the P CTAs of
+// a slot as one thread-block cluster.
+constexpr unsigned kVarCluster = SYMAR_VARIANT_CLUSTER;
 
 // Placement on the chip's two L2 halves (symar_place.cu): which half every SM sits on, and which half
 // homes copy 0 of every flag / counter pair of a heap.  `scratch`: 3 * kPairBytes of device memory,

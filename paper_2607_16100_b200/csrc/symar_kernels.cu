@@ -27,6 +27,8 @@
 //
 // No kernel contains a grid-wide barrier; every wait is one-directional (a CTA
 // waits for data or a signal FROM each peer) and bounded.
+#include <cstdlib>
+
 #include "symar_device.cuh"
 #include "symar_internal.h"
 
@@ -929,25 +931,61 @@ KernelFn ll_small_kernel_for(int dtype, int P, int words, bool dbg)
     return nullptr;
 }
 
-cudaError_t launch_kernel(KernelFn fn, int P, int ctas_per_rank, int threads, size_t smem_bytes,
-                          const KArgs &args, cudaStream_t stream)
+// `cluster`: the P CTAs of a slot (one per rank) are launched as one thread-block cluster, which puts them
+// on SMs of one GPC, i.e. on one half of the chip.  Nothing of a cluster is used in the kernels -- no
+// distributed shared memory, no cluster barrier: the ranks still meet through flags in global memory
+// only -- it is a statement about where the CTAs that signal one another run.
+static void launch_config(cudaLaunchConfig_t &cfg, cudaLaunchAttribute attr[2], int P, int ctas_per_rank, int threads,
+                          size_t smem_bytes, bool pdl, bool cluster, cudaStream_t stream)
 {
-    const dim3 grid((unsigned)ctas_per_rank, (unsigned)P, 1);
-    if (!args.pdl) {
-        fn<<<grid, dim3((unsigned)threads, 1, 1), smem_bytes, stream>>>(args);
-        return cudaGetLastError();
-    }
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim          = grid;
+    cfg                  = cudaLaunchConfig_t{};
+    cfg.gridDim          = dim3((unsigned)ctas_per_rank, (unsigned)P, 1);
     cfg.blockDim         = dim3((unsigned)threads, 1, 1);
     cfg.dynamicSmemBytes = smem_bytes;
     cfg.stream           = stream;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs    = attr;
-    cfg.numAttrs = 1;
+    cfg.attrs            = attr;
+    cfg.numAttrs         = 0;
+    if (pdl) {
+        attr[cfg.numAttrs].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[cfg.numAttrs].val.programmaticStreamSerializationAllowed = 1;
+        ++cfg.numAttrs;
+    }
+    if (cluster && P > 1) {
+        attr[cfg.numAttrs].id               = cudaLaunchAttributeClusterDimension;
+        attr[cfg.numAttrs].val.clusterDim.x = 1;
+        attr[cfg.numAttrs].val.clusterDim.y = (unsigned)P;
+        attr[cfg.numAttrs].val.clusterDim.z = 1;
+        ++cfg.numAttrs;
+    }
+}
+
+cudaError_t launch_kernel(KernelFn fn, int P, int ctas_per_rank, int threads, size_t smem_bytes,
+                          const KArgs &args, cudaStream_t stream, bool cluster)
+{
+    if (!args.pdl && !(cluster && P > 1)) {
+        fn<<<dim3((unsigned)ctas_per_rank, (unsigned)P, 1), dim3((unsigned)threads, 1, 1), smem_bytes, stream>>>(args);
+        return cudaGetLastError();
+    }
+    cudaLaunchConfig_t cfg;
+    cudaLaunchAttribute attr[2];
+    launch_config(cfg, attr, P, ctas_per_rank, threads, smem_bytes, args.pdl != 0, cluster, stream);
     return cudaLaunchKernelEx(&cfg, fn, args);
+}
+
+// Clusters of P CTAs (one slot's ranks) of `fn` that the device holds at once; 0 or minus the CUDA error
+// if such a cluster cannot be launched at all.
+int max_resident_clusters(KernelFn fn, int P, int threads, size_t smem_bytes)
+{
+    cudaLaunchConfig_t cfg;
+    cudaLaunchAttribute attr[2];
+    launch_config(cfg, attr, P, 1, threads, smem_bytes, false, true, nullptr);
+    int n = 0;
+    const cudaError_t e = cudaOccupancyMaxActiveClusters(&n, fn, &cfg);
+    if (e != cudaSuccess) {
+        (void)cudaGetLastError();
+        return -(int)e;                 // not launchable as clusters (the caller logs why)
+    }
+    return n;
 }
 
 }  // namespace symar

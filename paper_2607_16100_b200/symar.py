@@ -30,6 +30,7 @@ _ERR_NAMES = {
 }
 
 MAX_RANKS, MAX_CTAS, LL_SLOTS, LL_SLOT_VECS, ALIGN = 8, 160, 64, 1024, 8192
+VARIANT_CLUSTER = 0x40000000      # SYMAR_VARIANT_CLUSTER: the ranks of a slot launched as one thread-block cluster
 
 # every symbol include/symar.h declares: (name, restype, argtypes)
 SIGNATURES = [

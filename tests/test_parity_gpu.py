@@ -197,6 +197,7 @@ def test_sentinel_mode_accepts_payload_equal_to_the_sentinel(heaps):
 
 
 FORCE_PLAIN = 1 << 31
+CLUSTER = symar.VARIANT_CLUSTER
 
 
 @pytest.mark.parametrize("count", [1, 2, 3, 5, 8, 9, 63, 64, 1023, 4099, 40001])
@@ -213,7 +214,13 @@ FORCE_PLAIN = 1 << 31
                                           (symar.SENTINEL, FORCE_PLAIN), (symar.TWOSHOT_LL, FORCE_PLAIN),
                                           (symar.TWOSHOT_SENTINEL, FORCE_PLAIN),
                                           # two-shot: 16 or 8 bytes per thread and trip
-                                          (symar.TWOSHOT, FORCE_PLAIN), (symar.TWOSHOT, 0x40)])
+                                          (symar.TWOSHOT, FORCE_PLAIN), (symar.TWOSHOT, 0x40),
+                                          # the ranks of a slot launched as one thread-block cluster
+                                          (symar.ONESHOT, CLUSTER | 0x100), (symar.ONESHOT, CLUSTER),
+                                          (symar.TWOSHOT, CLUSTER), (symar.TWOSHOT, CLUSTER | 0x40),
+                                          (symar.LL, CLUSTER | 0x100), (symar.LL, CLUSTER | 0x2100),
+                                          (symar.LL, CLUSTER | 0x200), (symar.SENTINEL, CLUSTER),
+                                          (symar.TWOSHOT_LL, CLUSTER), (symar.TWOSHOT_SENTINEL, CLUSTER)])
 def test_unit_width_variants(heaps, algo, variant, P, dtype, dist, count):
     # every implementation variant of a kernel gives the same bits, whatever the ragged tail
     h = heaps[P]
@@ -221,10 +228,38 @@ def test_unit_width_variants(heaps, algo, variant, P, dtype, dist, count):
     h.set_variant(algo, variant)
     try:
         got = run(h, x, DT[dtype], algo)
-        assert h.last_kernel()[0] == variant & 0x7FFFFFFF
+        # (a cluster needs two ranks at least, and all clusters of a launch must be resident together:
+        # otherwise the same shape is launched plainly; the small launches here always fit)
+        asked = variant & 0x7FFFFFFF
+        if P == 1:
+            asked &= ~CLUSTER
+        assert h.last_kernel()[0] in ((asked,) if count < 5000 else (asked, asked & ~CLUSTER))
     finally:
         h.set_variant(algo, 0)
     assert_bits(got, O.allreduce(x), f"algo={algo} variant={variant:#x} P={P} {dtype} count={count}")
+
+
+def test_cluster_launch_falls_back_when_the_clusters_do_not_fit(heaps):
+    # 160 CTAs of 512 threads per rank cannot all be resident as clusters of eight (nor as plain CTAs): the
+    # library shrinks the grid to what fits and launches it plainly if the clusters still do not fit; a
+    # shape that fits keeps its clusters.  Same bits either way.
+    h = heaps[8]
+    x = synth.make_inputs("normal", "bf16", 8, 300001, seed=123)
+    want = O.allreduce(x)
+    try:
+        for algo in (symar.ONESHOT, symar.TWOSHOT):
+            h.set_variant(algo, CLUSTER)
+            h.set_launch(algo, 160, 512)
+            assert_bits(run(h, x, symar.BF16, algo), want, f"algo {algo}, 160 x 512")
+            big = h.last_kernel()[0] & CLUSTER
+            h.set_launch(algo, 8, 128)
+            assert_bits(run(h, x, symar.BF16, algo), want, f"algo {algo}, 8 x 128")
+            assert h.last_kernel()[0] & CLUSTER and h.last_choice()[1:] == (8, 128)
+            assert big in (0, CLUSTER)
+    finally:
+        for algo in (symar.ONESHOT, symar.TWOSHOT):
+            h.set_variant(algo, 0)
+            h.set_launch(algo, 0, 0)
 
 
 def test_ll_narrow_many_iterations_and_mixed_widths(heaps):
