@@ -12,6 +12,7 @@
 #include <new>
 #include <string>
 #include <tuple>
+#include <chrono>
 #include <vector>
 
 #include "symar_internal.h"
@@ -82,6 +83,8 @@ struct symheap {
     bool      pdl          = true;    // programmatic dependent launch of every kernel
     int       env_algo     = 0;       // SYMAR_ALGO override of SYMAR_AUTO, 0 = none
     bool      debug_log    = false;   // SYMAR_DEBUG=1: one stderr line per call
+    long      tune_timed[kAlgos] = {};   // tuner: graphs timed per algorithm, and the seconds that took
+    double    tune_secs[kAlgos]  = {};
     bool      tune_exhaustive = false;   // SYMAR_TUNE=exhaustive: the tuner prunes nothing
     int       tune_rotate = 0;        // tuner: > 0 = every call of a timing graph has its own buffers (that many pairs)
     bool      placed   = false;       // sm_half / home were measured cleanly
@@ -577,6 +580,11 @@ static int time_calls(symheap *h, cudaStream_t s, size_t count, int dtype, int a
                       double *us_out, double give_up_us = 0.0)
 {
     const size_t bytes = count * elem_size(dtype);
+    const auto wall0   = std::chrono::steady_clock::now();
+    struct Tally {
+        symheap *h; int algo; std::chrono::steady_clock::time_point t0;
+        ~Tally() { ++h->tune_timed[algo]; h->tune_secs[algo] += std::chrono::duration<double>(std::chrono::steady_clock::now() - t0).count(); }
+    } tally{h, algo, wall0};
     // Warm: every call on the same input and output.  Streaming (tune_rotate pairs): call k reads and writes its
     // own pair of buffers, as the calls of a decode step do; the graph then holds one call per pair.
     const size_t slice = round_up(bytes, kAlign);
@@ -680,8 +688,14 @@ static int tune_bucket(symheap *h, int dtype, int b, size_t bytes, cudaStream_t 
         if (bulk)
             variants = {bulk_variant(2, 1), bulk_variant(3, 1), bulk_variant(2, 2), bulk_variant(3, 0),
                         bulk_variant(4, 0), 4};
-        else if (algo == SYMAR_ONESHOT && bytes <= (1u << 20))
-            variants = {0, 0x100, 0x200};            // 16, 8 or 4 bytes per thread
+        else if (algo == SYMAR_ONESHOT && bytes <= (1u << 20)) {
+            // 16, 8 or 4 bytes per thread, each where it has ever won (exhaustive searches chose 4 bytes up to
+            // 256 B only, 8 bytes up to 64 KiB, 16 bytes from 2 KiB)
+            variants.clear();
+            if (bytes >= 2048 || h->tune_exhaustive) variants.push_back(0);
+            if (bytes <= (256u << 10) || h->tune_exhaustive) variants.push_back(0x100);
+            if (bytes <= 4096 || h->tune_exhaustive) variants.push_back(0x200);
+        }
         else if (algo == SYMAR_TWOSHOT && nvec < kCyclicMinVec)
             variants = {0, 0x40};                    // 16 or 8 bytes per thread and trip
         else if (algo == SYMAR_LL && bytes <= kLLSmallMaxBytes) {
@@ -768,9 +782,9 @@ static int tune_bucket(symheap *h, int dtype, int b, size_t bytes, cudaStream_t 
         if (!bulk && rc == SYMAR_OK && cands.size() > 1 && tn.us[algo][b] <= 1.2 * best_us) {
             std::sort(cands.begin(), cands.end(), [](const Cand &x, const Cand &y) { return x.us < y.us; });
             cands.resize(std::min<size_t>(cands.size(), 3));
-            // ... each also with the slot's ranks launched the other way (as one cluster, or not)
+            // ... the two fastest also with the slot's ranks launched the other way (as one cluster, or not)
             if (h->P > 1)
-                for (size_t i = 0, n = cands.size(); i < n; ++i) {
+                for (size_t i = 0, n = std::min<size_t>(cands.size(), 2); i < n; ++i) {
                     Cand other = cands[i];
                     other.cfg.variant ^= (int)kVarCluster;
                     cands.push_back(other);
@@ -848,6 +862,10 @@ static int autotune(symheap *h, int dtype, size_t only_bytes, int rotate = 0)
         rc = tune_bucket(h, dtype, b, (size_t)1 << b, s, tn, b > tn.lo_bucket ? b - 1 : -1);
     cudaStreamSynchronize(s);
     cudaStreamDestroy(s);
+    if (h->debug_log)
+        for (int a = SYMAR_ONESHOT; a < kAlgos; ++a)
+            if (h->tune_timed[a])
+                std::fprintf(stderr, "symar: tuner, algorithm %d: %ld graphs timed in %.2f s\n", a, h->tune_timed[a], h->tune_secs[a]);
     if (rc != SYMAR_OK) {
         h->tuned[dtype] = saved_tuned;
         return rc;
