@@ -162,19 +162,19 @@ static int round_threads(uint64_t want)
 static int bulk_variant(int stages, int tile_log2_over_4k) { return (stages << 8) | (tile_log2_over_4k << 12); }
 
 // LL, single-iteration kernel: the largest message it covers (64 slots x 256 threads x 8 bytes), and
-// the default hold-back of the first poll in steps of 64 cycles.  The hold-back pays once the P (P - 1)
-// rows in flight are enough to make polls and stores compete in L2 (measured at P = 8, 4 and 2: none
-// below about 100 KiB in flight, one store-to-poll hop -- 768 cycles -- from a megabyte up).
+// the default hold-back of the first poll in steps of 64 cycles.  A poll that leaves before the row has
+// landed costs a whole further round trip, one that leaves late costs its lateness; the best hold-back is
+// the store-to-visibility time, which grows with the rows in flight.  Measured with each slot's ranks
+// launched as a cluster (sweeps of the hold-back at P = 8, 4, 2 from 128 B to 128 KiB; the minimum is sharp:
+// 0.1 to 0.3 us lost two steps beside it): nothing up to 256 B, 128 cycles between two and among four
+// ranks up to 16 KiB, 256 cycles among eight, then growing to one full hop (768 cycles).
 constexpr uint64_t kLLSmallMaxBytes = (uint64_t)kLLSlots * kLLMaxThreads * 8;
 static unsigned ll_default_gap(int P, uint64_t bytes)
 {
-    const uint64_t in_flight = (uint64_t)P * (P - 1) * 2 * bytes;     // payload + flags, all ranks
-    if (P == 2 && bytes >= 4096 && in_flight < (192u << 10)) return 3;   // several CTAs per rank: measured -0.05 us
-    if (in_flight < (96u << 10)) return 0;
-    if (in_flight < (192u << 10)) return 2;
-    if (in_flight < (384u << 10)) return 8;
-    if (in_flight < (1u << 20)) return 10;
-    return 12;
+    if (bytes <= 256) return P == 4 ? 2 : 0;
+    if (P >= 8) return bytes <= (16u << 10) ? 4 : 12;
+    if (P == 4) return bytes <= (16u << 10) ? 2 : (bytes <= (32u << 10) ? 4 : (bytes <= (64u << 10) ? 8 : 10));
+    return 2;
 }
 
 // Whether the P CTAs of a slot are launched as one thread-block cluster (on SMs of one GPC, hence on one
@@ -293,7 +293,6 @@ static LaunchCfg default_shape(symheap *h, int algo, uint64_t nvec, KernelFn fn)
         c.variant = 0x100 | (ll_default_gap(P, bytes) << 12);
         units     = work * 2;
         c.threads = units <= 256 ? round_threads(units) : (units < 2048 ? 64 : (units <= 8192 ? 128 : 256));
-        if (P == 2 && units > 256) c.threads = (units <= 512 || units > 1024) ? 128 : 256;   // between two ranks: as the tuner chose
         c.ctas    = (int)std::min<uint64_t>((units + c.threads - 1) / c.threads, (uint64_t)kLLSlots);
         return c;
     }
@@ -318,11 +317,13 @@ static LaunchCfg default_cfg(symheap *h, int algo, uint64_t nvec, KernelFn fn)
 static int default_algo(int P, size_t bytes)
 {
     // the data+flag protocol leads at the smallest sizes (Sec. VII Obs. 1); measured here, with flag
-    // and counter reads placed on the reader's L2 half and each slot's ranks launched as a cluster: between
-    // two ranks within 0.1 us of one-shot either way up to 2 KiB (which of the two leads differs from GPU
-    // to GPU) and 0.03 to 0.1 us ahead from 4 to 32 KiB; among four within 0.1 us up to 4 KiB, among eight
-    // 0.15 us and more behind everywhere
-    if (P == 2 && bytes <= (32u << 10)) return SYMAR_LL;
+    // and counter reads placed on the reader's L2 half, each slot's ranks launched as a cluster and the
+    // first poll held back as above: between two ranks 1.37 to 1.50 us from 128 B to 64 KiB against
+    // one-shot's 1.30 to 1.56 (ahead from 4 KiB on everywhere, below that on some GPUs); among four
+    // 1.37 to 1.46 us up to 8 KiB against 1.40 to 1.53 (level or ahead); among eight 0.15 us and more
+    // behind everywhere
+    if (P == 2 && bytes <= (64u << 10)) return SYMAR_LL;
+    if (P == 4 && bytes <= (8u << 10)) return SYMAR_LL;
     // one-shot reads P times the bytes two-shot does and saves its second synchronisation: the
     // break-even moves up fourfold each time the rank count halves (measured 256 KiB, 1 MiB, 4 to 8 MiB)
     const size_t limit = (size_t)(256u << 10) * (size_t)(64 / (P * P));
@@ -700,10 +701,10 @@ static int tune_bucket(symheap *h, int dtype, int b, size_t bytes, cudaStream_t 
             variants = {0, 0x40};                    // 16 or 8 bytes per thread and trip
         else if (algo == SYMAR_LL && bytes <= kLLSmallMaxBytes) {
             // 8 bytes of payload per thread with the first poll held back by the default for this
-            // traffic, by a quarter of a hop less and more, and not at all; 16 bytes per thread
+            // size, by 128 cycles less and more, by half a hop more, and not at all; 16 bytes per thread
             const int g = (int)ll_default_gap(h->P, bytes);
             variants = {0x100 | (g << 12)};
-            for (int alt : {g - 4, g + 3, 0})
+            for (int alt : {g - 2, g + 2, g + 6, 0})
                 if (alt >= 0 && alt <= 15 && alt != g &&
                     std::find(variants.begin(), variants.end(), 0x100 | (alt << 12)) == variants.end())
                     variants.push_back(0x100 | (alt << 12));
