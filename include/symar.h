@@ -27,7 +27,8 @@
  * launch off; SYMAR_DEBUG = 1 logs every call's resolved algorithm and shape to stderr
  * (nothing is printed otherwise); SYMAR_TUNE = exhaustive makes allreduce_autotune time every
  * algorithm and shape at every size instead of pruning by the previous size's result;
- * SYMAR_PLACE = 0 turns the placement of flag and counter reads on the chip's L2 halves off.
+ * SYMAR_PLACE = 0 turns the placement of flag and counter reads on the chip's L2 halves off;
+ * SYMAR_CLUSTER = 0 keeps every launch a plain one (see SYMAR_VARIANT_CLUSTER).
  *
  * Threading: a heap may be used from one host thread and one stream at a time
  * (the per-CTA epoch counters live in the heap).  Calls on one stream are

@@ -170,8 +170,31 @@ static CollFn pick_coll(int op, int P)
 
 // Launch of one sibling collective.  `k` carries the heap addressing (as for the
 // AllReduce kernels) with in_off / out_off set; unit = 16, 4 or 2 bytes.
+static void coll_config(cudaLaunchConfig_t &cfg, cudaLaunchAttribute attr[2], int P, int ctas_per_rank, int threads,
+                        bool pdl, bool cluster, cudaStream_t stream)
+{
+    cfg          = cudaLaunchConfig_t{};
+    cfg.gridDim  = dim3((unsigned)ctas_per_rank, (unsigned)P, 1);
+    cfg.blockDim = dim3((unsigned)threads, 1, 1);
+    cfg.stream   = stream;
+    cfg.attrs    = attr;
+    cfg.numAttrs = 0;
+    if (pdl) {
+        attr[cfg.numAttrs].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[cfg.numAttrs].val.programmaticStreamSerializationAllowed = 1;
+        ++cfg.numAttrs;
+    }
+    if (cluster && P > 1) {       // the ranks of a slot on SMs of one GPC (placement only, as for the AllReduce kernels)
+        attr[cfg.numAttrs].id               = cudaLaunchAttributeClusterDimension;
+        attr[cfg.numAttrs].val.clusterDim.x = 1;
+        attr[cfg.numAttrs].val.clusterDim.y = (unsigned)P;
+        attr[cfg.numAttrs].val.clusterDim.z = 1;
+        ++cfg.numAttrs;
+    }
+}
+
 cudaError_t launch_collective(int op, int dtype, int P, int ctas_per_rank, int threads, const KArgs &k,
-                              uint64_t bytes, int root, int unit, cudaStream_t stream)
+                              uint64_t bytes, int root, int unit, cudaStream_t stream, bool cluster)
 {
     CollFn fn = dtype == SYMAR_F32 ? pick_coll<F32>(op, P) : pick_coll<BF16>(op, P);
     if (!fn) return cudaErrorInvalidValue;
@@ -180,21 +203,30 @@ cudaError_t launch_collective(int op, int dtype, int P, int ctas_per_rank, int t
     a.k.variant = (uint32_t)unit;
     a.bytes     = bytes;
     a.root      = root;
-    const dim3 grid((unsigned)ctas_per_rank, (unsigned)P, 1), block((unsigned)threads, 1, 1);
-    if (!k.pdl) {
-        fn<<<grid, block, 0, stream>>>(a);
+    if (!k.pdl && !(cluster && P > 1)) {
+        fn<<<dim3((unsigned)ctas_per_rank, (unsigned)P, 1), dim3((unsigned)threads, 1, 1), 0, stream>>>(a);
         return cudaGetLastError();
     }
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim  = grid;
-    cfg.blockDim = block;
-    cfg.stream   = stream;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs    = attr;
-    cfg.numAttrs = 1;
+    cudaLaunchConfig_t cfg;
+    cudaLaunchAttribute attr[2];
+    coll_config(cfg, attr, P, ctas_per_rank, threads, k.pdl != 0, cluster, stream);
     return cudaLaunchKernelEx(&cfg, fn, a);
+}
+
+// clusters of one slot's P CTAs of a collective kernel that the device holds at once (0: none can be launched)
+int collective_resident_clusters(int op, int dtype, int P, int threads)
+{
+    CollFn fn = dtype == SYMAR_F32 ? pick_coll<F32>(op, P) : pick_coll<BF16>(op, P);
+    if (!fn || P < 2) return 0;
+    cudaLaunchConfig_t cfg;
+    cudaLaunchAttribute attr[2];
+    coll_config(cfg, attr, P, 1, threads, false, true, nullptr);
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, fn, &cfg) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return 0;
+    }
+    return n;
 }
 
 // co-resident CTAs of a collective kernel at the given block size (they wait for one another)

@@ -82,6 +82,7 @@ struct symheap {
     uint64_t  spin_ns = 200000000ull;    // 200 ms: hundreds of times the longest call (a 256 MiB message takes 0.65 ms)
     bool      pdl          = true;    // programmatic dependent launch of every kernel
     int       env_algo     = 0;       // SYMAR_ALGO override of SYMAR_AUTO, 0 = none
+    bool      cluster_on   = true;    // SYMAR_CLUSTER=0: never launch a slot's ranks as a thread-block cluster
     bool      debug_log    = false;   // SYMAR_DEBUG=1: one stderr line per call
     long      tune_timed[kAlgos] = {};   // tuner: graphs timed per algorithm, and the seconds that took
     double    tune_secs[kAlgos]  = {};
@@ -363,7 +364,7 @@ static int make_plan(symheap *h, size_t in_off, size_t out_off, size_t count, in
     if (h->forced[algo].threads > 0) cfg.threads = h->forced[algo].threads;
     if (h->variant_forced[algo]) cfg.variant = (int)h->variant[algo];
     if (cfg.variant < 0) cfg.variant = 0;
-    bool cluster       = ((unsigned)cfg.variant & kVarCluster) != 0 && h->P > 1;
+    bool cluster       = ((unsigned)cfg.variant & kVarCluster) != 0 && h->P > 1 && h->cluster_on;
     const unsigned var = (unsigned)cfg.variant & ~kVarCluster;      // what the kernel sees
 
     cfg.threads = std::min<int>(std::max(32, (cfg.threads + 31) / 32 * 32),
@@ -562,7 +563,18 @@ static int run_collective(symheap *h, int op, const void *in, void *out, size_t 
         std::memcpy(a.sm_half, h->sm_half, sizeof a.sm_half);
         a.home = h->home;
     }
-    cudaError_t e = launch_collective(op, dtype, h->P, ctas, threads, a, bytes, root, unit, s);
+    // each slot's ranks as one cluster while the CTAs are few (the one-shot AllReduce's rule: these kernels
+    // have its structure; measured -0.03 to -0.13 us up to 64 KiB among eight ranks), if all clusters can be
+    // resident together
+    bool cluster = h->cluster_on && cluster_default(SYMAR_ONESHOT, h->P, op == 0 ? in_total : out_total);
+    if (cluster) {
+        auto key = std::make_tuple((const void *)(intptr_t)(0x1000 + op * 16 + dtype), -threads - 1);
+        auto it  = h->resident.find(key);
+        const int n = it != h->resident.end() ? it->second
+                                              : (h->resident[key] = collective_resident_clusters(op, dtype, h->P, threads));
+        cluster = n >= ctas;
+    }
+    cudaError_t e = launch_collective(op, dtype, h->P, ctas, threads, a, bytes, root, unit, s, cluster);
     if (e != cudaSuccess) return cuda_fail(e, "collective launch");
     h->last_algo    = SYMAR_ONESHOT;
     h->last_ctas    = ctas;
@@ -982,6 +994,7 @@ static int create_common(symheap_t **heap, int P, size_t bytes_per_rank, void *m
             for (int a = SYMAR_ONESHOT; a <= kLastAlgo; ++a) h->forced[a].threads = t;
     }
     if (const char *v = std::getenv("SYMAR_DEBUG")) h->debug_log = std::atoi(v) != 0;
+    if (const char *v = std::getenv("SYMAR_CLUSTER")) h->cluster_on = std::atoi(v) != 0;
     if (const char *v = std::getenv("SYMAR_TUNE")) h->tune_exhaustive = std::string(v) == "exhaustive";
     *heap = h;
     return SYMAR_OK;

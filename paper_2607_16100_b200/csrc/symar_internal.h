@@ -43,7 +43,8 @@ cudaError_t launch_check_selftest(const KArgs &args, cudaStream_t stream);
 
 // Sibling collectives (symar_coll.cu): op = 0 ReduceScatter, 1 AllGather, 2 Broadcast, 3 Reduce.
 cudaError_t launch_collective(int op, int dtype, int P, int ctas_per_rank, int threads, const KArgs &k,
-                              uint64_t bytes, int root, int unit, cudaStream_t stream);
+                              uint64_t bytes, int root, int unit, cudaStream_t stream, bool cluster = false);
+int collective_resident_clusters(int op, int dtype, int P, int threads);
 int collective_resident(int op, int dtype, int P, int threads, int num_sms);
 
 }  // namespace symar

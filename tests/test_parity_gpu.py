@@ -802,3 +802,28 @@ def test_prior_art_two_barrier_oneshot_gives_the_same_bits(heaps):
         assert_bits(run(h, x, symar.BF16, symar.TWOSHOT), O.allreduce(x))      # shares the done flags
     finally:
         h.set_variant(symar.ONESHOT, 0)
+
+
+def test_symar_cluster_env_keeps_every_launch_plain(monkeypatch):
+    # SYMAR_CLUSTER=0 (read when a heap is created): no launch carries the cluster attribute, whatever the
+    # built-in rule or a forced variant says; results are the same bits
+    monkeypatch.setenv("SYMAR_CLUSTER", "0")
+    h = symar.SymHeap.on_torch(4, 1 << 20)
+    monkeypatch.delenv("SYMAR_CLUSTER")
+    g = symar.SymHeap.on_torch(4, 1 << 20)
+    try:
+        x = synth.make_inputs("normal", "bf16", 4, 3001, seed=66)
+        want = O.allreduce(x)
+        for algo in (symar.LL, symar.ONESHOT):
+            assert_bits(run(h, x, symar.BF16, algo), want)
+            assert not h.last_kernel()[0] & CLUSTER
+            h.set_variant(algo, CLUSTER | 0x100)
+            assert_bits(run(h, x, symar.BF16, algo), want)
+            assert not h.last_kernel()[0] & CLUSTER
+            h.set_variant(algo, 0)
+        assert_bits(run(g, x, symar.BF16, symar.LL), want)
+        assert g.last_kernel()[0] & CLUSTER                       # the built-in choice for the data+flag protocol
+    finally:
+        torch.cuda.synchronize()
+        h.destroy()
+        g.destroy()
