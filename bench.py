@@ -546,8 +546,8 @@ def latency_suite(torch, symar, synth, hbm_gbs, quick=False, autotune=True):
                 "ratio_to_sol": p50_all["median"] / sol,
                 "sol_note": "empty launch = the smallest p50 over the repeats of a plain launch of the selector's grid and "
                             "block with programmatic dependent launch (the selector's own launch may also put each slot's "
-                            "ranks in one thread-block cluster; the plain empty launch is the lower of the two, so the "
-                            "stricter bound); flag round trip = the MEDIAN over SM pairs "
+                            "ranks in one thread-block cluster: the bound's empty launch never does); flag round trip = the MEDIAN over SM "
+                            "pairs "
                             "spread over the chip (the exchange needs every pair of ranks, wherever their CTAs sit; two hops "
                             "through L2 of a flag that is not placed), median over the repeats; the same bound with the "
                             "FASTEST pair follows.  The kernel's own exchange is one hop and a poll of a flag placed on the "
