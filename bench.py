@@ -369,9 +369,26 @@ def latency_suite(torch, symar, synth, hbm_gbs, quick=False, autotune=True):
         out["barrier_us"] = {"error": str(exc)}
 
     def empty_floor(cx, py, T, pdl=True, n=None):
+        """The launch floor of a grid (cx, py) of T threads: an empty kernel, with programmatic dependent launch
+        as the library launches; the smaller of the plain launch and the launch with each column's py CTAs as
+        one thread-block cluster (the library uses either, and the cluster launch is often the cheaper one)."""
         probe = symar.probe_empty_pdl if pdl else symar.probe_empty
         g = graph_of(torch, stream, lambda k, s: probe(cx, py, T, s), K)
-        return time_graph(torch, g, stream, K, n or reps)
+        r = time_graph(torch, g, stream, K, n or reps)
+        r["form"] = "plain"
+        if pdl and 2 <= py <= 8:
+            c_ = empty_floor_cluster(cx, py, T, n)
+            r["plain_p50"], r["slot_clusters_p50"] = r["p50"], c_
+            if c_ is not None and c_ < r["p50"]:
+                r["p50"], r["form"] = c_, "slot clusters"
+        return r
+
+    def empty_floor_cluster(cx, py, T, n=None):
+        try:
+            g = graph_of(torch, stream, lambda k, s: symar.probe_empty_cluster(cx, py, T, s), K)
+            return time_graph(torch, g, stream, K, n or reps)["p50"]
+        except symar.SymarError:
+            return None               # such a cluster cannot be launched
 
     for P in (8, 4):
         h = symar.SymHeap.on_torch(P, 24 << 20)
@@ -542,11 +559,15 @@ def latency_suite(torch, symar, synth, hbm_gbs, quick=False, autotune=True):
                 "oracle_cpu": oracle_us(O, load_inputs(8192)),
                 "sol_us": sol,
                 "sol_parts_us": {"empty_launch_same_shape": floor_us, "empty_launch_1x1": floor11["p50"],
-                                 "flag_round_trip": rt_us, "bytes_at_peak": t_bytes_us},
+                                 "flag_round_trip": rt_us, "bytes_at_peak": t_bytes_us,
+                                 "empty_launch_plain": floor.get("plain_p50"),
+                                 "empty_launch_slot_clusters": floor.get("slot_clusters_p50"),
+                                 "selector_launch_uses_slot_clusters":
+                                     bool(best.get("variant", 0) & symar.VARIANT_CLUSTER)},
                 "ratio_to_sol": p50_all["median"] / sol,
-                "sol_note": "empty launch = the smallest p50 over the repeats of a plain launch of the selector's grid and "
-                            "block with programmatic dependent launch (the selector's own launch may also put each slot's "
-                            "ranks in one thread-block cluster: the bound's empty launch never does); flag round trip = the MEDIAN over SM "
+                "sol_note": "empty launch = the smallest p50 over the repeats of an empty kernel in the selector's grid "
+                            "and block with programmatic dependent launch, launched plainly or with each slot's ranks as "
+                            "one thread-block cluster, whichever is cheaper; flag round trip = the MEDIAN over SM "
                             "pairs "
                             "spread over the chip (the exchange needs every pair of ranks, wherever their CTAs sit; two hops "
                             "through L2 of a flag that is not placed), median over the repeats; the same bound with the "

@@ -441,6 +441,9 @@ const char *symar_last_cuda_error(void);
 int symar_probe_empty(int grid_x, int grid_y, int block, void *cuda_stream);
 /* the launch floor with programmatic dependent launch (see symar_set_pdl) */
 int symar_probe_empty_pdl(int grid_x, int grid_y, int block, void *cuda_stream);
+/* the same with the grid_y (2..8) CTAs of every column launched as one thread-block cluster, as
+ * SYMAR_VARIANT_CLUSTER launches the ranks of a slot */
+int symar_probe_empty_cluster(int grid_x, int grid_y, int block, void *cuda_stream);
 int symar_probe_fence(int iterations, double *host_ns_per_fence);
 int symar_probe_pingpong(int iterations, double *host_ns_per_round_trip);
 /* The same between block 0 and block `partner_block` of a (partner_block + 1)-block

@@ -159,6 +159,25 @@ int symar_probe_empty_pdl(int grid_x, int grid_y, int block, void *cuda_stream)
     return cudaLaunchKernelEx(&cfg, empty_pdl_kernel) == cudaSuccess ? SYMAR_OK : SYMAR_ERR_CUDA;
 }
 
+int symar_probe_empty_cluster(int grid_x, int grid_y, int block, void *cuda_stream)
+{
+    if (grid_x < 1 || grid_y < 2 || grid_y > 8 || block < 1 || block > 1024) return SYMAR_ERR_INVAL;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim  = dim3(grid_x, grid_y, 1);
+    cfg.blockDim = dim3(block, 1, 1);
+    cfg.stream   = (cudaStream_t)cuda_stream;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[1].id               = cudaLaunchAttributeClusterDimension;     // the grid_y CTAs of a column as one cluster
+    attr[1].val.clusterDim.x = 1;
+    attr[1].val.clusterDim.y = (unsigned)grid_y;
+    attr[1].val.clusterDim.z = 1;
+    cfg.attrs    = attr;
+    cfg.numAttrs = 2;
+    return cudaLaunchKernelEx(&cfg, empty_pdl_kernel) == cudaSuccess ? SYMAR_OK : SYMAR_ERR_CUDA;
+}
+
 int symar_probe_fence(int iterations, double *host_ns_per_fence)
 {
     if (iterations < 1 || !host_ns_per_fence) return SYMAR_ERR_INVAL;

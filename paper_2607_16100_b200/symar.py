@@ -71,6 +71,7 @@ SIGNATURES = [
     ("symar_last_cuda_error", c_char_p, []),
     ("symar_probe_empty", c_int, [c_int, c_int, c_int, c_void_p]),
     ("symar_probe_empty_pdl", c_int, [c_int, c_int, c_int, c_void_p]),
+    ("symar_probe_empty_cluster", c_int, [c_int, c_int, c_int, c_void_p]),
     ("symar_probe_fence", c_int, [c_int, POINTER(c_double)]),
     ("symar_probe_pingpong", c_int, [c_int, POINTER(c_double)]),
     ("symar_probe_pingpong_pair", c_int, [c_int, c_int, POINTER(c_double), POINTER(c_int)]),
@@ -371,6 +372,10 @@ def probe_empty(grid_x: int, grid_y: int, block: int, stream: int = 0) -> None:
 
 def probe_empty_pdl(grid_x: int, grid_y: int, block: int, stream: int = 0) -> None:
     _ck(load().symar_probe_empty_pdl(grid_x, grid_y, block, stream), "symar_probe_empty_pdl")
+
+
+def probe_empty_cluster(grid_x: int, grid_y: int, block: int, stream: int = 0) -> None:
+    _ck(load().symar_probe_empty_cluster(grid_x, grid_y, block, stream), "symar_probe_empty_cluster")
 
 
 def probe_fence(iterations: int = 20000) -> float:
