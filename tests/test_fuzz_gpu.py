@@ -76,8 +76,13 @@ def test_random_call_sequences(P, seed):
                 algo = int(rng.choice(EXACT + [symar.TWOSHOT_ATOMIC]))
                 if rng.random() < 0.3 and algo != symar.AUTO:
                     h.set_launch(algo, int(rng.choice([1, 2, 3, 5, 8, 16, 40])), int(rng.choice([32, 64, 96, 128, 256, 512])))
-                if rng.random() < 0.2 and algo in (symar.ONESHOT, symar.LL):
-                    h.set_variant(algo, int(rng.choice([0x100, 0x200 if algo == symar.ONESHOT else 0x100, 1 << 31])))
+                if rng.random() < 0.3 and algo != symar.AUTO:
+                    # unit widths, the plain form, each slot's ranks as a cluster or not (whatever the built-in rule says)
+                    cl = symar.VARIANT_CLUSTER
+                    choices = {symar.ONESHOT: [0x100, 0x200, 1 << 31, cl, cl | 0x100],
+                               symar.LL: [0x100, 1 << 31, cl | 0x100, cl | 0x2100, cl | 0x200],
+                               symar.TWOSHOT: [0x40, 1 << 31, cl, cl | 0x40]}.get(algo, [1 << 31, cl])
+                    h.set_variant(algo, int(rng.choice(choices)))
                 if rng.random() < 0.15:
                     h.set_scratch_limit(int(rng.choice([0, 4096, 65536])))
                 if rng.random() < 0.2:
