@@ -228,7 +228,7 @@ int symar_reduce(symheap_t *heap, const void *in, void *out, size_t count,
  * are searched around the previous size's winner (SYMAR_TUNE = exhaustive in the
  * environment searches everything).  Synchronous; takes seconds.  OVERWRITES the
  * user region of every rank.  Before it is called, built-in defaults apply: the
- * data+flag protocol up to 64 KiB between two ranks and up to 8 KiB among four, else one-shot up to
+ * data+flag protocol up to 128 KiB between two ranks, 32 KiB among four and 256 B among eight, else one-shot up to
  * 256 KiB x (8 / P)^2 per rank, else two-shot, each in a launch shape that restates
  * what this tuner chose on B200 (within a few percent of a tuned call).          */
 int allreduce_autotune(symheap_t *heap, symar_dtype_t dtype);

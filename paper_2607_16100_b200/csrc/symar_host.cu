@@ -165,17 +165,18 @@ static int bulk_variant(int stages, int tile_log2_over_4k) { return (stages << 8
 // LL, single-iteration kernel: the largest message it covers (64 slots x 256 threads x 8 bytes), and
 // the default hold-back of the first poll in steps of 64 cycles.  A poll that leaves before the row has
 // landed costs a whole further round trip, one that leaves late costs its lateness; the best hold-back is
-// the store-to-visibility time, which grows with the rows in flight.  Measured with each slot's ranks
-// launched as a cluster (sweeps of the hold-back at P = 8, 4, 2 from 128 B to 128 KiB; the minimum is sharp:
-// 0.1 to 0.3 us lost two steps beside it): nothing up to 256 B, 128 cycles between two and among four
-// ranks up to 16 KiB, 256 cycles among eight, then growing to one full hop (768 cycles).
+// the store-to-visibility time less what the kernel does anyway between its stores and its first poll.
+// Measured with each slot's ranks launched as a cluster (sweeps at P = 8, 4, 2 from 128 B to 128 KiB; the
+// minimum is sharp: 0.06 to 0.15 us lost one step of 128 cycles beside it): nothing up to 256 B and
+// between two ranks up to 4 KiB, 128 cycles up to 16 KiB (256 among eight ranks in one CTA per rank),
+// then growing with the rows in flight to a full hop (768 cycles).
 constexpr uint64_t kLLSmallMaxBytes = (uint64_t)kLLSlots * kLLMaxThreads * 8;
 static unsigned ll_default_gap(int P, uint64_t bytes)
 {
-    if (bytes <= 256) return P == 4 ? 2 : 0;
-    if (P >= 8) return bytes <= (16u << 10) ? 4 : 12;
-    if (P == 4) return bytes <= (16u << 10) ? 2 : (bytes <= (32u << 10) ? 4 : (bytes <= (64u << 10) ? 8 : 10));
-    return 2;
+    if (bytes <= 256) return 0;
+    if (P >= 8) return bytes <= 2048 ? 4 : (bytes <= (16u << 10) ? 2 : (bytes <= (32u << 10) ? 12 : 8));
+    if (P == 4) return bytes <= (16u << 10) ? 2 : (bytes <= (32u << 10) ? 4 : (bytes <= (64u << 10) ? 6 : 8));
+    return bytes <= 4096 ? 0 : 2;
 }
 
 // Whether the P CTAs of a slot are launched as one thread-block cluster (on SMs of one GPC, hence on one
@@ -293,7 +294,7 @@ static LaunchCfg default_shape(symheap *h, int algo, uint64_t nvec, KernelFn fn)
         // per thread at every size it covers), first poll held back by the default for this traffic
         c.variant = 0x100 | (ll_default_gap(P, bytes) << 12);
         units     = work * 2;
-        c.threads = units <= 256 ? round_threads(units) : (units < 2048 ? 64 : (units <= 8192 ? 128 : 256));
+        c.threads = units <= 128 ? round_threads(units) : (units < 2048 ? 64 : (units <= 8192 ? 128 : 256));
         c.ctas    = (int)std::min<uint64_t>((units + c.threads - 1) / c.threads, (uint64_t)kLLSlots);
         return c;
     }
@@ -319,12 +320,12 @@ static int default_algo(int P, size_t bytes)
 {
     // the data+flag protocol leads at the smallest sizes (Sec. VII Obs. 1); measured here, with flag
     // and counter reads placed on the reader's L2 half, each slot's ranks launched as a cluster and the
-    // first poll held back as above: between two ranks 1.37 to 1.50 us from 128 B to 64 KiB against
-    // one-shot's 1.30 to 1.56 (ahead from 4 KiB on everywhere, below that on some GPUs); among four
-    // 1.37 to 1.46 us up to 8 KiB against 1.40 to 1.53 (level or ahead); among eight 0.15 us and more
-    // behind everywhere
-    if (P == 2 && bytes <= (64u << 10)) return SYMAR_LL;
-    if (P == 4 && bytes <= (8u << 10)) return SYMAR_LL;
+    // first poll held back as above: between two ranks 1.18 to 1.43 us from 128 B to 128 KiB against
+    // one-shot's 1.37 to 1.62; among four 1.18 to 1.50 us up to 32 KiB against 1.46 to 1.53; among eight
+    // 1.40 against 1.43 us at 128 B, level at 4 KiB, behind elsewhere
+    if (P == 2 && bytes <= kLLSmallMaxBytes) return SYMAR_LL;
+    if (P == 4 && bytes <= (32u << 10)) return SYMAR_LL;
+    if (P == 8 && bytes <= 256) return SYMAR_LL;
     // one-shot reads P times the bytes two-shot does and saves its second synchronisation: the
     // break-even moves up fourfold each time the rank count halves (measured 256 KiB, 1 MiB, 4 to 8 MiB)
     const size_t limit = (size_t)(256u << 10) * (size_t)(64 / (P * P));
