@@ -168,13 +168,13 @@ static int bulk_variant(int stages, int tile_log2_over_4k) { return (stages << 8
 // the store-to-visibility time less what the kernel does anyway between its stores and its first poll.
 // Measured with each slot's ranks launched as a cluster (sweeps at P = 8, 4, 2 from 128 B to 128 KiB; the
 // minimum is sharp: 0.06 to 0.15 us lost one step of 128 cycles beside it): nothing up to 256 B and
-// between two ranks up to 4 KiB, 128 cycles up to 16 KiB (256 among eight ranks in one CTA per rank),
-// then growing with the rows in flight to a full hop (768 cycles).
+// between two ranks up to 4 KiB, 128 cycles up to 16 KiB, then growing with the rows in flight to a full
+// hop (768 cycles).
 constexpr uint64_t kLLSmallMaxBytes = (uint64_t)kLLSlots * kLLMaxThreads * 8;
 static unsigned ll_default_gap(int P, uint64_t bytes)
 {
     if (bytes <= 256) return 0;
-    if (P >= 8) return bytes <= 2048 ? 4 : (bytes <= (16u << 10) ? 2 : (bytes <= (32u << 10) ? 12 : 8));
+    if (P >= 8) return bytes <= (16u << 10) ? 2 : (bytes <= (32u << 10) ? 12 : 8);
     if (P == 4) return bytes <= (16u << 10) ? 2 : (bytes <= (32u << 10) ? 4 : (bytes <= (64u << 10) ? 6 : 8));
     return bytes <= 4096 ? 0 : 2;
 }
@@ -294,7 +294,7 @@ static LaunchCfg default_shape(symheap *h, int algo, uint64_t nvec, KernelFn fn)
         // per thread at every size it covers), first poll held back by the default for this traffic
         c.variant = 0x100 | (ll_default_gap(P, bytes) << 12);
         units     = work * 2;
-        c.threads = units <= 128 ? round_threads(units) : (units < 2048 ? 64 : (units <= 8192 ? 128 : 256));
+        c.threads = units <= 64 ? round_threads(units) : (units < 2048 ? 64 : (units <= 8192 ? 128 : 256));
         c.ctas    = (int)std::min<uint64_t>((units + c.threads - 1) / c.threads, (uint64_t)kLLSlots);
         return c;
     }
