@@ -610,9 +610,16 @@ __device__ __forceinline__ ExchangePtrs exchange_ptrs(const KArgs &a, uint64_t f
 
 // STAMP >= 0 (instrumented instantiations only): phase stamp once this thread's signal is issued,
 // i.e. for a release signal once its fence has completed.
-template <int P, bool RELEASE, int STAMP = -1>
+struct NoHook {
+    __device__ __forceinline__ void operator()(uint32_t) const {}
+};
+
+// `after_count(want)` runs on every thread once the count has been read and the signals are on their way,
+// before the first poll: the place to publish counters whose stores should drain during the wait.
+template <int P, bool RELEASE, int STAMP = -1, typename Hook = NoHook>
 __device__ __forceinline__ bool flag_exchange_at(const KArgs &a, const ExchangePtrs &p, const uint32_t *count, int r,
-                                                 int c, bool silent, bool all_warps, uint32_t &want)
+                                                 int c, bool silent, bool all_warps, uint32_t &want,
+                                                 Hook after_count = Hook())
 {
     const uint32_t t    = threadIdx.x;
     const uint32_t lane = t & 31u;
@@ -622,6 +629,7 @@ __device__ __forceinline__ bool flag_exchange_at(const KArgs &a, const ExchangeP
     }
     if (STAMP >= 0) debug_phase(a, STAMP);
     const uint32_t n = ld_relaxed_u32(count);
+    after_count(n + 1);
     if (!all_warps && t >= 32) {
         want = n + 1;
         return true;
@@ -640,12 +648,13 @@ __device__ __forceinline__ bool flag_exchange_at(const KArgs &a, const ExchangeP
     }
 }
 
-template <int P, bool RELEASE, int STAMP = -1>
+template <int P, bool RELEASE, int STAMP = -1, typename Hook = NoHook>
 __device__ __forceinline__ bool flag_exchange(const KArgs &a, uint64_t flags_off, int pair, const uint32_t *count,
-                                              int r, int c, bool silent, bool all_warps, uint32_t &want)
+                                              int r, int c, bool silent, bool all_warps, uint32_t &want,
+                                              Hook after_count = Hook())
 {
-    return flag_exchange_at<P, RELEASE, STAMP>(a, exchange_ptrs<P>(a, flags_off, pair, r, c), count, r, c, silent,
-                                               all_warps, want);
+    return flag_exchange_at<P, RELEASE, STAMP, Hook>(a, exchange_ptrs<P>(a, flags_off, pair, r, c), count, r, c, silent,
+                                                     all_warps, want, after_count);
 }
 
 // Reduce-scatter + all-gather of one 16-byte vector: P loads, the rank-ordered

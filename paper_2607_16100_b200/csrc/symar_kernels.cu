@@ -246,14 +246,17 @@ __global__ void __launch_bounds__(kMaxThreads) twoshot_kernel(const KArgs a)
     if (DBG) debug_phase(a, 2);               // thread 0's share reduced, its stores issued
     __syncthreads();
     if (DBG) debug_phase(a, 3);               // the whole CTA's stores issued
-    if (DBG) flag_exchange<P, true, 5>(a, a.done_off, kPairDone, dcount, r, c, !ok, false, dwant);   // 5: release fence done, signal sent
-    else flag_exchange<P, true>(a, a.done_off, kPairDone, dcount, r, c, !ok, false, dwant);
+    // Both counts are published once the "done" signals are on their way and before the first poll: their
+    // stores (one copy each on the other half of the L2) drain during the wait instead of after it.  (Not
+    // earlier: before the handoff the release fence would have to wait for them too, measured +0.1 us
+    // between two ranks.)
+    auto publish = [&](uint32_t done_want) {
+        publish_u32(a, r, c, kCtrReady, rwant);
+        publish_u32(a, r, c, kCtrDone, done_want);
+    };
+    if (DBG) flag_exchange<P, true, 5>(a, a.done_off, kPairDone, dcount, r, c, !ok, false, dwant, publish);   // 5: release fence done, signal sent
+    else flag_exchange<P, true>(a, a.done_off, kPairDone, dcount, r, c, !ok, false, dwant, publish);
     if (DBG) debug_phase(a, 4);               // every peer's part has landed here
-    // (Measured and dropped: publishing the ready count before the handoff, as the one-shot kernel does
-    // before its data phase.  The release fence then also waits for that store's far copy: +0.1 us
-    // between two ranks, no gain among eight.)
-    publish_u32(a, r, c, kCtrReady, rwant);
-    publish_u32(a, r, c, kCtrDone, dwant);
     if (DBG) {
         debug_stamp_out(a);
         debug_phase(a, 7);
