@@ -355,6 +355,10 @@ __global__ void __launch_bounds__(kLLMaxThreads) ll_kernel(const KArgs a)
     const uint64_t n0 = ld_relaxed_u64(ep);
     if (DBG) debug_delay(a, r, c);
     if (DBG && a.dbg_mute == r) return;       // test hook: this rank never joins
+    // Every thread has read the counter, and where it will stand after this call is known: publish it now,
+    // so that its stores drain during the call and not after it.
+    __syncthreads();
+    publish_u64(a, r, c, kCtrLL, n0 + a.iters);
     if (DBG) debug_phase(a, 0);
 
     const char *in = seg_r + a.in_off;
@@ -439,8 +443,6 @@ __global__ void __launch_bounds__(kLLMaxThreads) ll_kernel(const KArgs a)
         // thread's send of iteration i, issued after that thread's receive of
         // iteration i-1 -- so the sub-buffer of parity (i+1)&1 is free.
     }
-    __syncthreads();          // every thread has read the counter before it moves
-    publish_u64(a, r, c, kCtrLL, n0 + a.iters);
     if (DBG) {
         debug_stamp_out(a);
         debug_phase(a, 7);
@@ -613,6 +615,10 @@ __global__ void __launch_bounds__(kMaxThreads) sentinel_kernel(const KArgs a)
     const uint64_t n0 = ld_relaxed_u64(ep);
     if (DBG) debug_delay(a, r, c);
     if (DBG && a.dbg_mute == r) return;       // test hook: this rank never joins
+    // Every thread has read the counter, and where it will stand after this call is known: publish it now,
+    // so that its stores drain during the call and not after it.
+    __syncthreads();
+    publish_u64(a, r, c, kCtrLL, n0 + a.iters);
 
     const char *in = seg_r + a.in_off;
     char *out      = seg_r + a.out_off;
@@ -676,8 +682,6 @@ __global__ void __launch_bounds__(kMaxThreads) sentinel_kernel(const KArgs a)
         }
         if (a.iters > 1) fence_acq_rel();
     }
-    __syncthreads();
-    publish_u64(a, r, c, kCtrLL, n0 + a.iters);
     if (DBG) {
         debug_stamp_out(a);
         debug_phase(a, 7);
@@ -767,6 +771,10 @@ __global__ void __launch_bounds__(kPushTwoshotMaxThreads) twoshot_push_kernel(co
     const uint64_t n0 = ld_relaxed_u64(ep);
     if (DBG) debug_delay(a, r, c);
     if (DBG && a.dbg_mute == r) return;       // test hook: this rank never joins
+    // Every thread has read the counter, and where it will stand after this call is known: publish it now,
+    // so that its stores drain during the call and not after it.
+    __syncthreads();
+    publish_u64(a, r, c, kCtrLL, n0 + a.iters);
 
     const char *in = seg_r + a.in_off;
     char *out      = seg_r + a.out_off;
@@ -852,8 +860,6 @@ __global__ void __launch_bounds__(kPushTwoshotMaxThreads) twoshot_push_kernel(co
         }
         if (SENT && a.iters > 1) fence_acq_rel();      // restored sentinels before the sub-buffer's next use
     }
-    __syncthreads();
-    publish_u64(a, r, c, kCtrLL, n0 + a.iters);
     if (DBG) {
         debug_stamp_out(a);
         debug_phase(a, 7);
